@@ -1,0 +1,167 @@
+/*
+ * powerattn.h -- C ABI of the PowerAttention block-sparse attention library for NVIDIA B200
+ * (sm_100a).
+ *
+ * The library computes causal block-sparse attention under the static mask of PowerAttention
+ * (arXiv 2503.03588): every query block attends to the key blocks at power-of-two block
+ * distances, to a local window of recent blocks and to the first ("sink") blocks.
+ *
+ * General conventions
+ *   - Every buffer is owned by the caller.  No entry point allocates or frees device memory
+ *     unless its comment says otherwise; scratch is passed in as `workspace`.
+ *   - "device" pointers are CUDA device pointers valid on the current device; "host" pointers
+ *     are ordinary process memory.  Each argument says which it is.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *     only enqueue work on it; none synchronises unless its comment says so.
+ *   - Tensors are bfloat16 unless stated; strides are in ELEMENTS; the head_dim axis is
+ *     contiguous (stride 1) and every row start must be 16-byte aligned.
+ *   - Grouped-query attention: query head h reads KV head floor(h / (n_q_heads / n_kv_heads)).
+ *   - Failures are returned as a pa_status; nothing aborts and no kernel traps.  Argument
+ *     checks run before any launch.  pa_last_error_message() gives a host-side description of
+ *     the calling thread's most recent failure.
+ */
+#ifndef POWERATTN_H_
+#define POWERATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PA_OK = 0,
+    PA_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, bad enum                    */
+    PA_ERR_SHAPE = 2,       /* unsupported head_dim / block / head grouping / strides       */
+    PA_ERR_ALIGNMENT = 3,   /* a pointer or stride breaks the 16-byte rule                  */
+    PA_ERR_LAYOUT = 4,      /* CSR arrays inconsistent with the problem (capacity, nnz)     */
+    PA_ERR_WORKSPACE = 5,   /* workspace missing or smaller than the *_workspace_bytes size */
+    PA_ERR_UNSUPPORTED = 6, /* the device is not an sm_100 GPU                              */
+    PA_ERR_CUDA = 7,        /* a CUDA runtime / driver call failed                          */
+    PA_ERR_TIMEOUT = 8      /* a bounded device-side wait gave up (see pa_prefill_status)   */
+} pa_status;
+
+const char *pa_status_string(pa_status s);
+/* Host string describing the calling thread's last failing call ("" if none). */
+const char *pa_last_error_message(void);
+/* major * 10000 + minor * 100 + patch */
+int pa_version(void);
+
+/* ------------------------------------------------------------------------------------------
+ * Layout: Algorithm 1 (Section 3.3) evaluated on blocks.
+ *
+ * With equal, aligned query and key blocks of `block` tokens, key block j is listed for query
+ * block i exactly when j <= i and ( i - j < window_blocks  or  (i - j) & (i - j - 1) == 0  or
+ * j < sink_blocks ).  The paper's sink is one block (kv_idx < B); `sink_blocks` generalises it.
+ * Distance 0 passes the power-of-two test, so the diagonal block is always listed and no row
+ * is empty.  n_qblocks = ceil(seq_len / block).  Rows are ascending without duplicates; the
+ * arrays are CSR: row i owns col_idx[row_ptr[i] .. row_ptr[i+1]).
+ * ------------------------------------------------------------------------------------------ */
+
+/* Host-only closed-form sizes.  n_qblocks, nnz: host pointers, written on success.
+ * Errors: PA_ERR_INVALID_ARG (seq_len < 1, block < 1, window/sink < 0, null outputs),
+ * PA_ERR_SHAPE (n_qblocks or nnz would not fit in int32). */
+pa_status pa_layout_size(int64_t seq_len, int32_t block, int32_t window_blocks,
+                         int32_t sink_blocks, int32_t *n_qblocks, int64_t *nnz);
+
+/* Writes the CSR on the device.  row_ptr: device int32[n_qblocks + 1]; col_idx: device
+ * int32[col_capacity], col_capacity >= nnz from pa_layout_size (else PA_ERR_LAYOUT, nothing
+ * launched).  Three small kernels are enqueued on `stream`; no scratch memory is used. */
+pa_status pa_build_layout(int64_t seq_len, int32_t block, int32_t window_blocks,
+                          int32_t sink_blocks, int32_t *row_ptr, int32_t *col_idx,
+                          int64_t col_capacity, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Prefill: Eq. (1) (Section 3.1) over the listed key blocks of each query block.
+ *
+ *   s_kv = softmax_scale * <Q[b,q,h,:], K[b,kv,hk,:]>          for kv in the listed blocks,
+ *   kv <= q inside the diagonal block (Algorithm 1's causal term), kv < seq_len;
+ *   LSE[b,h,q] = ln sum_kv exp(s_kv);   O[b,q,h,:] = sum_kv exp(s_kv - LSE) V[b,kv,hk,:].
+ *
+ * The kernel accepts ANY causal CSR whose rows are ascending, end with the diagonal block
+ * (col == row) and hold only cols <= row: the PowerAttention layout, dense causal, sliding
+ * window.  It applies token-level causality to the diagonal pair and the seq_len bound itself.
+ * Arithmetic: bf16 operands, fp32 accumulation (tensor cores), fp32 softmax; O rounded to
+ * bf16 or kept fp32; LSE fp32.
+ * ------------------------------------------------------------------------------------------ */
+
+typedef enum { PA_BF16 = 0, PA_F32 = 1 } pa_dtype;
+
+/* Element strides of a [batch, seq, head, head_dim] tensor; head_dim stride is 1. */
+typedef struct {
+    int64_t batch, seq, head;
+} pa_strides;
+
+typedef struct {
+    int32_t batch, n_q_heads, n_kv_heads, head_dim; /* head_dim in {64, 128}              */
+    int64_t seq_len;                                /* same for queries and keys          */
+    int32_t block;                                  /* tokens per block; must be 64       */
+    float softmax_scale;                            /* 0 => 1 / sqrt(head_dim)            */
+    pa_strides q, k, v, o;
+    pa_dtype o_dtype;
+} pa_prefill_params;
+
+/* Bytes of device scratch pa_prefill needs (a status block; 16-byte aligned start). */
+size_t pa_prefill_workspace_bytes(const pa_prefill_params *p);
+
+/* q, k, v: device bf16, read-only.  row_ptr [ceil(seq_len/block) + 1], col_idx [nnz]: device
+ * int32 CSR, shared by every batch entry and head (the mask does not depend on them).
+ * o: device, o_dtype, strides p->o.  lse: device fp32 [batch, n_q_heads, seq_len] contiguous.
+ * workspace: device, >= pa_prefill_workspace_bytes(p); cleared by the call itself.
+ * Enqueues one memset and one kernel.  Errors: PA_ERR_INVALID_ARG, PA_ERR_SHAPE,
+ * PA_ERR_ALIGNMENT, PA_ERR_LAYOUT (nnz < n_qblocks), PA_ERR_WORKSPACE, PA_ERR_UNSUPPORTED,
+ * PA_ERR_CUDA.  Outputs are undefined after a failure. */
+pa_status pa_prefill(const pa_prefill_params *p, const void *q, const void *k, const void *v,
+                     const int32_t *row_ptr, const int32_t *col_idx, int64_t nnz, void *o,
+                     float *lse, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Synchronises `stream` and reads back the status block a pa_prefill call left in `workspace`.
+ * Returns PA_OK, PA_ERR_TIMEOUT (a bounded barrier wait inside the kernel ran out; *detail, a
+ * host pointer that may be NULL, receives a code naming the wait) or PA_ERR_CUDA. */
+pa_status pa_prefill_status(const void *workspace, void *stream, int32_t *detail);
+
+/* ------------------------------------------------------------------------------------------
+ * Decode: one query token per sequence against its KV cache (Section 4.1: the same pattern in
+ * prefilling and decoding).  cache_lens[b] counts the cached keys INCLUDING the current token,
+ * so the query sits at position p = cache_lens[b] - 1, attends to itself, and its key blocks
+ * are row floor(p / block) of the layout; the last block holds (p mod block) + 1 keys.
+ * The block list is derived in closed form inside the kernel (no CSR is read).
+ * ------------------------------------------------------------------------------------------ */
+
+typedef struct {
+    int32_t batch, n_q_heads, n_kv_heads, head_dim; /* head_dim in {64, 128}; group <= 8   */
+    int32_t block, window_blocks, sink_blocks;      /* block must be 64                    */
+    int64_t max_len;                                /* cache capacity in tokens            */
+    float softmax_scale;                            /* 0 => 1 / sqrt(head_dim)             */
+    pa_strides k, v;                                /* cache [batch, max_len, n_kv_heads, D] */
+    pa_dtype o_dtype;
+} pa_decode_params;
+
+/* Bytes of device scratch for the split-K partial results (m, l, o[head_dim] per query head
+ * and chunk of the block list). */
+size_t pa_decode_workspace_bytes(const pa_decode_params *p);
+
+/* q: device bf16 [batch, n_q_heads, head_dim] contiguous.  k_cache, v_cache: device bf16 by
+ * strides.  cache_lens: device int32 [batch], each in [1, max_len] (a length outside that
+ * range makes the sequence's outputs zero and its LSE -inf; nothing faults).
+ * o: device [batch, n_q_heads, head_dim] contiguous, o_dtype.  lse: device fp32
+ * [batch, n_q_heads].  Enqueues two kernels: partial attention per (sequence, KV head, chunk),
+ * then the log-sum-exp combine  m = max m_c, l = sum l_c e^(m_c - m), o = sum o_c e^(m_c - m) / l.
+ * Calls that share a workspace must not overlap on the GPU. */
+pa_status pa_decode(const pa_decode_params *p, const void *q, const void *k_cache,
+                    const void *v_cache, const int32_t *cache_lens, void *o, float *lse,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/* The key-block list the decode kernel derives for one cache length, written on the device by
+ * the same device function the kernel uses: out_blocks device int32[capacity], out_count
+ * device int32[1].  Equals row floor((cache_len-1)/block) of pa_build_layout(cache_len, ...).
+ * capacity >= 64 + window_blocks + sink_blocks is always enough. */
+pa_status pa_decode_block_list(int64_t cache_len, int32_t block, int32_t window_blocks,
+                               int32_t sink_blocks, int32_t *out_blocks, int32_t *out_count,
+                               int32_t capacity, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* POWERATTN_H_ */

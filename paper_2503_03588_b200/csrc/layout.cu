@@ -1,0 +1,109 @@
+// pa_layout_size / pa_build_layout: the block-sparse CSR of Algorithm 1 (Section 3.3).
+#include "common.cuh"
+#include "layout_rule.cuh"
+
+namespace pa {
+
+__global__ void layout_count_kernel(int32_t nqb, int32_t W, int32_t S, int32_t *row_ptr)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i == 0) row_ptr[0] = 0;
+    if (i < nqb) row_ptr[i + 1] = row_length(i, W, S);
+}
+
+// In-place inclusive scan of row_ptr[1 .. nqb] by one block, tile by tile with a running carry.
+__global__ void layout_scan_kernel(int32_t nqb, int32_t *row_ptr)
+{
+    __shared__ int32_t warp_sums[32];
+    __shared__ int32_t carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) carry_s = 0;
+    __syncthreads();
+    for (int64_t base = 0; base < nqb; base += blockDim.x) {
+        const int64_t idx = base + tid;
+        int32_t v = idx < nqb ? row_ptr[idx + 1] : 0;
+        for (int o = 1; o < 32; o <<= 1) {
+            int32_t t = __shfl_up_sync(0xffffffffu, v, o);
+            if (lane >= o) v += t;
+        }
+        if (lane == 31) warp_sums[warp] = v;
+        __syncthreads();
+        if (warp == 0) {
+            int32_t s = lane < (int)(blockDim.x >> 5) ? warp_sums[lane] : 0;
+            for (int o = 1; o < 32; o <<= 1) {
+                int32_t t = __shfl_up_sync(0xffffffffu, s, o);
+                if (lane >= o) s += t;
+            }
+            warp_sums[lane] = s;
+        }
+        __syncthreads();
+        const int32_t carry = carry_s;
+        const int32_t before = warp > 0 ? warp_sums[warp - 1] : 0;
+        if (idx < nqb) row_ptr[idx + 1] = carry + before + v;
+        __syncthreads();
+        if (tid == (int)blockDim.x - 1) carry_s = carry + before + v;
+        __syncthreads();
+    }
+}
+
+struct StoreCols {
+    int32_t *out;
+    __device__ void operator()(int pos, int64_t j) const { out[pos] = (int32_t)j; }
+};
+
+__global__ void layout_fill_kernel(int32_t nqb, int32_t W, int32_t S, const int32_t *row_ptr,
+                                   int32_t *col_idx)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nqb) return;
+    for_each_key_block(i, W, S, StoreCols{col_idx + row_ptr[i]});
+}
+
+static pa_status check_layout_args(int64_t seq_len, int32_t block, int32_t W, int32_t S)
+{
+    if (seq_len < 1) return fail(PA_ERR_INVALID_ARG, "seq_len must be >= 1 (got %lld)", (long long)seq_len);
+    if (block < 1) return fail(PA_ERR_INVALID_ARG, "block must be >= 1 (got %d)", block);
+    if (W < 0 || S < 0) return fail(PA_ERR_INVALID_ARG, "window_blocks and sink_blocks must be >= 0");
+    return PA_OK;
+}
+
+}  // namespace pa
+
+extern "C" pa_status pa_layout_size(int64_t seq_len, int32_t block, int32_t window_blocks,
+                                    int32_t sink_blocks, int32_t *n_qblocks, int64_t *nnz)
+{
+    using namespace pa;
+    clear_error();
+    if (pa_status s = check_layout_args(seq_len, block, window_blocks, sink_blocks)) return s;
+    if (!n_qblocks || !nnz) return fail(PA_ERR_INVALID_ARG, "n_qblocks and nnz must be non-null");
+    const int64_t nqb = (seq_len + block - 1) / block;
+    if (nqb >= INT32_MAX) return fail(PA_ERR_SHAPE, "n_qblocks %lld does not fit in int32", (long long)nqb);
+    int64_t total = 0;
+    for (int64_t i = 0; i < nqb; ++i) total += row_length(i, window_blocks, sink_blocks);
+    if (total > INT32_MAX) return fail(PA_ERR_SHAPE, "nnz %lld does not fit in int32", (long long)total);
+    *n_qblocks = (int32_t)nqb;
+    *nnz = total;
+    return PA_OK;
+}
+
+extern "C" pa_status pa_build_layout(int64_t seq_len, int32_t block, int32_t window_blocks,
+                                     int32_t sink_blocks, int32_t *row_ptr, int32_t *col_idx,
+                                     int64_t col_capacity, void *stream)
+{
+    using namespace pa;
+    clear_error();
+    int32_t nqb = 0;
+    int64_t nnz = 0;
+    if (pa_status s = pa_layout_size(seq_len, block, window_blocks, sink_blocks, &nqb, &nnz)) return s;
+    if (!row_ptr || !col_idx) return fail(PA_ERR_INVALID_ARG, "row_ptr and col_idx must be non-null");
+    if (col_capacity < nnz)
+        return fail(PA_ERR_LAYOUT, "col_capacity %lld < nnz %lld", (long long)col_capacity, (long long)nnz);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int threads = 256;
+    const unsigned blocks = (unsigned)((nqb + threads - 1) / threads);
+    layout_count_kernel<<<blocks, threads, 0, st>>>(nqb, window_blocks, sink_blocks, row_ptr);
+    layout_scan_kernel<<<1, 1024, 0, st>>>(nqb, row_ptr);
+    layout_fill_kernel<<<blocks, threads, 0, st>>>(nqb, window_blocks, sink_blocks, row_ptr, col_idx);
+    PA_CUDA_OK(cudaGetLastError());
+    return PA_OK;
+}

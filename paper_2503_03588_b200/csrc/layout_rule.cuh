@@ -1,0 +1,55 @@
+// Algorithm 1 (Section 3.3) on block indices: the ascending list of key blocks of one query
+// block.  With equal, aligned query and key blocks the window and power-of-two terms depend on
+// the block distance d = i - j only, the sink term on j, and causality on j <= i.  The listed
+// set is the union of three ascending runs, merged here without duplicates:
+//   sink    j = 0 .. min(S, i+1) - 1
+//   power   j = i - 2^k for every 2^k <= i, k descending   (d = 0 is covered by the window run)
+//   window  j = max(0, i - max(W,1) + 1) .. i              (d = 0 always passes: 0 & -1 == 0)
+#pragma once
+
+#include <stdint.h>
+
+namespace pa {
+
+// Calls emit(pos, j) for every listed key block j of query block i in ascending order and
+// returns the row length.  i >= 0, W >= 0, S >= 0.
+template <typename Emit>
+__host__ __device__ inline int for_each_key_block(int64_t i, int32_t W, int32_t S, Emit emit)
+{
+    const int64_t w_eff = W > 1 ? W : 1;
+    const int64_t sink_end = (int64_t)S < i + 1 ? (int64_t)S : i + 1;  // sink run [0, sink_end)
+    int64_t js = 0;                                                    // sink cursor
+    int64_t jw = i - w_eff + 1 > 0 ? i - w_eff + 1 : 0;                // window cursor .. i
+    int64_t pw = 0;                                                    // current power distance
+    if (i >= 1) {
+        pw = 1;
+        while (pw * 2 <= i) pw *= 2;                                   // largest 2^k <= i
+    }
+    const int64_t kNone = INT64_MAX;
+    int n = 0;
+    while (true) {
+        const int64_t a = js < sink_end ? js : kNone;
+        const int64_t b = pw >= 1 ? i - pw : kNone;
+        const int64_t c = jw <= i ? jw : kNone;
+        int64_t j = a < b ? a : b;
+        j = j < c ? j : c;
+        if (j == kNone) break;
+        emit(n, j);
+        ++n;
+        if (a == j) ++js;
+        if (b == j) pw >>= 1;  // 2^k -> 2^(k-1) -> ... -> 1 -> 0 (exhausted)
+        if (c == j) ++jw;
+    }
+    return n;
+}
+
+struct NoEmit {
+    __host__ __device__ void operator()(int, int64_t) const {}
+};
+
+__host__ __device__ inline int row_length(int64_t i, int32_t W, int32_t S)
+{
+    return for_each_key_block(i, W, S, NoEmit());
+}
+
+}  // namespace pa
