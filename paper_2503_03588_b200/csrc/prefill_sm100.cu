@@ -1,0 +1,571 @@
+// pa_prefill: block-sparse causal attention forward (Eq. (1), Section 3.1) over the CSR
+// key-block lists of Algorithm 1 (Section 3.3), for sm_100a.
+//
+// One persistent CTA per SM walks work units (batch, KV head, query block, head quad).  A unit
+// holds two 128-row tiles ("slots"); a tile stacks two query heads of the KV group on the 64
+// tokens of the query block (the mask does not depend on the head, so they share the key list
+// and the K/V tiles).  Warp roles:
+//   warp 0      TMA producer: Q tiles once per unit, then the listed K/V blocks, gathered by block
+//               index, into a ring of shared-memory stages (128-byte swizzle)
+//   warp 1      tcgen05 issuer: S = Q K^T into tensor memory, later O += P V
+//   warp 2      tensor-memory allocation
+//   warps 4-7   online softmax of slot 0 (thread = tile row = TMEM lane)
+//   warps 8-11  online softmax of slot 1
+// The two slots alternate on the tensor pipe, so one slot's softmax overlaps the other's MMAs.
+// Every barrier wait is bounded; a wait that runs out records PA_ERR_TIMEOUT in the status
+// block, raises a CTA-wide abort flag and the CTA drains and exits (no trap, no endless spin).
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace pa {
+
+constexpr int kBlk = 64;               // tokens per query / key block
+constexpr int kThreads = 384;          // 12 warps
+constexpr int kStages = 4;             // K/V ring depth
+constexpr uint32_t kTmemCols = 512;    // S0 S1 (64 cols each) at 0, O0 O1 (D cols each) at 128
+constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
+
+struct PrefillArgs {
+    const int32_t *row_ptr, *col_idx;
+    void *o;
+    float *lse;
+    int32_t *status;  // [0] error code, [1] detail
+    int64_t o_sb, o_ss, o_sh;
+    int64_t N, n_units;
+    int32_t nqb, batch, Hq, Hkv, G, nsub, o_is_f32;
+    float scale_log2;
+};
+
+template <int D>
+struct SmemMap {
+    static constexpr uint32_t kQSub = 128 * 128;              // 128 rows x 64 features (128 B)
+    static constexpr uint32_t kQSlot = kQSub * (D / 64);
+    static constexpr uint32_t kQ = 0;
+    static constexpr uint32_t kPSlot = 128 * 128;             // 128 rows x 64 keys bf16
+    static constexpr uint32_t kP = kQ + 2 * kQSlot;
+    static constexpr uint32_t kKVSub = 64 * 128;              // 64 keys x 64 features
+    static constexpr uint32_t kKTile = kKVSub * (D / 64);
+    static constexpr uint32_t kStage = 2 * kKTile;            // K then V
+    static constexpr uint32_t kKV = kP + 2 * kPSlot;
+    static constexpr uint32_t kBars = kKV + kStages * kStage;
+    static constexpr uint32_t kTotal = kBars + 256;
+    static constexpr uint32_t kAlloc = kTotal + 1024;         // slack for 1024-byte alignment
+};
+
+// Barrier slots inside the barrier area (8 bytes each).
+enum : uint32_t {
+    BAR_Q_FULL = 0, BAR_Q_EMPTY = 1, BAR_KV_FULL = 2, BAR_KV_EMPTY = 2 + kStages,
+    BAR_S_FULL = 2 + 2 * kStages, BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2,
+    BAR_COUNT = BAR_O_DONE + 2
+};
+
+struct Unit {
+    int32_t b, hk, i, sub, rs, n;
+};
+
+__device__ __forceinline__ Unit decode_unit(const PrefillArgs &a, int64_t u)
+{
+    Unit r;
+    r.sub = (int32_t)(u % a.nsub);
+    u /= a.nsub;
+    r.hk = (int32_t)(u % a.Hkv);
+    u /= a.Hkv;
+    r.i = a.nqb - 1 - (int32_t)(u % a.nqb);  // long rows first
+    r.b = (int32_t)(u / a.nqb);
+    r.rs = __ldg(a.row_ptr + r.i);
+    r.n = __ldg(a.row_ptr + r.i + 1) - r.rs;
+    return r;
+}
+
+// Bounded mbarrier wait.  Returns false after a timeout (recorded once) or once another thread
+// of the CTA has raised the abort flag.
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                         int32_t *status, int code)
+{
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t it = 0;
+    while (true) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((++it & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitCycles) break;
+        }
+    }
+    if (atomicCAS(status, 0, (int)PA_ERR_TIMEOUT) == 0) status[1] = code;
+    *abort_flag = 1;
+    __threadfence_block();
+    return false;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+               const __grid_constant__ CUtensorMap tmV, const PrefillArgs a)
+{
+    using SM = SmemMap<D>;
+    constexpr int DH = D / 64;  // 64-feature (128-byte) sub-tiles per row
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+    const uint32_t bars = smem_base + SM::kBars;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + SM::kBars + BAR_COUNT * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::kBars + BAR_COUNT * 8 + 8);
+    auto bar = [&](uint32_t idx) { return bars + idx * 8u; };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(bar(BAR_Q_FULL), 1);
+        ptx::mbar_init(bar(BAR_Q_EMPTY), 1);
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(bar(BAR_KV_FULL + s), 1);
+            ptx::mbar_init(bar(BAR_KV_EMPTY + s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            ptx::mbar_init(bar(BAR_S_FULL + s), 1);
+            ptx::mbar_init(bar(BAR_P_FULL + s), 128);
+            ptx::mbar_init(bar(BAR_O_DONE + s), 1);
+        }
+        *abort_flag = 0;
+        ptx::fence_barrier_init();
+        ptx::fence_proxy_async_smem();
+    }
+    if (warp == 2) {
+        ptx::tmem_alloc(ptx::smem_u32(tmem_slot), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            ptx::prefetch_tensormap(&tmQ);
+            ptx::prefetch_tensormap(&tmK);
+            ptx::prefetch_tensormap(&tmV);
+            uint32_t kvc = 0, ul = 0;
+            bool ok = true;
+            for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
+                const Unit w = decode_unit(a, u);
+                if (w.n <= 0) continue;
+                if (ul > 0) ok = wait_bar(bar(BAR_Q_EMPTY), (ul - 1) & 1, abort_flag, a.status, 1);
+                if (!ok) break;
+                ptx::mbar_expect_tx(bar(BAR_Q_FULL), 2 * SM::kQSlot);
+                for (int s = 0; s < 2; ++s)
+                    for (int dh = 0; dh < DH; ++dh)
+                        ptx::tma_load_4d(smem_base + SM::kQ + s * SM::kQSlot + dh * SM::kQSub, &tmQ,
+                                         bar(BAR_Q_FULL), dh * 64, w.i * kBlk,
+                                         w.hk * a.G + w.sub * 4 + 2 * s, w.b);
+                for (int t = 0; t < w.n; ++t, ++kvc) {
+                    const int32_t j = __ldg(a.col_idx + w.rs + t);
+                    const uint32_t st = kvc % kStages;
+                    if (kvc >= (uint32_t)kStages) {
+                        ok = wait_bar(bar(BAR_KV_EMPTY + st), (kvc / kStages - 1) & 1, abort_flag,
+                                      a.status, 2);
+                        if (!ok) break;
+                    }
+                    const uint32_t dst = smem_base + SM::kKV + st * SM::kStage;
+                    ptx::mbar_expect_tx(bar(BAR_KV_FULL + st), SM::kStage);
+                    for (int dh = 0; dh < DH; ++dh)
+                        ptx::tma_load_4d(dst + dh * SM::kKVSub, &tmK, bar(BAR_KV_FULL + st), dh * 64,
+                                         j * kBlk, w.hk, w.b);
+                    for (int dh = 0; dh < DH; ++dh)
+                        ptx::tma_load_4d(dst + SM::kKTile + dh * SM::kKVSub, &tmV,
+                                         bar(BAR_KV_FULL + st), dh * 64, j * kBlk, w.hk, w.b);
+                }
+                ++ul;
+            }
+            if (!ok) {
+                // Drain: give copies already in flight a bounded chance to land before exit.
+                const uint32_t first = kvc > (uint32_t)kStages ? kvc - kStages : 0;
+                for (uint32_t c = first; c < kvc; ++c) {
+                    const long long t0 = clock64();
+                    while (!ptx::mbar_try_wait(bar(BAR_KV_FULL + c % kStages), (c / kStages) & 1) &&
+                           clock64() - t0 < 2000000ll) {
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ tcgen05 issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = ptx::idesc_bf16_f32(128, 64, 0);
+            constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(128, D, 1);
+            // S_s = Q_s K^T: A = Q tile (K-major), B = K block (K-major), 16 features per MMA.
+            auto issue_qk = [&](int s, uint32_t st) {
+                const uint32_t qa = smem_base + SM::kQ + s * SM::kQSlot;
+                const uint32_t kb = smem_base + SM::kKV + st * SM::kStage;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint64_t ad = ptx::smem_desc_sw128(qa + (kk / 4) * SM::kQSub + (kk % 4) * 32, 16, 1024);
+                    const uint64_t bd = ptx::smem_desc_sw128(kb + (kk / 4) * SM::kKVSub + (kk % 4) * 32, 16, 1024);
+                    ptx::umma_ss(tmem_base + s * 64, ad, bd, idesc_qk, kk > 0);
+                }
+            };
+            // O_s (+)= P_s V: A = P tile (K-major over keys), B = V block (MN-major: features
+            // contiguous), 16 keys per MMA.
+            auto issue_pv = [&](int s, uint32_t st, bool acc) {
+                const uint32_t pa_ = smem_base + SM::kP + s * SM::kPSlot;
+                const uint32_t vb = smem_base + SM::kKV + st * SM::kStage + SM::kKTile;
+#pragma unroll
+                for (int kk = 0; kk < kBlk / 16; ++kk) {
+                    const uint64_t ad = ptx::smem_desc_sw128(pa_ + kk * 32, 16, 1024);
+                    const uint64_t bd = ptx::smem_desc_sw128(vb + kk * 2048, SM::kKVSub, 1024);
+                    ptx::umma_ss(tmem_base + 128 + s * D, ad, bd, idesc_pv, (acc || kk > 0) ? 1u : 0u);
+                }
+            };
+            uint32_t kvc = 0, ul = 0, g = 0;
+            bool ok = true;
+            for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
+                const Unit w = decode_unit(a, u);
+                if (w.n <= 0) continue;
+                ok = wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 3);
+                if (!ok) break;
+                ok = wait_bar(bar(BAR_KV_FULL + kvc % kStages), (kvc / kStages) & 1, abort_flag, a.status, 4);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                for (int s = 0; s < 2; ++s) {
+                    issue_qk(s, kvc % kStages);
+                    ptx::umma_commit(bar(BAR_S_FULL + s));
+                }
+                if (w.n == 1) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                for (int t = 0; t < w.n && ok; ++t) {
+                    const uint32_t st = (kvc + t) % kStages;
+                    for (int s = 0; s < 2; ++s) {
+                        ok = wait_bar(bar(BAR_P_FULL + s), (g + t) & 1, abort_flag, a.status, 5);
+                        if (!ok) break;
+                        ptx::tc_fence_after_sync();
+                        issue_pv(s, st, t > 0);
+                        ptx::umma_commit(bar(BAR_O_DONE + s));
+                        if (s == 1) ptx::umma_commit(bar(BAR_KV_EMPTY + st));
+                        if (t + 1 < w.n) {
+                            const uint32_t c1 = kvc + t + 1;
+                            if (s == 0) {
+                                ok = wait_bar(bar(BAR_KV_FULL + c1 % kStages), (c1 / kStages) & 1,
+                                              abort_flag, a.status, 6);
+                                if (!ok) break;
+                                ptx::tc_fence_after_sync();
+                            }
+                            issue_qk(s, c1 % kStages);
+                            ptx::umma_commit(bar(BAR_S_FULL + s));
+                            if (s == 1 && t + 2 == w.n) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                        }
+                    }
+                }
+                kvc += w.n;
+                g += w.n;
+                ++ul;
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------------ online softmax
+        const int s = (warp - 4) >> 2;          // slot
+        const int quad = warp & 3;              // TMEM lane quadrant this warp may access
+        const int row = quad * 32 + lane;       // tile row = TMEM lane
+        const int qrow = row & 63;              // token inside the query block
+        const uint32_t t_s = tmem_base + ((uint32_t)(quad * 32) << 16) + s * 64;
+        const uint32_t t_o = tmem_base + ((uint32_t)(quad * 32) << 16) + 128 + s * D;
+        uint8_t *p_row = smem + SM::kP + s * SM::kPSlot + row * 128;
+        const float sl2 = a.scale_log2;
+        uint32_t g = 0;
+        bool ok = true;
+        for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
+            const Unit w = decode_unit(a, u);
+            const int head_local = w.sub * 4 + 2 * s + (row >> 6);
+            const int head = w.hk * a.G + head_local;
+            const int64_t tok = (int64_t)w.i * kBlk + qrow;
+            const bool valid = head_local < a.G && tok < a.N;
+            float m = -INFINITY, l = 0.f;
+            for (int t = 0; t < w.n; ++t, ++g) {
+                const int32_t j = __ldg(a.col_idx + w.rs + t);
+                ok = wait_bar(bar(BAR_S_FULL + s), g & 1, abort_flag, a.status, 7);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                uint32_t sr[64];
+                ptx::tmem_ld32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+                ptx::tmem_ld32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+                ptx::tmem_wait_ld();
+                // Algorithm 1's causal term acts inside the diagonal pair only.
+                if (j == w.i) {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c)
+                        if (c > qrow) sr[c] = 0xff800000u;  // -inf
+                }
+                float mx = __uint_as_float(sr[0]);
+#pragma unroll
+                for (int c = 1; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
+                const float m_new = fmaxf(m, mx * sl2);
+                const float alpha = ptx::ex2(m - m_new);
+                float sum = 0.f;
+                uint32_t pk[32];
+#pragma unroll
+                for (int c = 0; c < 64; c += 2) {
+                    const float p0 = ptx::ex2(fmaf(__uint_as_float(sr[c]), sl2, -m_new));
+                    const float p1 = ptx::ex2(fmaf(__uint_as_float(sr[c + 1]), sl2, -m_new));
+                    sum += p0 + p1;
+                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+                    pk[c >> 1] = *reinterpret_cast<const uint32_t *>(&h2);
+                }
+                l = l * alpha + sum;
+                m = m_new;
+                if (t > 0) {
+                    // P_s and O_s are free once the previous step's P V has completed.
+                    ok = wait_bar(bar(BAR_O_DONE + s), (g - 1) & 1, abort_flag, a.status, 8);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    if (__any_sync(0xffffffffu, alpha != 1.0f)) {
+#pragma unroll
+                        for (int ch = 0; ch < D / 32; ++ch) {
+                            uint32_t orr[32];
+                            ptx::tmem_ld32(t_o + ch * 32, orr);
+                            ptx::tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                            ptx::tmem_st32(t_o + ch * 32, orr);
+                        }
+                        ptx::tmem_wait_st();
+                    }
+                }
+                // P row: 64 bf16 = eight 16-byte chunks, chunk c stored at c ^ (row % 8).
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    *reinterpret_cast<uint4 *>(p_row + ((c ^ (row & 7)) << 4)) =
+                        make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                ptx::fence_proxy_async_smem();
+                ptx::tc_fence_before_sync();
+                ptx::mbar_arrive(bar(BAR_P_FULL + s));
+            }
+            if (!ok) break;
+            if (w.n <= 0) {  // empty row: defined outputs, no barrier traffic
+                if (valid) {
+                    for (int c = 0; c < D; ++c) {
+                        const int64_t oi = w.b * a.o_sb + tok * a.o_ss + head * a.o_sh + c;
+                        if (a.o_is_f32) reinterpret_cast<float *>(a.o)[oi] = 0.f;
+                        else reinterpret_cast<__nv_bfloat16 *>(a.o)[oi] = __float2bfloat16_rn(0.f);
+                    }
+                    a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = -INFINITY;
+                }
+                continue;
+            }
+            // Epilogue: O / l and LSE = ln sum exp(s) = (m + log2 l) ln 2.
+            ok = wait_bar(bar(BAR_O_DONE + s), (g - 1) & 1, abort_flag, a.status, 9);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            const float inv = 1.0f / l;
+            const int64_t obase = w.b * a.o_sb + tok * a.o_ss + (int64_t)head * a.o_sh;
+#pragma unroll
+            for (int ch = 0; ch < D / 32; ++ch) {
+                uint32_t orr[32];
+                ptx::tmem_ld32(t_o + ch * 32, orr);
+                ptx::tmem_wait_ld();
+                if (valid) {
+                    if (a.o_is_f32) {
+                        float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(a.o) + obase + ch * 32);
+#pragma unroll
+                        for (int c = 0; c < 8; ++c)
+                            dst[c] = make_float4(__uint_as_float(orr[4 * c]) * inv, __uint_as_float(orr[4 * c + 1]) * inv,
+                                                 __uint_as_float(orr[4 * c + 2]) * inv, __uint_as_float(orr[4 * c + 3]) * inv);
+                    } else {
+                        uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(a.o) + obase + ch * 32);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t h[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const __nv_bfloat162 h2 = __floats2bfloat162_rn(
+                                    __uint_as_float(orr[8 * c + 2 * e]) * inv, __uint_as_float(orr[8 * c + 2 * e + 1]) * inv);
+                                h[e] = *reinterpret_cast<const uint32_t *>(&h2);
+                            }
+                            dst[c] = make_uint4(h[0], h[1], h[2], h[3]);
+                        }
+                    }
+                }
+            }
+            if (valid) a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = (m + log2f(l)) * 0.6931471805599453f;
+            ptx::tc_fence_before_sync();
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 2) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ---------------------------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static pa_status get_encode_fn(EncodeTiledFn *out)
+{
+    static EncodeTiledFn cached = nullptr;
+    if (!cached) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        PA_CUDA_OK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+        if (qres != cudaDriverEntryPointSuccess || !fn)
+            return fail(PA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+        cached = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    *out = cached;
+    return PA_OK;
+}
+
+// Tensor map over a bf16 [batch, seq, head, D] tensor with dimensions ordered
+// (feature, token, head, batch) so that a box of `box_heads` heads x 64 tokens x 64 features
+// lands in shared memory as rows head * 64 + token of 128 bytes each (128-byte swizzle).
+static pa_status make_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int D, int64_t N,
+                          int heads, int batch, const pa_strides &s, int box_heads, const char *what)
+{
+    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)heads, (cuuint64_t)batch};
+    const cuuint64_t strides[3] = {(cuuint64_t)s.seq * 2, (cuuint64_t)s.head * 2,
+                                   (cuuint64_t)(s.batch > 0 ? s.batch : s.seq * N) * 2};
+    const cuuint32_t box[4] = {64, 64, (cuuint32_t)box_heads, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims,
+                           strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(PA_ERR_CUDA, "cuTensorMapEncodeTiled failed for %s (CUresult %d)", what, (int)r);
+    return PA_OK;
+}
+
+static pa_status check_strides(const pa_strides &s, int D, const char *what)
+{
+    if (s.seq < D || s.head < D || s.batch < 0)
+        return fail(PA_ERR_SHAPE, "%s strides must be >= head_dim", what);
+    if ((s.seq % 8) || (s.head % 8) || (s.batch % 8))
+        return fail(PA_ERR_ALIGNMENT, "%s strides must be multiples of 8 elements (16 bytes)", what);
+    if (s.seq >= ((int64_t)1 << 38) || s.head >= ((int64_t)1 << 38) || s.batch >= ((int64_t)1 << 38))
+        return fail(PA_ERR_SHAPE, "%s strides too large for a tensor map", what);
+    return PA_OK;
+}
+
+static pa_status check_prefill(const pa_prefill_params *p)
+{
+    if (!p) return fail(PA_ERR_INVALID_ARG, "params must be non-null");
+    if (p->batch < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->seq_len < 1)
+        return fail(PA_ERR_INVALID_ARG, "batch, head counts and seq_len must be positive");
+    if (p->o_dtype != PA_BF16 && p->o_dtype != PA_F32) return fail(PA_ERR_INVALID_ARG, "bad o_dtype");
+    if (!(p->softmax_scale >= 0.f) || isinf(p->softmax_scale))
+        return fail(PA_ERR_INVALID_ARG, "softmax_scale must be finite and >= 0 (0 = default)");
+    if (p->head_dim != 64 && p->head_dim != 128) return fail(PA_ERR_SHAPE, "head_dim must be 64 or 128");
+    if (p->block != kBlk) return fail(PA_ERR_SHAPE, "block must be 64");
+    if (p->n_q_heads % p->n_kv_heads) return fail(PA_ERR_SHAPE, "n_q_heads must be a multiple of n_kv_heads");
+    if (p->n_q_heads < 2) return fail(PA_ERR_SHAPE, "n_q_heads must be >= 2");
+    if (p->seq_len > ((int64_t)1 << 30)) return fail(PA_ERR_SHAPE, "seq_len too large");
+    if (pa_status s = check_strides(p->q, p->head_dim, "q")) return s;
+    if (pa_status s = check_strides(p->k, p->head_dim, "k")) return s;
+    if (pa_status s = check_strides(p->v, p->head_dim, "v")) return s;
+    if (pa_status s = check_strides(p->o, p->head_dim, "o")) return s;
+    return PA_OK;
+}
+
+constexpr size_t kPrefillWorkspace = 256;
+
+}  // namespace pa
+
+extern "C" size_t pa_prefill_workspace_bytes(const pa_prefill_params *p)
+{
+    (void)p;
+    return pa::kPrefillWorkspace;
+}
+
+extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const void *k,
+                                const void *v, const int32_t *row_ptr, const int32_t *col_idx,
+                                int64_t nnz, void *o, float *lse, void *workspace,
+                                size_t workspace_bytes, void *stream)
+{
+    using namespace pa;
+    clear_error();
+    if (pa_status s = check_prefill(p)) return s;
+    if (!q || !k || !v || !row_ptr || !col_idx || !o || !lse)
+        return fail(PA_ERR_INVALID_ARG, "q, k, v, row_ptr, col_idx, o and lse must be non-null");
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o))
+        return fail(PA_ERR_ALIGNMENT, "q, k, v and o must be 16-byte aligned");
+    const int64_t nqb = (p->seq_len + kBlk - 1) / kBlk;
+    if (nnz < nqb)
+        return fail(PA_ERR_LAYOUT, "nnz %lld < n_qblocks %lld: every row lists its diagonal block",
+                    (long long)nnz, (long long)nqb);
+    if (!workspace || workspace_bytes < kPrefillWorkspace)
+        return fail(PA_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", kPrefillWorkspace, workspace_bytes);
+    if (!aligned16(workspace)) return fail(PA_ERR_ALIGNMENT, "workspace must be 16-byte aligned");
+    if (pa_status s = require_sm100()) return s;
+
+    EncodeTiledFn enc = nullptr;
+    if (pa_status s = get_encode_fn(&enc)) return s;
+    CUtensorMap tmQ, tmK, tmV;
+    const int D = p->head_dim;
+    if (pa_status s = make_map(enc, &tmQ, q, D, p->seq_len, p->n_q_heads, p->batch, p->q, 2, "q")) return s;
+    if (pa_status s = make_map(enc, &tmK, k, D, p->seq_len, p->n_kv_heads, p->batch, p->k, 1, "k")) return s;
+    if (pa_status s = make_map(enc, &tmV, v, D, p->seq_len, p->n_kv_heads, p->batch, p->v, 1, "v")) return s;
+
+    PrefillArgs a;
+    a.row_ptr = row_ptr;
+    a.col_idx = col_idx;
+    a.o = o;
+    a.lse = lse;
+    a.status = static_cast<int32_t *>(workspace);
+    a.o_sb = p->o.batch; a.o_ss = p->o.seq; a.o_sh = p->o.head;
+    a.N = p->seq_len;
+    a.nqb = (int32_t)nqb;
+    a.batch = p->batch; a.Hq = p->n_q_heads; a.Hkv = p->n_kv_heads;
+    a.G = p->n_q_heads / p->n_kv_heads;
+    a.nsub = (a.G + 3) / 4;
+    a.n_units = (int64_t)p->batch * nqb * a.Hkv * a.nsub;
+    a.o_is_f32 = p->o_dtype == PA_F32;
+    const float scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.0f / sqrtf((float)D);
+    a.scale_log2 = scale * 1.4426950408889634f;
+
+    int dev = 0, sms = 0;
+    PA_CUDA_OK(cudaGetDevice(&dev));
+    PA_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const unsigned grid = (unsigned)(a.n_units < sms ? a.n_units : sms);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PA_CUDA_OK(cudaMemsetAsync(workspace, 0, kPrefillWorkspace, st));
+    if (D == 128) {
+        PA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)SmemMap<128>::kAlloc));
+        prefill_kernel<128><<<grid, kThreads, SmemMap<128>::kAlloc, st>>>(tmQ, tmK, tmV, a);
+    } else {
+        PA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)SmemMap<64>::kAlloc));
+        prefill_kernel<64><<<grid, kThreads, SmemMap<64>::kAlloc, st>>>(tmQ, tmK, tmV, a);
+    }
+    PA_CUDA_OK(cudaGetLastError());
+    return PA_OK;
+}
+
+extern "C" pa_status pa_prefill_status(const void *workspace, void *stream, int32_t *detail)
+{
+    using namespace pa;
+    clear_error();
+    if (!workspace) return fail(PA_ERR_INVALID_ARG, "workspace must be non-null");
+    int32_t host[2] = {0, 0};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PA_CUDA_OK(cudaMemcpyAsync(host, workspace, sizeof host, cudaMemcpyDeviceToHost, st));
+    PA_CUDA_OK(cudaStreamSynchronize(st));
+    if (detail) *detail = host[1];
+    if (host[0] == (int32_t)PA_ERR_TIMEOUT)
+        return fail(PA_ERR_TIMEOUT, "a bounded wait inside the prefill kernel ran out (wait id %d)", host[1]);
+    if (host[0] != 0) return fail(PA_ERR_CUDA, "unexpected device status %d", host[0]);
+    return PA_OK;
+}

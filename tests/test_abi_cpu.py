@@ -1,0 +1,105 @@
+"""CPU-side checks of the C ABI: the library loads without a GPU, exports every declared symbol,
+and its host logic (closed-form layout sizes, argument validation) behaves as the header says."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def pa():
+    from paper_2503_03588_b200 import build as _build
+
+    _build.build()
+    import paper_2503_03588_b200.binding as binding
+
+    return binding
+
+
+def test_every_declared_symbol_is_exported(pa):
+    header = open(os.path.join(ROOT, "include", "powerattn.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(pa_[a-z_0-9]+)\s*\(", header))
+    assert declared, "no declarations parsed"
+    assert declared == set(pa.EXPORTS)
+    for name in declared:
+        assert hasattr(pa.lib, name), name
+
+
+def test_status_strings_and_version(pa):
+    assert pa.pa_version() >= 100
+    for code, name in enumerate(pa.STATUS_NAMES):
+        assert pa.pa_status_string(code) == name
+
+
+def test_layout_size_matches_oracle(pa, oracle):
+    for N in (1, 63, 64, 65, 2048, 4096 + 17, 32768):
+        for W in (0, 1, 5, 9):
+            for S in (0, 1, 3):
+                nqb, nnz = pa.pa_layout_size(N, 64, W, S)
+                rp, ci = oracle.block_layout(N, 64, W, S)
+                assert nqb == len(rp) - 1 and nnz == int(rp[-1]) == len(ci), (N, W, S)
+    # the paper's 256-token blocks and other block sizes
+    for B in (4, 256):
+        nqb, nnz = pa.pa_layout_size(32768, B, 5, 1)
+        rp, _ = oracle.block_layout(32768, B, 5, 1)
+        assert (nqb, nnz) == (len(rp) - 1, int(rp[-1]))
+
+
+def test_active_block_counts_of_the_workloads(pa):
+    expect = {2048: 215, 4096: 502, 8192: 1141, 16384: 2548, 32768: 5619, 65536: 12274,
+              131072: 26609, 262144: 57328}
+    for N, nnz in expect.items():
+        assert pa.pa_layout_size(N, 64, 5, 1) == (N // 64, nnz)
+    assert pa.pa_layout_size(2048, 64, 1, 1) == (32, 187)
+
+
+def test_argument_validation_happens_before_any_launch(pa):
+    """These calls must fail on the host (no GPU is present in the CPU test run)."""
+    with pytest.raises(pa.PaError, match="PA_ERR_INVALID_ARG"):
+        pa.pa_layout_size(0, 64, 5, 1)
+    with pytest.raises(pa.PaError, match="PA_ERR_INVALID_ARG"):
+        pa.pa_layout_size(128, 64, -1, 1)
+    null = ctypes.c_void_p(0)
+    st = pa.lib.pa_build_layout(4096, 64, 5, 1, null, null, 10**6, null)
+    assert pa.pa_status_string(st) == "PA_ERR_INVALID_ARG"
+    buf = (ctypes.c_int32 * 64)()
+    st = pa.lib.pa_build_layout(4096, 64, 5, 1, ctypes.addressof(buf), ctypes.addressof(buf), 10, null)
+    assert pa.pa_status_string(st) == "PA_ERR_LAYOUT"
+    assert b"col_capacity" in pa.lib.pa_last_error_message()
+
+    s = pa.pa_strides(0, 512, 128)
+    good = pa.pa_prefill_params(1, 4, 2, 128, 4096, 64, 0.0, s, s, s, s, pa.PA_BF16)
+    p = ctypes.addressof(buf)
+
+    def prefill_status(params, q=p, nnz=10**6, ws=p, ws_bytes=256):
+        return pa.pa_status_string(pa.lib.pa_prefill(ctypes.byref(params), q, p, p, p, p, nnz, p, p, ws,
+                                                     ws_bytes, null))
+
+    bad = pa.pa_prefill_params.from_buffer_copy(good); bad.head_dim = 96
+    assert prefill_status(bad) == "PA_ERR_SHAPE"
+    bad = pa.pa_prefill_params.from_buffer_copy(good); bad.block = 128
+    assert prefill_status(bad) == "PA_ERR_SHAPE"
+    bad = pa.pa_prefill_params.from_buffer_copy(good); bad.n_q_heads = 3
+    assert prefill_status(bad) == "PA_ERR_SHAPE"
+    bad = pa.pa_prefill_params.from_buffer_copy(good); bad.q = pa.pa_strides(0, 516, 128)
+    assert prefill_status(bad) == "PA_ERR_ALIGNMENT"
+    assert prefill_status(good, q=0) == "PA_ERR_INVALID_ARG"
+    assert prefill_status(good, q=p + 4) == "PA_ERR_ALIGNMENT"
+    assert prefill_status(good, nnz=3) == "PA_ERR_LAYOUT"
+    assert prefill_status(good, ws_bytes=8) == "PA_ERR_WORKSPACE"
+
+    dgood = pa.pa_decode_params(2, 4, 2, 128, 64, 5, 1, 4096, 0.0, s, s, pa.PA_BF16)
+    assert pa.pa_decode_workspace_bytes(dgood) == 2 * 4 * (5 + 1 + 6) * 130 * 4
+    dbad = pa.pa_decode_params.from_buffer_copy(dgood); dbad.n_q_heads = 40
+    assert pa.pa_decode_workspace_bytes(dbad) == 0
+    st = pa.lib.pa_decode(ctypes.byref(dbad), p, p, p, p, p, p, p, 10**6, null)
+    assert pa.pa_status_string(st) == "PA_ERR_SHAPE"
+    st = pa.lib.pa_decode(ctypes.byref(dgood), p, p, p, p, p, p, p, 16, null)
+    assert pa.pa_status_string(st) == "PA_ERR_WORKSPACE"
+    st = pa.lib.pa_decode_block_list(0, 64, 5, 1, p, p, 64, null)
+    assert pa.pa_status_string(st) == "PA_ERR_INVALID_ARG"

@@ -1,0 +1,137 @@
+"""GPU: pa_prefill against the fp64 oracle -- element by element on sizes the oracle finishes in
+seconds, on sampled rows at the full workload sizes, plus closed-form checks at any size."""
+import numpy as np
+import pytest
+import torch
+
+import synth_inputs as si
+from util import compare
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pa():
+    import paper_2503_03588_b200 as pa_
+
+    return pa_
+
+
+def _gpu_prefill(pa, Q, K, V, W, S, scale=0.0, o_dtype=torch.bfloat16, layout=None):
+    N = Q.shape[1]
+    rp, ci = layout if layout is not None else pa.pa_build_layout(N, 64, W, S)
+    o, lse, ws = pa.pa_prefill(Q.cuda(), K.cuda(), V.cuda(), rp, ci, softmax_scale=scale, o_dtype=o_dtype)
+    pa.pa_prefill_status(ws)   # synchronises; raises on a device-side timeout
+    return o, lse
+
+
+def _full_compare(pa, oracle, Q, K, V, W, S, scale=0.0, o_dtype=torch.bfloat16, what=""):
+    o, lse = _gpu_prefill(pa, Q, K, V, W, S, scale, o_dtype)
+    o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, W, S, scale=scale if scale else None)
+    return compare(o, lse, o_ref, lse_ref, what)
+
+
+def test_tiny_config(pa, oracle):
+    """Batch 1, 2/2 heads, seq 2048, head_dim 64, window 1, sink 1, scale 1/sqrt(64)."""
+    w = si.TINY_PREFILL
+    Q, K, V = si.prefill_inputs(w)
+    st = _full_compare(pa, oracle, Q, K, V, w.window_blocks, w.sink_blocks, what=w.name)
+    print(w.name, st)
+
+
+@pytest.mark.parametrize("N,Hq,Hkv,D,W,S", [
+    (64, 2, 2, 64, 5, 1),        # one block
+    (1, 2, 1, 128, 5, 1),        # one token
+    (200, 4, 2, 128, 5, 1),      # ragged tail
+    (1000, 7, 1, 128, 5, 1),     # one full 7-head group, ragged
+    (1536, 28, 4, 128, 5, 1),    # the 7B-like head shape
+    (777, 8, 2, 64, 0, 0),       # pure power-of-two pattern
+    (900, 6, 2, 128, 30, 2),     # window covers everything: dense causal
+    (1300, 16, 2, 64, 3, 3),     # group of 8 (two full quads)
+])
+def test_small_shapes(pa, oracle, N, Hq, Hkv, D, W, S):
+    Q = si.bf16_randn((2, N, Hq, D), 100 + N)
+    K = si.bf16_randn((2, N, Hkv, D), 200 + N)
+    V = si.bf16_randn((2, N, Hkv, D), 300 + N)
+    _full_compare(pa, oracle, Q, K, V, W, S, what=f"N={N} Hq={Hq} Hkv={Hkv} D={D} W={W} S={S}")
+
+
+def test_peaky_logits_fp32_output_and_custom_scale(pa, oracle):
+    N, Hq, Hkv, D = 1500, 14, 2, 128
+    Q, K, V = si.bf16_randn((1, N, Hq, D), 1), si.bf16_randn((1, N, Hkv, D), 2, 3.0), si.bf16_randn((1, N, Hkv, D), 3)
+    _full_compare(pa, oracle, Q, K, V, 5, 1, what="peaky bf16")
+    _full_compare(pa, oracle, Q, K, V, 5, 1, scale=0.05, o_dtype=torch.float32, what="fp32 out")
+
+
+def test_strided_inputs(pa, oracle):
+    """Q, K, V as head-slices of one fused QKV tensor (non-contiguous sequence stride)."""
+    N, Hq, Hkv, D = 700, 8, 2, 128
+    qkv = si.bf16_randn((1, N, Hq + 2 * Hkv, D), 5).cuda()
+    Q, K, V = qkv[:, :, :Hq], qkv[:, :, Hq:Hq + Hkv], qkv[:, :, Hq + Hkv:]
+    rp, ci = pa.pa_build_layout(N, 64, 5, 1)
+    o, lse, ws = pa.pa_prefill(Q, K, V, rp, ci)
+    pa.pa_prefill_status(ws)
+    o_ref, lse_ref, _ = oracle.prefill(Q.cpu().contiguous(), K.cpu().contiguous(), V.cpu().contiguous(), 64, 5, 1)
+    compare(o, lse, o_ref, lse_ref, "strided")
+
+
+def test_other_causal_layouts_through_the_same_kernel(pa, oracle):
+    """Dense causal and sliding-window CSRs (built on the host here) run through pa_prefill."""
+    N, Hq, Hkv, D = 1100, 8, 2, 128
+    Q, K, V = si.bf16_randn((1, N, Hq, D), 7), si.bf16_randn((1, N, Hkv, D), 8), si.bf16_randn((1, N, Hkv, D), 9)
+    for use_power, W, S in [(False, 18, 0), (False, 4, 1)]:
+        rp, ci = oracle.block_layout(N, 64, W, S, use_power=use_power)
+        layout = (torch.as_tensor(rp).cuda(), torch.as_tensor(ci).cuda())
+        o, lse = _gpu_prefill(pa, Q, K, V, W, S, layout=layout)
+        o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, W, S, use_power=use_power)
+        compare(o, lse, o_ref, lse_ref, f"use_power={use_power} W={W}")
+
+
+def test_constant_keys_count_the_attended_tokens(pa, oracle):
+    """K rows all equal => LSE_q - s_q = ln |A_q|, |A_q| = 64 * #blocks(row) - (63 - q mod 64);
+    holds at any size, so it is checked at 32K with the 7B-like heads."""
+    N, Hq, Hkv, D, W, S = 32768, 28, 4, 128, 5, 1
+    krow = si.bf16_randn((D,), 41)
+    K = krow.expand(1, N, Hkv, D).contiguous()
+    Q, V = si.bf16_randn((1, N, Hq, D), 42), si.bf16_randn((1, N, Hkv, D), 43)
+    o, lse = _gpu_prefill(pa, Q, K, V, W, S)
+    rp, _ = oracle.block_layout(N, 64, W, S)
+    nblk = np.diff(rp).astype(np.int64)
+    qpos = np.arange(N)
+    n_att = 64 * nblk[qpos // 64] - (63 - qpos % 64)
+    s = (Q[0].double() @ krow.double()).numpy() / np.sqrt(D)          # [N, Hq]
+    got = lse[0].double().cpu().numpy().T                              # [N, Hq]
+    assert np.abs(got - s - np.log(n_att)[:, None]).max() < 1e-3
+    # V constant => every output row equals it (sum of weights is 1)
+    vrow = si.bf16_randn((D,), 44)
+    Vc = vrow.expand(1, N, Hkv, D).contiguous()
+    o, _ = _gpu_prefill(pa, Q, si.bf16_randn((1, N, Hkv, D), 45), Vc, W, S)
+    assert (o[0].float().cpu() - vrow.float()).abs().max() < 2e-2
+
+
+def _sampled_rows(N, rng, n_random=96):
+    """Query positions spanning the first and last blocks, power-of-two block boundaries and a
+    seeded random sample."""
+    rows = {0, 1, 63, 64, 65, N - 1, N - 64, N - 65}
+    k = 1
+    while 64 * k < N:
+        for off in (-1, 0, 1, 37):
+            r = 64 * k + off
+            if 0 <= r < N:
+                rows.add(r)
+        k *= 2
+    rows.update(int(x) for x in rng.integers(0, N, n_random))
+    return sorted(rows)
+
+
+@pytest.mark.parametrize("w", [si.PREFILL_32K, si.PREFILL_128K], ids=lambda w: w.name)
+def test_full_size_workloads_on_sampled_rows(pa, oracle, w):
+    """The benchmark's launch configuration; the oracle evaluates sampled query rows, all heads."""
+    Q, K, V = si.prefill_inputs(w)
+    o, lse = _gpu_prefill(pa, Q, K, V, w.window_blocks, w.sink_blocks)
+    rows = _sampled_rows(w.seq_len, np.random.default_rng(w.seed))
+    o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, w.window_blocks, w.sink_blocks, rows=rows)
+    ridx = torch.as_tensor(rows).cuda()
+    st = compare(o[:, ridx], lse[:, :, ridx], o_ref, lse_ref, w.name)
+    print(w.name, st)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
