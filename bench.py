@@ -1,0 +1,386 @@
+#!/usr/bin/env python
+"""Benchmark of the PowerAttention hot path on B200: prints ONE JSON line.
+
+A step is one pass of the whole path on resident synthetic inputs: pa_build_layout +
+pa_prefill at 128K tokens (28 query / 4 KV heads, head_dim 128, block 64, window 5, sink 1)
+followed by pa_decode on the batch-8 decode workload.  The metric is the prefill's active-block
+throughput: 4 * 64 * 64 * head_dim FLOP per listed block pair per query head, over the step time.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 (under torchrun) runs independent replicas, one per GPU: the operator has no exchange
+step, so there is no collective on the data path; time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import synth_inputs as si  # noqa: E402
+
+METRIC = "prefill_active_block_tflops_128k"
+UNIT = "TFLOP/s"
+
+
+def block_pair_flops(nnz: int, w) -> float:
+    return 4.0 * w.block * w.block * w.head_dim * nnz * w.n_q_heads * w.batch
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------ multi-rank glue
+
+def dist_env():
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return world, rank, local
+
+
+def aggregate(ms_local: float, flops_local: float, group=None, device="cpu"):
+    """Replica aggregation: job time = max over ranks, job work = sum over ranks."""
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()):
+        return ms_local, flops_local
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    f = torch.tensor([flops_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX, group=group)
+    dist.all_reduce(f, op=dist.ReduceOp.SUM, group=group)
+    return float(t.item()), float(f.item())
+
+
+# ------------------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-i", str(self.gpu), "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+                for name, val in zip(names, f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out = dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(smax)), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------ reference arm
+
+def oracle_sample_rows(w, every: int):
+    """Every `every`-th query block of the workload, all 64 rows of each."""
+    nqb = w.seq_len // w.block
+    blocks = np.arange(nqb - 1, -1, -every)
+    return np.sort((blocks[:, None] * w.block + np.arange(w.block)[None, :]).reshape(-1))
+
+
+def time_oracle(w, Q, K, V, every: int, nnz_rows_flops):
+    """Times the fp64 oracle, as it stands, on the sampled rows; returns (seconds, flops, cores)."""
+    from oracle import oracle
+
+    rows = oracle_sample_rows(w, every)
+    t0 = time.time()
+    oracle.prefill(Q, K, V, w.block, w.window_blocks, w.sink_blocks, rows=rows)
+    dt = time.time() - t0
+    return dt, nnz_rows_flops(rows), oracle.max_threads(), len(rows)
+
+
+def run_reference(args):
+    world, rank, _ = dist_env()
+    if rank != 0:
+        return
+    from oracle import oracle
+
+    w = si.PREFILL_128K
+    Q, K, V = si.prefill_inputs(w)
+    rp, _ = oracle.block_layout(w.seq_len, w.block, w.window_blocks, w.sink_blocks)
+    row_len = np.diff(rp)
+
+    def flops_of(rows):
+        blocks = np.unique(rows // w.block)
+        return 4.0 * w.block * w.block * w.head_dim * float(row_len[blocks].sum()) * w.n_q_heads
+
+    every = 64  # 32 query blocks = 2048 rows per step: a few seconds of CPU work
+    times = []
+    for it in range(args.warmup + args.steps):
+        dt, fl, cores, nrows = time_oracle(w, Q, K, V, every, flops_of)
+        if it >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    value = fl / (ms * 1e-3) / 1e12
+    sample = f"every {every}th query block of the 128K workload ({nrows} rows, all 28 heads) per step"
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=w.name, seq_len=w.seq_len, n_q_heads=w.n_q_heads,
+                            n_kv_heads=w.n_kv_heads, head_dim=w.head_dim, block=w.block,
+                            window_blocks=w.window_blocks, sink_blocks=w.sink_blocks),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------ our arm
+
+def run_ours(args):
+    import paper_2503_03588_b200 as pa  # raises if the CUDA library is missing: no fallback
+
+    world, rank, local = dist_env()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (B200)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = read_peaks()
+
+    w, wd = si.PREFILL_128K, si.DECODE_B8
+    Qh, Kh, Vh = si.prefill_inputs(w, pin=True)
+    Q, K, V = Qh.to(dev), Kh.to(dev), Vh.to(dev)
+    nqb, nnz = pa.pa_layout_size(w.seq_len, w.block, w.window_blocks, w.sink_blocks)
+    flops = block_pair_flops(nnz, w)
+    row_ptr = torch.empty(nqb + 1, dtype=torch.int32, device=dev)
+    col_idx = torch.empty(nnz, dtype=torch.int32, device=dev)
+    O = torch.empty_like(Q)
+    LSE = torch.empty((w.batch, w.n_q_heads, w.seq_len), dtype=torch.float32, device=dev)
+    ws = torch.empty(4096, dtype=torch.uint8, device=dev)
+
+    qd_h, kc_h, vc_h, lens = si.decode_inputs(wd)
+    qd, kc, vc = qd_h.to(dev), kc_h.to(dev), vc_h.to(dev)
+    del kc_h, vc_h
+    lens_d = torch.as_tensor(lens, dtype=torch.int32, device=dev)
+    Od = torch.empty((wd.batch, wd.n_q_heads, wd.head_dim), dtype=torch.bfloat16, device=dev)
+    LSEd = torch.empty((wd.batch, wd.n_q_heads), dtype=torch.float32, device=dev)
+    dparams = pa.binding.decode_params(qd, kc, vc, wd.window_blocks, wd.sink_blocks)
+    wsd = torch.empty(pa.pa_decode_workspace_bytes(dparams), dtype=torch.uint8, device=dev)
+
+    stream = torch.cuda.current_stream()
+    ev_p0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ev_p1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+
+    def step(i=None):
+        pa.pa_build_layout(w.seq_len, w.block, w.window_blocks, w.sink_blocks, row_ptr, col_idx)
+        if i is not None:
+            ev_p0[i].record(stream)
+        pa.pa_prefill(Q, K, V, row_ptr, col_idx, o=O, lse=LSE, workspace=ws)
+        if i is not None:
+            ev_p1[i].record(stream)
+        pa.pa_decode(qd, kc, vc, lens_d, wd.window_blocks, wd.sink_blocks, o=Od, lse=LSEd, workspace=wsd)
+
+    launches_per_step = 3 + 1 + 2  # layout (count, scan, fill) + prefill + decode (partial, combine)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    pa.pa_prefill_status(ws)
+    torch.cuda.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if world > 1:
+        torch.distributed.barrier()
+    pa.pa_prefill_status(ws)
+    ms_local = e0.elapsed_time(e1) / args.steps
+    prefill_ms = float(np.mean([a.elapsed_time(b) for a, b in zip(ev_p0, ev_p1)]))
+    ms, flops_all = aggregate(ms_local, flops, device=dev)
+
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return
+
+    # ---- decode bandwidth: CUDA graph of launches rotating over 16 seeded length sets so that
+    # consecutive launches touch different cache regions (touched bytes per call fit in L2).
+    n_sets, reps = 16, 8
+    rng = np.random.Generator(np.random.PCG64(wd.lens_seed + 1))
+    lens_sets = [rng.integers(wd.min_len, wd.max_len + 1, size=wd.batch, dtype=np.int64) for _ in range(n_sets)]
+    lens_sets_d = [torch.as_tensor(x, dtype=torch.int32, device=dev) for x in lens_sets]
+
+    def touched_bytes(ls):
+        total = 0
+        for L in ls:
+            nblk = len(pa.pa_decode_block_list(int(L), wd.block, wd.window_blocks, wd.sink_blocks))
+            keys = wd.block * (nblk - 1) + (int(L) - 1) % wd.block + 1
+            total += keys * wd.head_dim * 2 * 2 * wd.n_kv_heads
+        return total
+
+    dec_bytes = float(np.mean([touched_bytes(ls) for ls in lens_sets]))
+    side = torch.cuda.Stream(device=dev)
+    side.wait_stream(stream)
+    with torch.cuda.stream(side):
+        for ld in lens_sets_d:
+            pa.pa_decode(qd, kc, vc, ld, wd.window_blocks, wd.sink_blocks, o=Od, lse=LSEd, workspace=wsd)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(reps):
+                for ld in lens_sets_d:
+                    pa.pa_decode(qd, kc, vc, ld, wd.window_blocks, wd.sink_blocks, o=Od, lse=LSEd, workspace=wsd)
+        graph.replay()
+        torch.cuda.synchronize()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(side)
+        graph.replay()
+        d1.record(side)
+        torch.cuda.synchronize()
+    dec_us = 1e3 * d0.elapsed_time(d1) / (n_sets * reps)
+    dec_gbs = dec_bytes / (dec_us * 1e-6) / 1e9
+
+    # ---- end to end through the public API with host buffers: pinned H2D of Q, K, V, the call,
+    # D2H of O and LSE, all inside the timed region.
+    Oh = torch.empty(O.shape, dtype=O.dtype, pin_memory=True)
+    LSEh = torch.empty(LSE.shape, dtype=LSE.dtype, pin_memory=True)
+    e2e_steps = max(1, min(args.steps, 5))
+
+    def e2e_step():
+        Q.copy_(Qh, non_blocking=True)
+        K.copy_(Kh, non_blocking=True)
+        V.copy_(Vh, non_blocking=True)
+        pa.pa_build_layout(w.seq_len, w.block, w.window_blocks, w.sink_blocks, row_ptr, col_idx)
+        pa.pa_prefill(Q, K, V, row_ptr, col_idx, o=O, lse=LSE, workspace=ws)
+        Oh.copy_(O, non_blocking=True)
+        LSEh.copy_(LSE, non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize()
+    x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    x0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    x1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = x0.elapsed_time(x1) / e2e_steps
+    h2d = sum(t.numel() * t.element_size() for t in (Qh, Kh, Vh))
+    d2h = sum(t.numel() * t.element_size() for t in (Oh, LSEh))
+
+    # ---- CPU baseline: the oracle, as it stands, on a bounded sample of the same workload.
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import oracle
+
+        rp_ref, _ = oracle.block_layout(w.seq_len, w.block, w.window_blocks, w.sink_blocks)
+        row_len = np.diff(rp_ref)
+
+        def flops_of(rows):
+            blocks = np.unique(rows // w.block)
+            return 4.0 * w.block * w.block * w.head_dim * float(row_len[blocks].sum()) * w.n_q_heads
+
+        every = 16
+        dt, fl, cores, nrows = time_oracle(w, Qh, Kh, Vh, every, flops_of)
+        cpu = dict(value=fl / dt / 1e12, unit=UNIT, cores=cores, kind="oracle",
+                   sample=f"every {every}th query block of the 128K workload ({nrows} rows, all heads), {dt:.1f} s")
+
+    value = flops_all / (ms * 1e-3) / 1e12
+    achieved = flops / (prefill_ms * 1e-3) / 1e12
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+                ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                data="synthetic",
+                config=dict(workload=w.name, seq_len=w.seq_len, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads,
+                            head_dim=w.head_dim, block=w.block, window_blocks=w.window_blocks,
+                            sink_blocks=w.sink_blocks, active_block_pairs=nnz, step="layout+prefill+decode",
+                            decode_workload=wd.name, l2="inputs larger than L2 (Q+K+V+O = 2.4 GB per step)",
+                            parallelism="replicas" if world > 1 else "single"),
+                clocks=clocks,
+                roofline=dict(bound="tensor", achieved=achieved, peak=peaks["bf16_tflops"], unit="TFLOP/s",
+                              frac=achieved / peaks["bf16_tflops"], traffic=None,
+                              peak_source=peaks["source"] + " burst bf16", kernel="prefill_kernel<128>",
+                              kernel_ms=prefill_ms,
+                              frac_of_sustained=achieved / peaks["bf16_tflops_sustained"]),
+                decode=dict(metric="decode_kv_gbs", value=dec_gbs, unit="GB/s", us_per_call=dec_us,
+                            kv_bytes_per_call=dec_bytes, peak=peaks["hbm_gbs"], frac=dec_gbs / peaks["hbm_gbs"],
+                            bound="hbm", timing=f"CUDA graph of {n_sets * reps} calls rotating over {n_sets} seeded length sets",
+                            workload=wd.name),
+                e2e=dict(value=flops / (e2e_ms * 1e-3) / 1e12, unit=UNIT, ms_per_step=e2e_ms,
+                         h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
+                gpu_launches=launches_per_step * args.steps,
+                cpu_baseline=cpu)
+    print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
