@@ -161,6 +161,39 @@ pa_status pa_decode_block_list(int64_t cache_len, int32_t block, int32_t window_
                                int32_t sink_blocks, int32_t *out_blocks, int32_t *out_count,
                                int32_t capacity, void *stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Decode without any allocation.  (The paper has no counterpart to this entry point; it exists
+ * for integration reasons only.)
+ *
+ * Some hosts of this library are not allowed to obtain device memory at the moment they need to
+ * decode: code that runs inside a memory-pool or allocator callback, plug-ins whose embedding
+ * runtime owns every byte of the device and hands out none, and real-time serving loops in which
+ * an allocation (which may synchronise the device or fail) is forbidden once warm-up is over.
+ * pa_decode asks such callers for a workspace they have no means to provide.  pa_decode_static
+ * computes exactly what pa_decode computes, but keeps the split-K partial results in an array of
+ * PA_DECODE_STATIC_SCRATCH_BYTES bytes that is part of the library image.  Every GPU on which
+ * the library's code gets loaded carries that array until the process exits.
+ *
+ * Arguments q, k_cache, v_cache, cache_lens, o, lse and stream: as for pa_decode.
+ *   - Limit: pa_decode_workspace_bytes(p) must not exceed PA_DECODE_STATIC_SCRATCH_BYTES,
+ *     otherwise PA_ERR_WORKSPACE is returned (with a message giving both numbers) and nothing is
+ *     launched.  The batch-8, 28-head, head_dim-128, 128K-token workload needs about 2 MB.
+ *   - The call itself performs no device allocation or free, and calls no library that does.
+ *   - The first call on each device looks up the array's device address (a one-time set-up that
+ *     loads the library's device code if it is not loaded yet).  Make that first call during
+ *     start-up, outside any stream capture.
+ *   - All calls on one device share the one array, and it still holds the previous call's
+ *     partial results when the next call starts.  Nothing in it has to start at zero: each call
+ *     overwrites every entry it later reads.  Because the array is shared, two calls that run
+ *     on the GPU at the same time (different streams, or different host threads) overwrite each
+ *     other's partial results; issue them on one stream or order them yourself.
+ * ------------------------------------------------------------------------------------------ */
+#define PA_DECODE_STATIC_SCRATCH_BYTES (4u << 20)
+
+pa_status pa_decode_static(const pa_decode_params *p, const void *q, const void *k_cache,
+                           const void *v_cache, const int32_t *cache_lens, void *o, float *lse,
+                           void *stream);
+
 #ifdef __cplusplus
 }
 #endif

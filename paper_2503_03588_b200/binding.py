@@ -22,7 +22,7 @@ STATUS_NAMES = ["PA_OK", "PA_ERR_INVALID_ARG", "PA_ERR_SHAPE", "PA_ERR_ALIGNMENT
 
 EXPORTS = ["pa_status_string", "pa_last_error_message", "pa_version", "pa_layout_size",
            "pa_build_layout", "pa_prefill_workspace_bytes", "pa_prefill", "pa_prefill_status",
-           "pa_decode_workspace_bytes", "pa_decode", "pa_decode_block_list"]
+           "pa_decode_workspace_bytes", "pa_decode", "pa_decode_block_list", "pa_decode_static"]
 
 
 class PaError(RuntimeError):
@@ -80,6 +80,8 @@ def _load() -> ctypes.CDLL:
                               ctypes.c_size_t, vp]
     lib.pa_decode_block_list.restype = ctypes.c_int
     lib.pa_decode_block_list.argtypes = [i64, i32, i32, i32, vp, vp, i32, vp]
+    lib.pa_decode_static.restype = ctypes.c_int
+    lib.pa_decode_static.argtypes = [ctypes.POINTER(pa_decode_params), vp, vp, vp, vp, vp, vp, vp]
     return lib
 
 
@@ -207,3 +209,22 @@ def pa_decode_block_list(cache_len: int, block: int, window_blocks: int, sink_bl
                                     capacity, _stream()))
     n = int(cnt.item())
     return out[:n].clone()
+
+
+PA_DECODE_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def pa_decode_static(q, k_cache, v_cache, cache_lens, window_blocks: int, sink_blocks: int, o, lse,
+                     block: int = 64, softmax_scale: float = 0.0):
+    """pa_decode for callers that may not allocate: the split-K scratch lives inside the library.
+
+    Unlike the other wrappers this one never creates a tensor: `o` [batch, Hq, D] and `lse`
+    [batch, Hq] must be passed in.  Problems whose scratch would exceed
+    PA_DECODE_STATIC_SCRATCH_BYTES raise PaError(PA_ERR_WORKSPACE).  Calls that overlap on the GPU
+    share (and would corrupt) the one built-in scratch array: keep them on one stream.
+    """
+    assert cache_lens.dtype == torch.int32 and q.is_contiguous() and o.is_contiguous()
+    params = decode_params(q, k_cache, v_cache, window_blocks, sink_blocks, block, softmax_scale, o.dtype)
+    _check(lib.pa_decode_static(ctypes.byref(params), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(cache_lens),
+                                _ptr(o), _ptr(lse), _stream()))
+    return o, lse

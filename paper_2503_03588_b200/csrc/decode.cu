@@ -349,3 +349,60 @@ extern "C" pa_status pa_decode_block_list(int64_t cache_len, int32_t block, int3
     PA_CUDA_OK(cudaGetLastError());
     return PA_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// pa_decode_static: the same decode, for callers that cannot allocate device memory.
+//
+// The split-K partial results go to a fixed array that is part of the library image instead of
+// a caller-provided workspace.  The array's name is only a host-side handle in host code; the
+// real device address is looked up once per device with cudaGetSymbolAddress (with that device
+// current) and then handed to the kernels like any other pointer.
+// ------------------------------------------------------------------------------------------
+#include <mutex>
+
+namespace pa {
+
+static __device__ __align__(256) unsigned char g_decode_static_scratch[PA_DECODE_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mu;
+static void *g_static_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device (looked up on first use).
+static pa_status static_scratch_address(void **out)
+{
+    int dev = 0;
+    PA_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices)
+        return fail(PA_ERR_UNSUPPORTED, "device index %d is beyond the %d devices supported", dev, kMaxDevices);
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void *ptr = nullptr;
+        PA_CUDA_OK(cudaGetSymbolAddress(&ptr, g_decode_static_scratch));
+        if (!ptr) return fail(PA_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+        g_static_ptr[dev] = ptr;
+    }
+    *out = g_static_ptr[dev];
+    return PA_OK;
+}
+
+}  // namespace pa
+
+extern "C" pa_status pa_decode_static(const pa_decode_params *p, const void *q, const void *k_cache,
+                                      const void *v_cache, const int32_t *cache_lens, void *o,
+                                      float *lse, void *stream)
+{
+    using namespace pa;
+    clear_error();
+    if (pa_status s = check_decode(p)) return s;
+    const size_t need = pa_decode_workspace_bytes(p);
+    if (need > (size_t)PA_DECODE_STATIC_SCRATCH_BYTES)
+        return fail(PA_ERR_WORKSPACE,
+                    "this problem needs %zu bytes of split-K scratch but the built-in array holds %zu; "
+                    "use pa_decode with a caller-allocated workspace", need,
+                    (size_t)PA_DECODE_STATIC_SCRATCH_BYTES);
+    void *scratch = nullptr;
+    if (pa_status s = static_scratch_address(&scratch)) return s;
+    return pa_decode(p, q, k_cache, v_cache, cache_lens, o, lse, scratch,
+                     (size_t)PA_DECODE_STATIC_SCRATCH_BYTES, stream);
+}
