@@ -368,6 +368,32 @@ def run_ours(args):
         torch.distributed.destroy_process_group()
 
 
+def run_case(args):
+    """A small single-kernel case for profiler captures: a few launches, nothing else."""
+    import paper_2503_03588_b200 as pa
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    if args.case == "prefill32k":
+        w = si.PREFILL_32K
+        Q, K, V = (t.to(dev) for t in si.prefill_inputs(w))
+        rp, ci = pa.pa_build_layout(w.seq_len, w.block, w.window_blocks, w.sink_blocks)
+        o, lse, ws = pa.pa_prefill(Q, K, V, rp, ci)
+        for _ in range(args.steps):
+            pa.pa_prefill(Q, K, V, rp, ci, o=o, lse=lse, workspace=ws)
+        pa.pa_prefill_status(ws)
+    else:
+        wd = si.DECODE_B8
+        qd, kc, vc, lens = si.decode_inputs(wd)
+        qd, kc, vc = qd.to(dev), kc.to(dev), vc.to(dev)
+        lens_d = torch.as_tensor(lens, dtype=torch.int32, device=dev)
+        o, lse, ws = pa.pa_decode(qd, kc, vc, lens_d, wd.window_blocks, wd.sink_blocks)
+        for _ in range(args.steps):
+            pa.pa_decode(qd, kc, vc, lens_d, wd.window_blocks, wd.sink_blocks, o=o, lse=lse, workspace=ws)
+    torch.cuda.synchronize()
+    print(json.dumps(dict(case=args.case, launches=args.steps + 1)))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -375,7 +401,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--case", default=None, choices=["prefill32k", "decode"],
+                    help="run only a small single-kernel case (for profiler captures)")
     args = ap.parse_args()
+    if args.case:
+        run_case(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -26,7 +26,8 @@ namespace pa {
 constexpr int kBlk = 64;               // tokens per query / key block
 constexpr int kThreads = 384;          // 12 warps
 constexpr int kStages = 4;             // K/V ring depth
-constexpr uint32_t kTmemCols = 512;    // S0 S1 (64 cols each) at 0, O0 O1 (D cols each) at 128
+constexpr uint32_t kTmemCols = 512;    // S[slot][buf] 64 cols each at 0..255, O0 O1 (D cols each) at 256
+constexpr float kRescaleThreshold = 8.0f;  // base-2 logits: rescale O only when the row max grows by more
 constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
 
 struct PrefillArgs {
@@ -59,7 +60,7 @@ struct SmemMap {
 // Barrier slots inside the barrier area (8 bytes each).
 enum : uint32_t {
     BAR_Q_FULL = 0, BAR_Q_EMPTY = 1, BAR_KV_FULL = 2, BAR_KV_EMPTY = 2 + kStages,
-    BAR_S_FULL = 2 + 2 * kStages, BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2,
+    BAR_S_FULL = 2 + 2 * kStages, BAR_P_FULL = BAR_S_FULL + 4, BAR_O_DONE = BAR_P_FULL + 2,
     BAR_COUNT = BAR_O_DONE + 2
 };
 
@@ -127,7 +128,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::mbar_init(bar(BAR_KV_EMPTY + s), 1);
         }
         for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(bar(BAR_S_FULL + s), 1);
+            ptx::mbar_init(bar(BAR_S_FULL + 2 * s), 1);
+            ptx::mbar_init(bar(BAR_S_FULL + 2 * s + 1), 1);
             ptx::mbar_init(bar(BAR_P_FULL + s), 128);
             ptx::mbar_init(bar(BAR_O_DONE + s), 1);
         }
@@ -196,67 +198,92 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ tcgen05 issuer
-        if (lane == 0) {
+        // The whole warp runs the (uniform) control flow and the barrier waits; one elected lane
+        // issues the MMAs and commits.  Descriptors: the high word is constant per operand kind
+        // (stride 1024 B between 8-row groups, version 1, 128-byte swizzle); the low word holds
+        // the start address >> 4 (plus the leading-dimension offset for the MN-major V operand).
+        {
+            const bool leader = ptx::elect_one();
             constexpr uint32_t idesc_qk = ptx::idesc_bf16_f32(128, 64, 0);
             constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(128, D, 1);
+            constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+            const uint32_t q_lo = ((smem_base + SM::kQ) >> 4) | (1u << 16);
+            const uint32_t p_lo = ((smem_base + SM::kP) >> 4) | (1u << 16);
+            const uint32_t k_lo = ((smem_base + SM::kKV) >> 4) | (1u << 16);
+            const uint32_t v_lo = ((smem_base + SM::kKV + SM::kKTile) >> 4) | ((SM::kKVSub >> 4) << 16);
             // S_s = Q_s K^T: A = Q tile (K-major), B = K block (K-major), 16 features per MMA.
-            auto issue_qk = [&](int s, uint32_t st) {
-                const uint32_t qa = smem_base + SM::kQ + s * SM::kQSlot;
-                const uint32_t kb = smem_base + SM::kKV + st * SM::kStage;
+            auto issue_qk = [&](int s, uint32_t buf, uint32_t st) {
+                const uint32_t qa = q_lo + s * (SM::kQSlot >> 4);
+                const uint32_t kb = k_lo + st * (SM::kStage >> 4);
+                const uint32_t dst = tmem_base + (2 * s + buf) * 64;
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint64_t ad = ptx::smem_desc_sw128(qa + (kk / 4) * SM::kQSub + (kk % 4) * 32, 16, 1024);
-                    const uint64_t bd = ptx::smem_desc_sw128(kb + (kk / 4) * SM::kKVSub + (kk % 4) * 32, 16, 1024);
-                    ptx::umma_ss(tmem_base + s * 64, ad, bd, idesc_qk, kk > 0);
-                }
+                for (int kk = 0; kk < D / 16; ++kk)
+                    ptx::umma_ss_lohi(dst, qa + (((kk / 4) * SM::kQSub + (kk % 4) * 32) >> 4), desc_hi,
+                                      kb + (((kk / 4) * SM::kKVSub + (kk % 4) * 32) >> 4), desc_hi, idesc_qk,
+                                      kk > 0 ? 1u : 0u);
             };
             // O_s (+)= P_s V: A = P tile (K-major over keys), B = V block (MN-major: features
             // contiguous), 16 keys per MMA.
             auto issue_pv = [&](int s, uint32_t st, bool acc) {
-                const uint32_t pa_ = smem_base + SM::kP + s * SM::kPSlot;
-                const uint32_t vb = smem_base + SM::kKV + st * SM::kStage + SM::kKTile;
+                const uint32_t pa_ = p_lo + s * (SM::kPSlot >> 4);
+                const uint32_t vb = v_lo + st * (SM::kStage >> 4);
+                const uint32_t dst = tmem_base + 256 + s * D;
 #pragma unroll
-                for (int kk = 0; kk < kBlk / 16; ++kk) {
-                    const uint64_t ad = ptx::smem_desc_sw128(pa_ + kk * 32, 16, 1024);
-                    const uint64_t bd = ptx::smem_desc_sw128(vb + kk * 2048, SM::kKVSub, 1024);
-                    ptx::umma_ss(tmem_base + 128 + s * D, ad, bd, idesc_pv, (acc || kk > 0) ? 1u : 0u);
-                }
+                for (int kk = 0; kk < kBlk / 16; ++kk)
+                    ptx::umma_ss_lohi(dst, pa_ + ((kk * 32) >> 4), desc_hi, vb + ((kk * 2048) >> 4), desc_hi,
+                                      idesc_pv, (acc || kk > 0) ? 1u : 0u);
             };
             uint32_t kvc = 0, ul = 0, g = 0;
             bool ok = true;
             for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
                 const Unit w = decode_unit(a, u);
                 if (w.n <= 0) continue;
-                ok = wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 3);
+                ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 3));
                 if (!ok) break;
-                ok = wait_bar(bar(BAR_KV_FULL + kvc % kStages), (kvc / kStages) & 1, abort_flag, a.status, 4);
-                if (!ok) break;
-                ptx::tc_fence_after_sync();
-                for (int s = 0; s < 2; ++s) {
-                    issue_qk(s, kvc % kStages);
-                    ptx::umma_commit(bar(BAR_S_FULL + s));
+                // Prologue: S of the first two steps (S is double-buffered per slot).
+                for (int t0 = 0; t0 < 2 && t0 < w.n && ok; ++t0) {
+                    const uint32_t c0 = kvc + t0;
+                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_KV_FULL + c0 % kStages), (c0 / kStages) & 1,
+                                                          abort_flag, a.status, 4));
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    if (leader) {
+                        for (int s = 0; s < 2; ++s) {
+                            issue_qk(s, (g + t0) & 1, c0 % kStages);
+                            ptx::umma_commit(bar(BAR_S_FULL + 2 * s + ((g + t0) & 1)));
+                        }
+                    }
+                    __syncwarp();
                 }
-                if (w.n == 1) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                if (!ok) break;
+                if (w.n <= 2 && leader) ptx::umma_commit(bar(BAR_Q_EMPTY));
                 for (int t = 0; t < w.n && ok; ++t) {
                     const uint32_t st = (kvc + t) % kStages;
                     for (int s = 0; s < 2; ++s) {
-                        ok = wait_bar(bar(BAR_P_FULL + s), (g + t) & 1, abort_flag, a.status, 5);
+                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + s), (g + t) & 1, abort_flag, a.status, 5));
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
-                        issue_pv(s, st, t > 0);
-                        ptx::umma_commit(bar(BAR_O_DONE + s));
-                        if (s == 1) ptx::umma_commit(bar(BAR_KV_EMPTY + st));
-                        if (t + 1 < w.n) {
-                            const uint32_t c1 = kvc + t + 1;
+                        if (leader) {
+                            issue_pv(s, st, t > 0);
+                            ptx::umma_commit(bar(BAR_O_DONE + s));
+                            if (s == 1) ptx::umma_commit(bar(BAR_KV_EMPTY + st));
+                        }
+                        __syncwarp();
+                        if (t + 2 < w.n) {
+                            // S buffer (g + t) & 1 of this slot was consumed by the softmax of step t.
+                            const uint32_t c2 = kvc + t + 2;
                             if (s == 0) {
-                                ok = wait_bar(bar(BAR_KV_FULL + c1 % kStages), (c1 / kStages) & 1,
-                                              abort_flag, a.status, 6);
+                                ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_KV_FULL + c2 % kStages),
+                                                                      (c2 / kStages) & 1, abort_flag, a.status, 6));
                                 if (!ok) break;
                                 ptx::tc_fence_after_sync();
                             }
-                            issue_qk(s, c1 % kStages);
-                            ptx::umma_commit(bar(BAR_S_FULL + s));
-                            if (s == 1 && t + 2 == w.n) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                            if (leader) {
+                                issue_qk(s, (g + t) & 1, c2 % kStages);
+                                ptx::umma_commit(bar(BAR_S_FULL + 2 * s + ((g + t) & 1)));
+                                if (s == 1 && t + 3 == w.n) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                            }
+                            __syncwarp();
                         }
                     }
                 }
@@ -272,8 +299,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const int quad = warp & 3;              // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;       // tile row = TMEM lane
         const int qrow = row & 63;              // token inside the query block
-        const uint32_t t_s = tmem_base + ((uint32_t)(quad * 32) << 16) + s * 64;
-        const uint32_t t_o = tmem_base + ((uint32_t)(quad * 32) << 16) + 128 + s * D;
+        const uint32_t t_s0 = tmem_base + ((uint32_t)(quad * 32) << 16) + 2 * s * 64;
+        const uint32_t t_o = tmem_base + ((uint32_t)(quad * 32) << 16) + 256 + s * D;
         uint8_t *p_row = smem + SM::kP + s * SM::kPSlot + row * 128;
         const float sl2 = a.scale_log2;
         uint32_t g = 0;
@@ -287,11 +314,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             float m = -INFINITY, l = 0.f;
             for (int t = 0; t < w.n; ++t, ++g) {
                 const int32_t j = __ldg(a.col_idx + w.rs + t);
-                ok = wait_bar(bar(BAR_S_FULL + s), g & 1, abort_flag, a.status, 7);
+                ok = wait_bar(bar(BAR_S_FULL + 2 * s + (g & 1)), (g >> 1) & 1, abort_flag, a.status, 7);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 uint32_t sr[64];
+                const uint32_t t_s = t_s0 + (g & 1) * 64;
                 ptx::tmem_ld32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
                 ptx::tmem_ld32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
                 ptx::tmem_wait_ld();
@@ -301,21 +329,36 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     for (int c = 0; c < 64; ++c)
                         if (c > qrow) sr[c] = 0xff800000u;  // -inf
                 }
-                float mx = __uint_as_float(sr[0]);
+                float mx4[4] = {__uint_as_float(sr[0]), __uint_as_float(sr[1]), __uint_as_float(sr[2]),
+                                __uint_as_float(sr[3])};
 #pragma unroll
-                for (int c = 1; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
-                const float m_new = fmaxf(m, mx * sl2);
-                const float alpha = ptx::ex2(m - m_new);
-                float sum = 0.f;
+                for (int c = 4; c < 64; c += 4) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) mx4[e] = fmaxf(mx4[e], __uint_as_float(sr[c + e]));
+                }
+                const float mx2 = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
+                // Lazy rescaling: keep the old reference max unless the row max grew by more than
+                // the threshold; exp2(s - m) then stays below 2^threshold, and O / l at the end is
+                // exact whatever reference was used.
+                const bool grow = t == 0 || mx2 > m + kRescaleThreshold;
+                const float m_new = grow ? mx2 : m;
+                const float alpha = grow ? ptx::ex2(m - m_new) : 1.0f;
+                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
                 uint32_t pk[32];
 #pragma unroll
-                for (int c = 0; c < 64; c += 2) {
-                    const float p0 = ptx::ex2(fmaf(__uint_as_float(sr[c]), sl2, -m_new));
-                    const float p1 = ptx::ex2(fmaf(__uint_as_float(sr[c + 1]), sl2, -m_new));
-                    sum += p0 + p1;
-                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-                    pk[c >> 1] = *reinterpret_cast<const uint32_t *>(&h2);
+                for (int c = 0; c < 64; c += 4) {
+                    float pv[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        pv[e] = ptx::ex2(fmaf(__uint_as_float(sr[c + e]), sl2, -m_new));
+                        sum4[e] += pv[e];
+                    }
+                    const __nv_bfloat162 h01 = __floats2bfloat162_rn(pv[0], pv[1]);
+                    const __nv_bfloat162 h23 = __floats2bfloat162_rn(pv[2], pv[3]);
+                    pk[c >> 1] = *reinterpret_cast<const uint32_t *>(&h01);
+                    pk[(c >> 1) + 1] = *reinterpret_cast<const uint32_t *>(&h23);
                 }
+                const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
                 l = l * alpha + sum;
                 m = m_new;
                 if (t > 0) {
