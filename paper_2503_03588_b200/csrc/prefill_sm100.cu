@@ -4,10 +4,13 @@
 // One persistent CTA per SM walks work units (batch, KV head, query block, head quad).  A unit
 // holds two 128-row tiles ("slots"); a tile stacks two query heads of the KV group on the 64
 // tokens of the query block (the mask does not depend on the head, so they share the key list
-// and the K/V tiles).  Warp roles:
-//   warp 0      TMA producer: Q tiles once per unit, then the listed K/V blocks, gathered by block
-//               index, into a ring of shared-memory stages (128-byte swizzle)
-//   warp 1      tcgen05 issuer: S = Q K^T into tensor memory, later O += P V
+// and the K/V tiles).  The key list is walked two blocks at a time: the gathered blocks are put
+// side by side in shared memory so that S = Q K^T runs with N = 128 and O += P V with K = 128
+// (a row of odd length ends with a single-block step, N = 64).  Warp roles:
+//   warp 0      TMA producer: Q tiles once per unit, then the listed K and V blocks, gathered by
+//               block index, into two rings of shared-memory pair tiles (128-byte swizzle)
+//   warp 1      tcgen05 issuer: S = Q K^T into tensor memory; O += P V with P read from tensor
+//               memory (it overlays the S columns it was computed from)
 //   warp 2      tensor-memory allocation
 //   warps 4-7   online softmax of slot 0 (thread = tile row = TMEM lane)
 //   warps 8-11  online softmax of slot 1
@@ -25,8 +28,9 @@ namespace pa {
 
 constexpr int kBlk = 64;               // tokens per query / key block
 constexpr int kThreads = 384;          // 12 warps
-constexpr int kStages = 4;             // K/V ring depth
-constexpr uint32_t kTmemCols = 512;    // S[slot][buf] 64 cols each at 0..255, O0 O1 (D cols each) at 256
+constexpr int kKStages = 3;            // K pair-tile ring depth
+constexpr int kVStages = 2;            // V pair-tile ring depth
+constexpr uint32_t kTmemCols = 512;    // slot s: S/P at columns [128 s, 128 s + 128), O at 256 + s D
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logits: rescale O only when the row max grows by more
 constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
 
@@ -46,21 +50,21 @@ struct SmemMap {
     static constexpr uint32_t kQSub = 128 * 128;              // 128 rows x 64 features (128 B)
     static constexpr uint32_t kQSlot = kQSub * (D / 64);
     static constexpr uint32_t kQ = 0;
-    static constexpr uint32_t kPSlot = 128 * 128;             // 128 rows x 64 keys bf16
-    static constexpr uint32_t kP = kQ + 2 * kQSlot;
-    static constexpr uint32_t kKVSub = 64 * 128;              // 64 keys x 64 features
-    static constexpr uint32_t kKTile = kKVSub * (D / 64);
-    static constexpr uint32_t kStage = 2 * kKTile;            // K then V
-    static constexpr uint32_t kKV = kP + 2 * kPSlot;
-    static constexpr uint32_t kBars = kKV + kStages * kStage;
+    static constexpr uint32_t kBlkSub = 64 * 128;             // one block: 64 keys x 64 features
+    static constexpr uint32_t kPairSub = 2 * kBlkSub;         // two blocks stacked: 128 keys x 64 features
+    static constexpr uint32_t kPairTile = kPairSub * (D / 64);
+    static constexpr uint32_t kK = kQ + 2 * kQSlot;
+    static constexpr uint32_t kV = kK + kKStages * kPairTile;
+    static constexpr uint32_t kBars = kV + kVStages * kPairTile;
     static constexpr uint32_t kTotal = kBars + 256;
     static constexpr uint32_t kAlloc = kTotal + 1024;         // slack for 1024-byte alignment
 };
 
 // Barrier slots inside the barrier area (8 bytes each).
 enum : uint32_t {
-    BAR_Q_FULL = 0, BAR_Q_EMPTY = 1, BAR_KV_FULL = 2, BAR_KV_EMPTY = 2 + kStages,
-    BAR_S_FULL = 2 + 2 * kStages, BAR_P_FULL = BAR_S_FULL + 4, BAR_O_DONE = BAR_P_FULL + 2,
+    BAR_Q_FULL = 0, BAR_Q_EMPTY = 1, BAR_K_FULL = 2, BAR_K_EMPTY = BAR_K_FULL + kKStages,
+    BAR_V_FULL = BAR_K_EMPTY + kKStages, BAR_V_EMPTY = BAR_V_FULL + kVStages,
+    BAR_S_FULL = BAR_V_EMPTY + kVStages, BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2,
     BAR_COUNT = BAR_O_DONE + 2
 };
 
@@ -123,13 +127,16 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     if (threadIdx.x == 0) {
         ptx::mbar_init(bar(BAR_Q_FULL), 1);
         ptx::mbar_init(bar(BAR_Q_EMPTY), 1);
-        for (int s = 0; s < kStages; ++s) {
-            ptx::mbar_init(bar(BAR_KV_FULL + s), 1);
-            ptx::mbar_init(bar(BAR_KV_EMPTY + s), 1);
+        for (int s = 0; s < kKStages; ++s) {
+            ptx::mbar_init(bar(BAR_K_FULL + s), 1);
+            ptx::mbar_init(bar(BAR_K_EMPTY + s), 1);
+        }
+        for (int s = 0; s < kVStages; ++s) {
+            ptx::mbar_init(bar(BAR_V_FULL + s), 1);
+            ptx::mbar_init(bar(BAR_V_EMPTY + s), 1);
         }
         for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(bar(BAR_S_FULL + 2 * s), 1);
-            ptx::mbar_init(bar(BAR_S_FULL + 2 * s + 1), 1);
+            ptx::mbar_init(bar(BAR_S_FULL + s), 1);
             ptx::mbar_init(bar(BAR_P_FULL + s), 128);
             ptx::mbar_init(bar(BAR_O_DONE + s), 1);
         }
@@ -152,7 +159,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::prefetch_tensormap(&tmQ);
             ptx::prefetch_tensormap(&tmK);
             ptx::prefetch_tensormap(&tmV);
-            uint32_t kvc = 0, ul = 0;
+            uint32_t pc = 0, ul = 0;  // pair steps and units issued so far by this CTA
             bool ok = true;
             for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
                 const Unit w = decode_unit(a, u);
@@ -165,33 +172,40 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         ptx::tma_load_4d(smem_base + SM::kQ + s * SM::kQSlot + dh * SM::kQSub, &tmQ,
                                          bar(BAR_Q_FULL), dh * 64, w.i * kBlk,
                                          w.hk * a.G + w.sub * 4 + 2 * s, w.b);
-                for (int t = 0; t < w.n; ++t, ++kvc) {
-                    const int32_t j = __ldg(a.col_idx + w.rs + t);
-                    const uint32_t st = kvc % kStages;
-                    if (kvc >= (uint32_t)kStages) {
-                        ok = wait_bar(bar(BAR_KV_EMPTY + st), (kvc / kStages - 1) & 1, abort_flag,
-                                      a.status, 2);
+                const int np = (w.n + 1) >> 1;
+                for (int tp = 0; tp < np; ++tp, ++pc) {
+                    const int nb = w.n - 2 * tp >= 2 ? 2 : 1;
+                    const int32_t j0 = __ldg(a.col_idx + w.rs + 2 * tp);
+                    const int32_t j1 = nb == 2 ? __ldg(a.col_idx + w.rs + 2 * tp + 1) : 0;
+                    // K pair tile: [feature half][key 0..127][64 features]; block h fills keys 64 h ..
+                    const uint32_t ks = pc % kKStages, vs = pc % kVStages;
+                    if (pc >= (uint32_t)kKStages) {
+                        ok = wait_bar(bar(BAR_K_EMPTY + ks), (pc / kKStages - 1) & 1, abort_flag, a.status, 2);
                         if (!ok) break;
                     }
-                    const uint32_t dst = smem_base + SM::kKV + st * SM::kStage;
-                    ptx::mbar_expect_tx(bar(BAR_KV_FULL + st), SM::kStage);
-                    for (int dh = 0; dh < DH; ++dh)
-                        ptx::tma_load_4d(dst + dh * SM::kKVSub, &tmK, bar(BAR_KV_FULL + st), dh * 64,
-                                         j * kBlk, w.hk, w.b);
-                    for (int dh = 0; dh < DH; ++dh)
-                        ptx::tma_load_4d(dst + SM::kKTile + dh * SM::kKVSub, &tmV,
-                                         bar(BAR_KV_FULL + st), dh * 64, j * kBlk, w.hk, w.b);
+                    const uint32_t kdst = smem_base + SM::kK + ks * SM::kPairTile;
+                    ptx::mbar_expect_tx(bar(BAR_K_FULL + ks), nb * DH * SM::kBlkSub);
+                    for (int h = 0; h < nb; ++h)
+                        for (int dh = 0; dh < DH; ++dh)
+                            ptx::tma_load_4d(kdst + dh * SM::kPairSub + h * SM::kBlkSub, &tmK, bar(BAR_K_FULL + ks),
+                                             dh * 64, (h ? j1 : j0) * kBlk, w.hk, w.b);
+                    if (pc >= (uint32_t)kVStages) {
+                        ok = wait_bar(bar(BAR_V_EMPTY + vs), (pc / kVStages - 1) & 1, abort_flag, a.status, 3);
+                        if (!ok) break;
+                    }
+                    const uint32_t vdst = smem_base + SM::kV + vs * SM::kPairTile;
+                    ptx::mbar_expect_tx(bar(BAR_V_FULL + vs), nb * DH * SM::kBlkSub);
+                    for (int h = 0; h < nb; ++h)
+                        for (int dh = 0; dh < DH; ++dh)
+                            ptx::tma_load_4d(vdst + dh * SM::kPairSub + h * SM::kBlkSub, &tmV, bar(BAR_V_FULL + vs),
+                                             dh * 64, (h ? j1 : j0) * kBlk, w.hk, w.b);
                 }
                 ++ul;
             }
             if (!ok) {
                 // Drain: give copies already in flight a bounded chance to land before exit.
-                const uint32_t first = kvc > (uint32_t)kStages ? kvc - kStages : 0;
-                for (uint32_t c = first; c < kvc; ++c) {
-                    const long long t0 = clock64();
-                    while (!ptx::mbar_try_wait(bar(BAR_KV_FULL + c % kStages), (c / kStages) & 1) &&
-                           clock64() - t0 < 2000000ll) {
-                    }
+                const long long t0 = clock64();
+                while (clock64() - t0 < 4000000ll) {
                 }
             }
         }
@@ -204,91 +218,95 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         // the start address >> 4 (plus the leading-dimension offset for the MN-major V operand).
         {
             const bool leader = ptx::elect_one();
-            constexpr uint32_t idesc_qk = ptx::idesc_bf16_f32(128, 64, 0);
+            constexpr uint32_t idesc_qk2 = ptx::idesc_bf16_f32(128, 128, 0);
+            constexpr uint32_t idesc_qk1 = ptx::idesc_bf16_f32(128, 64, 0);
             constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(128, D, 1);
             constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
             const uint32_t q_lo = ((smem_base + SM::kQ) >> 4) | (1u << 16);
-            const uint32_t p_lo = ((smem_base + SM::kP) >> 4) | (1u << 16);
-            const uint32_t k_lo = ((smem_base + SM::kKV) >> 4) | (1u << 16);
-            const uint32_t v_lo = ((smem_base + SM::kKV + SM::kKTile) >> 4) | ((SM::kKVSub >> 4) << 16);
-            // S_s = Q_s K^T: A = Q tile (K-major), B = K block (K-major), 16 features per MMA.
-            auto issue_qk = [&](int s, uint32_t buf, uint32_t st) {
+            const uint32_t k_lo = ((smem_base + SM::kK) >> 4) | (1u << 16);
+            const uint32_t v_lo = ((smem_base + SM::kV) >> 4) | ((SM::kPairSub >> 4) << 16);
+            // S_s = Q_s K^T: A = Q tile (K-major), B = K pair tile (K-major, 64 nb keys),
+            // 16 features per MMA.
+            auto issue_qk = [&](int s, uint32_t ks, int nb) {
                 const uint32_t qa = q_lo + s * (SM::kQSlot >> 4);
-                const uint32_t kb = k_lo + st * (SM::kStage >> 4);
-                const uint32_t dst = tmem_base + (2 * s + buf) * 64;
+                const uint32_t kb = k_lo + ks * (SM::kPairTile >> 4);
+                const uint32_t dst = tmem_base + s * 128;
+                const uint32_t idesc = nb == 2 ? idesc_qk2 : idesc_qk1;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk)
                     ptx::umma_ss_lohi(dst, qa + (((kk / 4) * SM::kQSub + (kk % 4) * 32) >> 4), desc_hi,
-                                      kb + (((kk / 4) * SM::kKVSub + (kk % 4) * 32) >> 4), desc_hi, idesc_qk,
+                                      kb + (((kk / 4) * SM::kPairSub + (kk % 4) * 32) >> 4), desc_hi, idesc,
                                       kk > 0 ? 1u : 0u);
             };
-            // O_s (+)= P_s V: A = P tile (K-major over keys), B = V block (MN-major: features
-            // contiguous), 16 keys per MMA.
-            auto issue_pv = [&](int s, uint32_t st, bool acc) {
-                const uint32_t pa_ = p_lo + s * (SM::kPSlot >> 4);
-                const uint32_t vb = v_lo + st * (SM::kStage >> 4);
+            // O_s (+)= P_s V: A = P (tensor memory, bf16 pairs in the first 32 nb columns of the
+            // slot's S region), B = V pair tile (MN-major: features contiguous), 16 keys per MMA.
+            auto issue_pv = [&](int s, uint32_t vs, int nb, bool acc) {
+                const uint32_t vb = v_lo + vs * (SM::kPairTile >> 4);
                 const uint32_t dst = tmem_base + 256 + s * D;
+                const uint32_t pa_ = tmem_base + s * 128;
 #pragma unroll
-                for (int kk = 0; kk < kBlk / 16; ++kk)
-                    ptx::umma_ss_lohi(dst, pa_ + ((kk * 32) >> 4), desc_hi, vb + ((kk * 2048) >> 4), desc_hi,
-                                      idesc_pv, (acc || kk > 0) ? 1u : 0u);
+                for (int kk = 0; kk < 8; ++kk)
+                    if (kk < 4 * nb)
+                        ptx::umma_ts_lohi(dst, pa_ + kk * 8, vb + ((kk * 2048) >> 4), desc_hi, idesc_pv,
+                                          (acc || kk > 0) ? 1u : 0u);
             };
-            uint32_t kvc = 0, ul = 0, g = 0;
+            uint32_t pc = 0, ul = 0;
             bool ok = true;
             for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
                 const Unit w = decode_unit(a, u);
                 if (w.n <= 0) continue;
-                ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 3));
+                const int np = (w.n + 1) >> 1;
+                ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 4));
                 if (!ok) break;
-                // Prologue: S of the first two steps (S is double-buffered per slot).
-                for (int t0 = 0; t0 < 2 && t0 < w.n && ok; ++t0) {
-                    const uint32_t c0 = kvc + t0;
-                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_KV_FULL + c0 % kStages), (c0 / kStages) & 1,
-                                                          abort_flag, a.status, 4));
-                    if (!ok) break;
-                    ptx::tc_fence_after_sync();
-                    if (leader) {
-                        for (int s = 0; s < 2; ++s) {
-                            issue_qk(s, (g + t0) & 1, c0 % kStages);
-                            ptx::umma_commit(bar(BAR_S_FULL + 2 * s + ((g + t0) & 1)));
-                        }
-                    }
-                    __syncwarp();
-                }
+                ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + pc % kKStages), (pc / kKStages) & 1,
+                                                      abort_flag, a.status, 5));
                 if (!ok) break;
-                if (w.n <= 2 && leader) ptx::umma_commit(bar(BAR_Q_EMPTY));
-                for (int t = 0; t < w.n && ok; ++t) {
-                    const uint32_t st = (kvc + t) % kStages;
+                ptx::tc_fence_after_sync();
+                if (leader) {
+                    const int nb0 = w.n >= 2 ? 2 : 1;
                     for (int s = 0; s < 2; ++s) {
-                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + s), (g + t) & 1, abort_flag, a.status, 5));
+                        issue_qk(s, pc % kKStages, nb0);
+                        ptx::umma_commit(bar(BAR_S_FULL + s));
+                    }
+                    ptx::umma_commit(bar(BAR_K_EMPTY + pc % kKStages));
+                    if (np == 1) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                }
+                __syncwarp();
+                for (int tp = 0; tp < np && ok; ++tp) {
+                    const uint32_t c = pc + tp;
+                    const int nb = w.n - 2 * tp >= 2 ? 2 : 1;
+                    const int nb1 = w.n - 2 * (tp + 1) >= 2 ? 2 : 1;
+                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_V_FULL + c % kVStages), (c / kVStages) & 1,
+                                                          abort_flag, a.status, 6));
+                    if (!ok) break;
+                    for (int s = 0; s < 2; ++s) {
+                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + s), c & 1, abort_flag, a.status, 7));
                         if (!ok) break;
+                        if (tp + 1 < np && s == 0) {
+                            ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + (c + 1) % kKStages),
+                                                                  ((c + 1) / kKStages) & 1, abort_flag, a.status, 8));
+                            if (!ok) break;
+                        }
                         ptx::tc_fence_after_sync();
                         if (leader) {
-                            issue_pv(s, st, t > 0);
-                            ptx::umma_commit(bar(BAR_O_DONE + s));
-                            if (s == 1) ptx::umma_commit(bar(BAR_KV_EMPTY + st));
+                            issue_pv(s, c % kVStages, nb, tp > 0);
+                            if (tp + 1 == np) ptx::umma_commit(bar(BAR_O_DONE + s));
+                            if (s == 1) ptx::umma_commit(bar(BAR_V_EMPTY + c % kVStages));
+                            if (tp + 1 < np) {
+                                // The next S overwrites this slot's S/P columns; MMAs of one
+                                // issuer execute in order, so P has been consumed by then.
+                                issue_qk(s, (c + 1) % kKStages, nb1);
+                                ptx::umma_commit(bar(BAR_S_FULL + s));
+                                if (s == 1) {
+                                    ptx::umma_commit(bar(BAR_K_EMPTY + (c + 1) % kKStages));
+                                    if (tp + 2 == np) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                                }
+                            }
                         }
                         __syncwarp();
-                        if (t + 2 < w.n) {
-                            // S buffer (g + t) & 1 of this slot was consumed by the softmax of step t.
-                            const uint32_t c2 = kvc + t + 2;
-                            if (s == 0) {
-                                ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_KV_FULL + c2 % kStages),
-                                                                      (c2 / kStages) & 1, abort_flag, a.status, 6));
-                                if (!ok) break;
-                                ptx::tc_fence_after_sync();
-                            }
-                            if (leader) {
-                                issue_qk(s, (g + t) & 1, c2 % kStages);
-                                ptx::umma_commit(bar(BAR_S_FULL + 2 * s + ((g + t) & 1)));
-                                if (s == 1 && t + 3 == w.n) ptx::umma_commit(bar(BAR_Q_EMPTY));
-                            }
-                            __syncwarp();
-                        }
                     }
                 }
-                kvc += w.n;
-                g += w.n;
+                pc += np;
                 ++ul;
             }
         }
@@ -299,11 +317,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const int quad = warp & 3;              // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;       // tile row = TMEM lane
         const int qrow = row & 63;              // token inside the query block
-        const uint32_t t_s0 = tmem_base + ((uint32_t)(quad * 32) << 16) + 2 * s * 64;
+        const uint32_t t_s = tmem_base + ((uint32_t)(quad * 32) << 16) + s * 128;
         const uint32_t t_o = tmem_base + ((uint32_t)(quad * 32) << 16) + 256 + s * D;
-        uint8_t *p_row = smem + SM::kP + s * SM::kPSlot + row * 128;
         const float sl2 = a.scale_log2;
-        uint32_t g = 0;
+        uint32_t pc = 0, ul = 0;
         bool ok = true;
         for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
             const Unit w = decode_unit(a, u);
@@ -311,81 +328,86 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const int head = w.hk * a.G + head_local;
             const int64_t tok = (int64_t)w.i * kBlk + qrow;
             const bool valid = head_local < a.G && tok < a.N;
+            const int np = (w.n + 1) >> 1;
             float m = -INFINITY, l = 0.f;
-            for (int t = 0; t < w.n; ++t, ++g) {
-                const int32_t j = __ldg(a.col_idx + w.rs + t);
-                ok = wait_bar(bar(BAR_S_FULL + 2 * s + (g & 1)), (g >> 1) & 1, abort_flag, a.status, 7);
+            for (int tp = 0; tp < np; ++tp, ++pc) {
+                const int nb = w.n - 2 * tp >= 2 ? 2 : 1;
+                // Algorithm 1's causal term acts inside the diagonal pair (col == row) only.
+                const bool diag0 = __ldg(a.col_idx + w.rs + 2 * tp) == w.i;
+                const bool diag1 = nb == 2 && __ldg(a.col_idx + w.rs + 2 * tp + 1) == w.i;
+                ok = wait_bar(bar(BAR_S_FULL + s), pc & 1, abort_flag, a.status, 9);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                uint32_t sr[64];
-                const uint32_t t_s = t_s0 + (g & 1) * 64;
-                ptx::tmem_ld32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
-                ptx::tmem_ld32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
-                ptx::tmem_wait_ld();
-                // Algorithm 1's causal term acts inside the diagonal pair only.
-                if (j == w.i) {
+                // Pass 1: row maximum over the 64 nb logits.
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                for (int h = 0; h < nb; ++h) {
+                    uint32_t sr[64];
+                    ptx::tmem_ld32(t_s + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+                    ptx::tmem_ld32(t_s + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+                    ptx::tmem_wait_ld();
+                    if (h ? diag1 : diag0) {
 #pragma unroll
-                    for (int c = 0; c < 64; ++c)
-                        if (c > qrow) sr[c] = 0xff800000u;  // -inf
-                }
-                float mx4[4] = {__uint_as_float(sr[0]), __uint_as_float(sr[1]), __uint_as_float(sr[2]),
-                                __uint_as_float(sr[3])};
+                        for (int c = 0; c < 64; ++c)
+                            if (c > qrow) sr[c] = 0xff800000u;  // -inf
+                    }
 #pragma unroll
-                for (int c = 4; c < 64; c += 4) {
+                    for (int c = 0; c < 64; c += 4) {
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) mx4[e] = fmaxf(mx4[e], __uint_as_float(sr[c + e]));
+                        for (int e = 0; e < 4; ++e) mx4[e] = fmaxf(mx4[e], __uint_as_float(sr[c + e]));
+                    }
                 }
                 const float mx2 = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
                 // Lazy rescaling: keep the old reference max unless the row max grew by more than
                 // the threshold; exp2(s - m) then stays below 2^threshold, and O / l at the end is
                 // exact whatever reference was used.
-                const bool grow = t == 0 || mx2 > m + kRescaleThreshold;
+                const bool grow = tp == 0 || mx2 > m + kRescaleThreshold;
                 const float m_new = grow ? mx2 : m;
                 const float alpha = grow ? ptx::ex2(m - m_new) : 1.0f;
+                if (tp > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
+                    // O_s is quiescent: the S just waited for was issued after the previous P V.
+#pragma unroll
+                    for (int ch = 0; ch < D / 32; ++ch) {
+                        uint32_t orr[32];
+                        ptx::tmem_ld32(t_o + ch * 32, orr);
+                        ptx::tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                        ptx::tmem_st32(t_o + ch * 32, orr);
+                    }
+                }
+                // Pass 2: P = exp2(s - m) as bf16 pairs into the first columns of the S region
+                // (block h -> columns [32 h, 32 h + 32)); row sum from the unrounded values.
                 float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-                uint32_t pk[32];
+                for (int h = 0; h < nb; ++h) {
+                    uint32_t sr[64];
+                    ptx::tmem_ld32(t_s + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+                    ptx::tmem_ld32(t_s + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+                    ptx::tmem_wait_ld();
+                    if (h ? diag1 : diag0) {
 #pragma unroll
-                for (int c = 0; c < 64; c += 4) {
-                    float pv[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        pv[e] = ptx::ex2(fmaf(__uint_as_float(sr[c + e]), sl2, -m_new));
-                        sum4[e] += pv[e];
+                        for (int c = 0; c < 64; ++c)
+                            if (c > qrow) sr[c] = 0xff800000u;  // -inf
                     }
-                    const __nv_bfloat162 h01 = __floats2bfloat162_rn(pv[0], pv[1]);
-                    const __nv_bfloat162 h23 = __floats2bfloat162_rn(pv[2], pv[3]);
-                    pk[c >> 1] = *reinterpret_cast<const uint32_t *>(&h01);
-                    pk[(c >> 1) + 1] = *reinterpret_cast<const uint32_t *>(&h23);
-                }
-                const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-                l = l * alpha + sum;
-                m = m_new;
-                if (t > 0) {
-                    // P_s and O_s are free once the previous step's P V has completed.
-                    ok = wait_bar(bar(BAR_O_DONE + s), (g - 1) & 1, abort_flag, a.status, 8);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    ptx::tc_fence_after_sync();
-                    if (__any_sync(0xffffffffu, alpha != 1.0f)) {
+                    uint32_t pk[32];
 #pragma unroll
-                        for (int ch = 0; ch < D / 32; ++ch) {
-                            uint32_t orr[32];
-                            ptx::tmem_ld32(t_o + ch * 32, orr);
-                            ptx::tmem_wait_ld();
+                    for (int c = 0; c < 64; c += 4) {
+                        float pv[4];
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-                            ptx::tmem_st32(t_o + ch * 32, orr);
+                        for (int e = 0; e < 4; ++e) {
+                            pv[e] = ptx::ex2(fmaf(__uint_as_float(sr[c + e]), sl2, -m_new));
+                            sum4[e] += pv[e];
                         }
-                        ptx::tmem_wait_st();
+                        const __nv_bfloat162 h01 = __floats2bfloat162_rn(pv[0], pv[1]);
+                        const __nv_bfloat162 h23 = __floats2bfloat162_rn(pv[2], pv[3]);
+                        pk[c >> 1] = *reinterpret_cast<const uint32_t *>(&h01);
+                        pk[(c >> 1) + 1] = *reinterpret_cast<const uint32_t *>(&h23);
                     }
+                    ptx::tmem_st32(t_s + h * 32, pk);
                 }
-                // P row: 64 bf16 = eight 16-byte chunks, chunk c stored at c ^ (row % 8).
-#pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    *reinterpret_cast<uint4 *>(p_row + ((c ^ (row & 7)) << 4)) =
-                        make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-                ptx::fence_proxy_async_smem();
+                l = l * alpha + (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                m = m_new;
+                ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(bar(BAR_P_FULL + s));
             }
@@ -402,9 +424,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 continue;
             }
             // Epilogue: O / l and LSE = ln sum exp(s) = (m + log2 l) ln 2.
-            ok = wait_bar(bar(BAR_O_DONE + s), (g - 1) & 1, abort_flag, a.status, 9);
+            ok = wait_bar(bar(BAR_O_DONE + s), ul & 1, abort_flag, a.status, 10);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
+            ++ul;
             ptx::tc_fence_after_sync();
             const float inv = 1.0f / l;
             const int64_t obase = w.b * a.o_sb + tok * a.o_ss + (int64_t)head * a.o_sh;
