@@ -14,6 +14,7 @@
 //   warp 2      tensor-memory allocation
 //   warps 4-7   online softmax of slot 0 (thread = tile row = TMEM lane)
 //   warps 8-11  online softmax of slot 1
+// Warps 0-3 give registers back (setmaxnreg) and the softmax warpgroups take them.
 // The two slots alternate on the tensor pipe, so one slot's softmax overlaps the other's MMAs.
 // Every barrier wait is bounded; a wait that runs out records PA_ERR_TIMEOUT in the status
 // block, raises a CTA-wide abort flag and the CTA drains and exits (no trap, no endless spin).
@@ -27,7 +28,7 @@
 namespace pa {
 
 constexpr int kBlk = 64;               // tokens per query / key block
-constexpr int kThreads = 384;          // 12 warps
+constexpr int kThreads = 384;          // 12 warps: one control warpgroup, two softmax warpgroups
 constexpr int kKStages = 3;            // K pair-tile ring depth
 constexpr int kVStages = 2;            // V pair-tile ring depth
 constexpr uint32_t kTmemCols = 512;    // slot s: S/P at columns [128 s, 128 s + 128), O at 256 + s D
@@ -153,6 +154,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
+    if (warp < 4) ptx::setmaxnreg_dec<40>();
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -313,6 +315,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         __syncwarp();
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ online softmax
+        ptx::setmaxnreg_inc<232>();
         const int s = (warp - 4) >> 2;          // slot
         const int quad = warp & 3;              // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;       // tile row = TMEM lane
@@ -329,73 +332,43 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const int64_t tok = (int64_t)w.i * kBlk + qrow;
             const bool valid = head_local < a.G && tok < a.N;
             const int np = (w.n + 1) >> 1;
+            // Algorithm 1's causal term acts inside the diagonal pair (col == row) only; rows end
+            // with that block.
+            const bool last_is_diag = w.n > 0 && __ldg(a.col_idx + w.rs + w.n - 1) == w.i;
             float m = -INFINITY, l = 0.f;
             for (int tp = 0; tp < np; ++tp, ++pc) {
                 const int nb = w.n - 2 * tp >= 2 ? 2 : 1;
-                // Algorithm 1's causal term acts inside the diagonal pair (col == row) only.
-                const bool diag0 = __ldg(a.col_idx + w.rs + 2 * tp) == w.i;
-                const bool diag1 = nb == 2 && __ldg(a.col_idx + w.rs + 2 * tp + 1) == w.i;
                 ok = wait_bar(bar(BAR_S_FULL + s), pc & 1, abort_flag, a.status, 9);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                // Pass 1: row maximum over the 64 nb logits.
-                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                // One online-softmax step per 64-key half.  The exponentials are taken against the
+                // reference maximum m carried from earlier steps (lazy rescaling: m moves only when
+                // the row maximum exceeds it by more than the threshold, so exp2(s - m) stays below
+                // 2^threshold and O / l at the end is exact whatever reference was used).  The rare
+                // half whose maximum does move is recomputed from the logits still in registers.
                 for (int h = 0; h < nb; ++h) {
                     uint32_t sr[64];
                     ptx::tmem_ld32(t_s + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
                     ptx::tmem_ld32(t_s + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
                     ptx::tmem_wait_ld();
-                    if (h ? diag1 : diag0) {
+                    if (last_is_diag && 2 * tp + h == w.n - 1) {
 #pragma unroll
                         for (int c = 0; c < 64; ++c)
                             if (c > qrow) sr[c] = 0xff800000u;  // -inf
                     }
-#pragma unroll
-                    for (int c = 0; c < 64; c += 4) {
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) mx4[e] = fmaxf(mx4[e], __uint_as_float(sr[c + e]));
-                    }
-                }
-                const float mx2 = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
-                // Lazy rescaling: keep the old reference max unless the row max grew by more than
-                // the threshold; exp2(s - m) then stays below 2^threshold, and O / l at the end is
-                // exact whatever reference was used.
-                const bool grow = tp == 0 || mx2 > m + kRescaleThreshold;
-                const float m_new = grow ? mx2 : m;
-                const float alpha = grow ? ptx::ex2(m - m_new) : 1.0f;
-                if (tp > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
-                    // O_s is quiescent: the S just waited for was issued after the previous P V.
-#pragma unroll
-                    for (int ch = 0; ch < D / 32; ++ch) {
-                        uint32_t orr[32];
-                        ptx::tmem_ld32(t_o + ch * 32, orr);
-                        ptx::tmem_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-                        ptx::tmem_st32(t_o + ch * 32, orr);
-                    }
-                }
-                // Pass 2: P = exp2(s - m) as bf16 pairs into the first columns of the S region
-                // (block h -> columns [32 h, 32 h + 32)); row sum from the unrounded values.
-                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-                for (int h = 0; h < nb; ++h) {
-                    uint32_t sr[64];
-                    ptx::tmem_ld32(t_s + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
-                    ptx::tmem_ld32(t_s + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
-                    ptx::tmem_wait_ld();
-                    if (h ? diag1 : diag0) {
-#pragma unroll
-                        for (int c = 0; c < 64; ++c)
-                            if (c > qrow) sr[c] = 0xff800000u;  // -inf
-                    }
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
                     uint32_t pk[32];
+                    const float neg_m = -m;
 #pragma unroll
                     for (int c = 0; c < 64; c += 4) {
                         float pv[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            pv[e] = ptx::ex2(fmaf(__uint_as_float(sr[c + e]), sl2, -m_new));
+                            const float x = __uint_as_float(sr[c + e]);
+                            mx4[e] = fmaxf(mx4[e], x);
+                            pv[e] = ptx::ex2(fmaf(x, sl2, neg_m));
                             sum4[e] += pv[e];
                         }
                         const __nv_bfloat162 h01 = __floats2bfloat162_rn(pv[0], pv[1]);
@@ -403,10 +376,60 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         pk[c >> 1] = *reinterpret_cast<const uint32_t *>(&h01);
                         pk[(c >> 1) + 1] = *reinterpret_cast<const uint32_t *>(&h23);
                     }
+                    const float mx2 = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
+                    const bool first = tp == 0 && h == 0;
+                    const bool grow = first || mx2 > m + kRescaleThreshold;
+                    if (__any_sync(0xffffffffu, grow)) {
+                        const float m_new = grow ? mx2 : m;
+                        const float alpha = grow ? ptx::ex2(m - m_new) : 1.0f;  // 0 on the first half
+                        l *= alpha;
+                        m = m_new;
+                        if (tp > 0) {
+                            // O_s is quiescent: the S just waited for was issued after the previous P V.
+#pragma unroll 1
+                            for (int ch = 0; ch < D / 32; ++ch) {
+                                uint32_t orr[32];
+                                ptx::tmem_ld32(t_o + ch * 32, orr);
+                                ptx::tmem_wait_ld();
+#pragma unroll
+                                for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                                ptx::tmem_st32(t_o + ch * 32, orr);
+                            }
+                        }
+                        if (h == 1) {
+                            // The first half's P of this step is already stored: bring it to the new reference.
+                            uint32_t pr[32];
+                            ptx::tmem_ld32(t_s, pr);
+                            ptx::tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) {
+                                const float lo = __uint_as_float(pr[c] << 16) * alpha;
+                                const float hi = __uint_as_float(pr[c] & 0xffff0000u) * alpha;
+                                const __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
+                                pr[c] = *reinterpret_cast<const uint32_t *>(&h2);
+                            }
+                            ptx::tmem_st32(t_s, pr);
+                        }
+                        sum4[0] = sum4[1] = sum4[2] = sum4[3] = 0.f;
+#pragma unroll
+                        for (int c = 0; c < 64; c += 4) {
+                            float pv[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                pv[e] = ptx::ex2(fmaf(__uint_as_float(sr[c + e]), sl2, -m));
+                                sum4[e] += pv[e];
+                            }
+                            const __nv_bfloat162 h01 = __floats2bfloat162_rn(pv[0], pv[1]);
+                            const __nv_bfloat162 h23 = __floats2bfloat162_rn(pv[2], pv[3]);
+                            pk[c >> 1] = *reinterpret_cast<const uint32_t *>(&h01);
+                            pk[(c >> 1) + 1] = *reinterpret_cast<const uint32_t *>(&h23);
+                        }
+                    }
+                    l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                    // P (bf16 pairs) goes to the first columns of the S region: half h -> [32 h, 32 h + 32).
+                    // Half 0 overwrites logits that were just read; half 1's logits sit at [64, 128).
                     ptx::tmem_st32(t_s + h * 32, pk);
                 }
-                l = l * alpha + (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-                m = m_new;
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(bar(BAR_P_FULL + s));
