@@ -4,18 +4,16 @@
 // One persistent CTA per SM walks work units (batch, KV head, query block, head quad).  A unit
 // holds two 128-row tiles ("slots"); a tile stacks two query heads of the KV group on the 64
 // tokens of the query block (the mask does not depend on the head, so they share the key list
-// and the K/V tiles).  The key list is walked two blocks at a time: the gathered blocks are put
-// side by side in shared memory so that S = Q K^T runs with N = 128 and O += P V with K = 128
-// (a row of odd length ends with a single-block step, N = 64).  Warp roles:
+// and the K/V tiles).  The key list is walked one 64-key block per step.  Warp roles:
 //   warp 0      TMA producer: Q tiles once per unit, then the listed K and V blocks, gathered by
-//               block index, into two rings of shared-memory pair tiles (128-byte swizzle)
-//   warp 1      tcgen05 issuer: S = Q K^T into tensor memory; O += P V with P read from tensor
-//               memory (it overlays the S columns it was computed from)
+//               block index, into two rings of shared-memory tiles (128-byte swizzle)
+//   warp 1      tcgen05 issuer: S = Q K^T into tensor memory (two S buffers per slot, so the
+//               logits of step t+1 are ready while the softmax works on step t); O += P V with
+//               P read from tensor memory (it overlays the S buffer it was computed from)
 //   warp 2      tensor-memory allocation
 //   warps 4-7   online softmax of slot 0 (thread = tile row = TMEM lane)
 //   warps 8-11  online softmax of slot 1
 // Warps 0-3 give registers back (setmaxnreg) and the softmax warpgroups take them.
-// The two slots alternate on the tensor pipe, so one slot's softmax overlaps the other's MMAs.
 // Every barrier wait is bounded; a wait that runs out records PA_ERR_TIMEOUT in the status
 // block, raises a CTA-wide abort flag and the CTA drains and exits (no trap, no endless spin).
 #include <cuda.h>
@@ -29,9 +27,9 @@ namespace pa {
 
 constexpr int kBlk = 64;               // tokens per query / key block
 constexpr int kThreads = 384;          // 12 warps: one control warpgroup, two softmax warpgroups
-constexpr int kKStages = 3;            // K pair-tile ring depth
-constexpr int kVStages = 2;            // V pair-tile ring depth
-constexpr uint32_t kTmemCols = 512;    // slot s: S/P at columns [128 s, 128 s + 128), O at 256 + s D
+constexpr int kKStages = 5;            // K block ring depth
+constexpr int kVStages = 5;            // V block ring depth
+constexpr uint32_t kTmemCols = 512;    // slot s: S/P buffers at columns 128 s + 64 b, O at 256 + s D
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logits: rescale O only when the row max grows by more
 constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
 
@@ -51,12 +49,11 @@ struct SmemMap {
     static constexpr uint32_t kQSub = 128 * 128;              // 128 rows x 64 features (128 B)
     static constexpr uint32_t kQSlot = kQSub * (D / 64);
     static constexpr uint32_t kQ = 0;
-    static constexpr uint32_t kBlkSub = 64 * 128;             // one block: 64 keys x 64 features
-    static constexpr uint32_t kPairSub = 2 * kBlkSub;         // two blocks stacked: 128 keys x 64 features
-    static constexpr uint32_t kPairTile = kPairSub * (D / 64);
+    static constexpr uint32_t kBlkSub = 64 * 128;             // 64 keys x 64 features
+    static constexpr uint32_t kBlkTile = kBlkSub * (D / 64);  // one K or V block
     static constexpr uint32_t kK = kQ + 2 * kQSlot;
-    static constexpr uint32_t kV = kK + kKStages * kPairTile;
-    static constexpr uint32_t kBars = kV + kVStages * kPairTile;
+    static constexpr uint32_t kV = kK + kKStages * kBlkTile;
+    static constexpr uint32_t kBars = kV + kVStages * kBlkTile;
     static constexpr uint32_t kTotal = kBars + 256;
     static constexpr uint32_t kAlloc = kTotal + 1024;         // slack for 1024-byte alignment
 };
@@ -65,8 +62,8 @@ struct SmemMap {
 enum : uint32_t {
     BAR_Q_FULL = 0, BAR_Q_EMPTY = 1, BAR_K_FULL = 2, BAR_K_EMPTY = BAR_K_FULL + kKStages,
     BAR_V_FULL = BAR_K_EMPTY + kKStages, BAR_V_EMPTY = BAR_V_FULL + kVStages,
-    BAR_S_FULL = BAR_V_EMPTY + kVStages, BAR_P_FULL = BAR_S_FULL + 2, BAR_O_DONE = BAR_P_FULL + 2,
-    BAR_COUNT = BAR_O_DONE + 2
+    BAR_S_FULL = BAR_V_EMPTY + kVStages,  // [slot][buffer]
+    BAR_P_FULL = BAR_S_FULL + 4, BAR_O_DONE = BAR_P_FULL + 2, BAR_COUNT = BAR_O_DONE + 2
 };
 
 struct Unit {
@@ -136,8 +133,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::mbar_init(bar(BAR_V_FULL + s), 1);
             ptx::mbar_init(bar(BAR_V_EMPTY + s), 1);
         }
+        for (int s = 0; s < 4; ++s) ptx::mbar_init(bar(BAR_S_FULL + s), 1);
         for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(bar(BAR_S_FULL + s), 1);
             ptx::mbar_init(bar(BAR_P_FULL + s), 128);
             ptx::mbar_init(bar(BAR_O_DONE + s), 1);
         }
@@ -161,7 +158,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::prefetch_tensormap(&tmQ);
             ptx::prefetch_tensormap(&tmK);
             ptx::prefetch_tensormap(&tmV);
-            uint32_t pc = 0, ul = 0;  // pair steps and units issued so far by this CTA
+            uint32_t kc = 0, ul = 0;  // key blocks and units issued so far by this CTA
             bool ok = true;
             for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
                 const Unit w = decode_unit(a, u);
@@ -174,33 +171,25 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         ptx::tma_load_4d(smem_base + SM::kQ + s * SM::kQSlot + dh * SM::kQSub, &tmQ,
                                          bar(BAR_Q_FULL), dh * 64, w.i * kBlk,
                                          w.hk * a.G + w.sub * 4 + 2 * s, w.b);
-                const int np = (w.n + 1) >> 1;
-                for (int tp = 0; tp < np; ++tp, ++pc) {
-                    const int nb = w.n - 2 * tp >= 2 ? 2 : 1;
-                    const int32_t j0 = __ldg(a.col_idx + w.rs + 2 * tp);
-                    const int32_t j1 = nb == 2 ? __ldg(a.col_idx + w.rs + 2 * tp + 1) : 0;
-                    // K pair tile: [feature half][key 0..127][64 features]; block h fills keys 64 h ..
-                    const uint32_t ks = pc % kKStages, vs = pc % kVStages;
-                    if (pc >= (uint32_t)kKStages) {
-                        ok = wait_bar(bar(BAR_K_EMPTY + ks), (pc / kKStages - 1) & 1, abort_flag, a.status, 2);
+                for (int t = 0; t < w.n; ++t, ++kc) {
+                    const int32_t j = __ldg(a.col_idx + w.rs + t);
+                    const uint32_t ks = kc % kKStages, vs = kc % kVStages;
+                    if (kc >= (uint32_t)kKStages) {
+                        ok = wait_bar(bar(BAR_K_EMPTY + ks), (kc / kKStages - 1) & 1, abort_flag, a.status, 2);
                         if (!ok) break;
                     }
-                    const uint32_t kdst = smem_base + SM::kK + ks * SM::kPairTile;
-                    ptx::mbar_expect_tx(bar(BAR_K_FULL + ks), nb * DH * SM::kBlkSub);
-                    for (int h = 0; h < nb; ++h)
-                        for (int dh = 0; dh < DH; ++dh)
-                            ptx::tma_load_4d(kdst + dh * SM::kPairSub + h * SM::kBlkSub, &tmK, bar(BAR_K_FULL + ks),
-                                             dh * 64, (h ? j1 : j0) * kBlk, w.hk, w.b);
-                    if (pc >= (uint32_t)kVStages) {
-                        ok = wait_bar(bar(BAR_V_EMPTY + vs), (pc / kVStages - 1) & 1, abort_flag, a.status, 3);
+                    ptx::mbar_expect_tx(bar(BAR_K_FULL + ks), SM::kBlkTile);
+                    for (int dh = 0; dh < DH; ++dh)
+                        ptx::tma_load_4d(smem_base + SM::kK + ks * SM::kBlkTile + dh * SM::kBlkSub, &tmK,
+                                         bar(BAR_K_FULL + ks), dh * 64, j * kBlk, w.hk, w.b);
+                    if (kc >= (uint32_t)kVStages) {
+                        ok = wait_bar(bar(BAR_V_EMPTY + vs), (kc / kVStages - 1) & 1, abort_flag, a.status, 3);
                         if (!ok) break;
                     }
-                    const uint32_t vdst = smem_base + SM::kV + vs * SM::kPairTile;
-                    ptx::mbar_expect_tx(bar(BAR_V_FULL + vs), nb * DH * SM::kBlkSub);
-                    for (int h = 0; h < nb; ++h)
-                        for (int dh = 0; dh < DH; ++dh)
-                            ptx::tma_load_4d(vdst + dh * SM::kPairSub + h * SM::kBlkSub, &tmV, bar(BAR_V_FULL + vs),
-                                             dh * 64, (h ? j1 : j0) * kBlk, w.hk, w.b);
+                    ptx::mbar_expect_tx(bar(BAR_V_FULL + vs), SM::kBlkTile);
+                    for (int dh = 0; dh < DH; ++dh)
+                        ptx::tma_load_4d(smem_base + SM::kV + vs * SM::kBlkTile + dh * SM::kBlkSub, &tmV,
+                                         bar(BAR_V_FULL + vs), dh * 64, j * kBlk, w.hk, w.b);
                 }
                 ++ul;
             }
@@ -215,100 +204,97 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     } else if (warp == 1) {
         // ------------------------------------------------------------------ tcgen05 issuer
         // The whole warp runs the (uniform) control flow and the barrier waits; one elected lane
-        // issues the MMAs and commits.  Descriptors: the high word is constant per operand kind
-        // (stride 1024 B between 8-row groups, version 1, 128-byte swizzle); the low word holds
-        // the start address >> 4 (plus the leading-dimension offset for the MN-major V operand).
+        // issues the MMAs and commits.  MMAs of one issuer execute in issue order, which is what
+        // lets the S of step t+2 overwrite the buffer whose P was read by the P V of step t.
+        // Descriptors: the high word is constant per operand kind (stride 1024 B between 8-row
+        // groups, version 1, 128-byte swizzle); the low word holds the start address >> 4 (plus
+        // the leading-dimension offset for the MN-major V operand).
         {
             const bool leader = ptx::elect_one();
-            constexpr uint32_t idesc_qk2 = ptx::idesc_bf16_f32(128, 128, 0);
-            constexpr uint32_t idesc_qk1 = ptx::idesc_bf16_f32(128, 64, 0);
+            constexpr uint32_t idesc_qk = ptx::idesc_bf16_f32(128, 64, 0);
             constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(128, D, 1);
             constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
             const uint32_t q_lo = ((smem_base + SM::kQ) >> 4) | (1u << 16);
             const uint32_t k_lo = ((smem_base + SM::kK) >> 4) | (1u << 16);
-            const uint32_t v_lo = ((smem_base + SM::kV) >> 4) | ((SM::kPairSub >> 4) << 16);
-            // S_s = Q_s K^T: A = Q tile (K-major), B = K pair tile (K-major, 64 nb keys),
-            // 16 features per MMA.
-            auto issue_qk = [&](int s, uint32_t ks, int nb) {
+            const uint32_t v_lo = ((smem_base + SM::kV) >> 4) | ((SM::kBlkSub >> 4) << 16);
+            // S = Q K^T: A = Q tile (K-major), B = K block (K-major), 16 features per MMA.
+            auto issue_qk = [&](int s, uint32_t buf, uint32_t ks) {
                 const uint32_t qa = q_lo + s * (SM::kQSlot >> 4);
-                const uint32_t kb = k_lo + ks * (SM::kPairTile >> 4);
-                const uint32_t dst = tmem_base + s * 128;
-                const uint32_t idesc = nb == 2 ? idesc_qk2 : idesc_qk1;
+                const uint32_t kb = k_lo + ks * (SM::kBlkTile >> 4);
+                const uint32_t dst = tmem_base + s * 128 + buf * 64;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk)
                     ptx::umma_ss_lohi(dst, qa + (((kk / 4) * SM::kQSub + (kk % 4) * 32) >> 4), desc_hi,
-                                      kb + (((kk / 4) * SM::kPairSub + (kk % 4) * 32) >> 4), desc_hi, idesc,
+                                      kb + (((kk / 4) * SM::kBlkSub + (kk % 4) * 32) >> 4), desc_hi, idesc_qk,
                                       kk > 0 ? 1u : 0u);
             };
-            // O_s (+)= P_s V: A = P (tensor memory, bf16 pairs in the first 32 nb columns of the
-            // slot's S region), B = V pair tile (MN-major: features contiguous), 16 keys per MMA.
-            auto issue_pv = [&](int s, uint32_t vs, int nb, bool acc) {
-                const uint32_t vb = v_lo + vs * (SM::kPairTile >> 4);
+            // O (+)= P V: A = P (tensor memory: bf16 pairs in the first 32 columns of the S buffer),
+            // B = V block (MN-major: features contiguous), 16 keys per MMA.
+            auto issue_pv = [&](int s, uint32_t buf, uint32_t vs, bool acc) {
+                const uint32_t vb = v_lo + vs * (SM::kBlkTile >> 4);
                 const uint32_t dst = tmem_base + 256 + s * D;
-                const uint32_t pa_ = tmem_base + s * 128;
+                const uint32_t pa_ = tmem_base + s * 128 + buf * 64;
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    if (kk < 4 * nb)
-                        ptx::umma_ts_lohi(dst, pa_ + kk * 8, vb + ((kk * 2048) >> 4), desc_hi, idesc_pv,
-                                          (acc || kk > 0) ? 1u : 0u);
+                for (int kk = 0; kk < kBlk / 16; ++kk)
+                    ptx::umma_ts_lohi(dst, pa_ + kk * 8, vb + ((kk * 2048) >> 4), desc_hi, idesc_pv,
+                                      (acc || kk > 0) ? 1u : 0u);
             };
-            uint32_t pc = 0, ul = 0;
+            uint32_t kc = 0, ul = 0;
             bool ok = true;
             for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
                 const Unit w = decode_unit(a, u);
                 if (w.n <= 0) continue;
-                const int np = (w.n + 1) >> 1;
                 ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 4));
                 if (!ok) break;
-                ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + pc % kKStages), (pc / kKStages) & 1,
-                                                      abort_flag, a.status, 5));
-                if (!ok) break;
-                ptx::tc_fence_after_sync();
-                if (leader) {
-                    const int nb0 = w.n >= 2 ? 2 : 1;
-                    for (int s = 0; s < 2; ++s) {
-                        issue_qk(s, pc % kKStages, nb0);
-                        ptx::umma_commit(bar(BAR_S_FULL + s));
+                // Prologue: S of the first two steps.
+                for (int t0 = 0; t0 < 2 && t0 < w.n && ok; ++t0) {
+                    const uint32_t c0 = kc + t0;
+                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + c0 % kKStages), (c0 / kKStages) & 1,
+                                                          abort_flag, a.status, 5));
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    if (leader) {
+                        for (int s = 0; s < 2; ++s) {
+                            issue_qk(s, c0 & 1, c0 % kKStages);
+                            ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c0 & 1)));
+                        }
+                        ptx::umma_commit(bar(BAR_K_EMPTY + c0 % kKStages));
                     }
-                    ptx::umma_commit(bar(BAR_K_EMPTY + pc % kKStages));
-                    if (np == 1) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                    __syncwarp();
                 }
-                __syncwarp();
-                for (int tp = 0; tp < np && ok; ++tp) {
-                    const uint32_t c = pc + tp;
-                    const int nb = w.n - 2 * tp >= 2 ? 2 : 1;
-                    const int nb1 = w.n - 2 * (tp + 1) >= 2 ? 2 : 1;
+                if (!ok) break;
+                if (w.n <= 2 && leader) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                for (int t = 0; t < w.n && ok; ++t) {
+                    const uint32_t c = kc + t;
                     ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_V_FULL + c % kVStages), (c / kVStages) & 1,
                                                           abort_flag, a.status, 6));
                     if (!ok) break;
+                    if (t + 2 < w.n) {
+                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + (c + 2) % kKStages),
+                                                              ((c + 2) / kKStages) & 1, abort_flag, a.status, 8));
+                        if (!ok) break;
+                    }
                     for (int s = 0; s < 2; ++s) {
                         ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + s), c & 1, abort_flag, a.status, 7));
                         if (!ok) break;
-                        if (tp + 1 < np && s == 0) {
-                            ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + (c + 1) % kKStages),
-                                                                  ((c + 1) / kKStages) & 1, abort_flag, a.status, 8));
-                            if (!ok) break;
-                        }
                         ptx::tc_fence_after_sync();
                         if (leader) {
-                            issue_pv(s, c % kVStages, nb, tp > 0);
-                            if (tp + 1 == np) ptx::umma_commit(bar(BAR_O_DONE + s));
+                            issue_pv(s, c & 1, c % kVStages, t > 0);
+                            ptx::umma_commit(bar(BAR_O_DONE + s));
                             if (s == 1) ptx::umma_commit(bar(BAR_V_EMPTY + c % kVStages));
-                            if (tp + 1 < np) {
-                                // The next S overwrites this slot's S/P columns; MMAs of one
-                                // issuer execute in order, so P has been consumed by then.
-                                issue_qk(s, (c + 1) % kKStages, nb1);
-                                ptx::umma_commit(bar(BAR_S_FULL + s));
+                            if (t + 2 < w.n) {
+                                issue_qk(s, c & 1, (c + 2) % kKStages);
+                                ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c & 1)));
                                 if (s == 1) {
-                                    ptx::umma_commit(bar(BAR_K_EMPTY + (c + 1) % kKStages));
-                                    if (tp + 2 == np) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                                    ptx::umma_commit(bar(BAR_K_EMPTY + (c + 2) % kKStages));
+                                    if (t + 3 == w.n) ptx::umma_commit(bar(BAR_Q_EMPTY));
                                 }
                             }
                         }
                         __syncwarp();
                     }
                 }
-                pc += np;
+                kc += w.n;
                 ++ul;
             }
         }
@@ -320,10 +306,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const int quad = warp & 3;              // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;       // tile row = TMEM lane
         const int qrow = row & 63;              // token inside the query block
-        const uint32_t t_s = tmem_base + ((uint32_t)(quad * 32) << 16) + s * 128;
+        const uint32_t t_s0 = tmem_base + ((uint32_t)(quad * 32) << 16) + s * 128;
         const uint32_t t_o = tmem_base + ((uint32_t)(quad * 32) << 16) + 256 + s * D;
         const float sl2 = a.scale_log2;
-        uint32_t pc = 0, ul = 0;
+        const uint64_t sl2_2 = ptx::pack_f32x2(sl2, sl2);
+        uint32_t kc = 0;
         bool ok = true;
         for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
             const Unit w = decode_unit(a, u);
@@ -331,104 +318,117 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const int head = w.hk * a.G + head_local;
             const int64_t tok = (int64_t)w.i * kBlk + qrow;
             const bool valid = head_local < a.G && tok < a.N;
-            const int np = (w.n + 1) >> 1;
             // Algorithm 1's causal term acts inside the diagonal pair (col == row) only; rows end
             // with that block.
             const bool last_is_diag = w.n > 0 && __ldg(a.col_idx + w.rs + w.n - 1) == w.i;
             float m = -INFINITY, l = 0.f;
-            for (int tp = 0; tp < np; ++tp, ++pc) {
-                const int nb = w.n - 2 * tp >= 2 ? 2 : 1;
-                ok = wait_bar(bar(BAR_S_FULL + s), pc & 1, abort_flag, a.status, 9);
+            for (int t = 0; t < w.n; ++t, ++kc) {
+                const uint32_t t_s = t_s0 + (kc & 1) * 64;
+                ok = wait_bar(bar(BAR_S_FULL + 2 * s + (kc & 1)), (kc >> 1) & 1, abort_flag, a.status, 9);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                // One online-softmax step per 64-key half.  The exponentials are taken against the
-                // reference maximum m carried from earlier steps (lazy rescaling: m moves only when
-                // the row maximum exceeds it by more than the threshold, so exp2(s - m) stays below
-                // 2^threshold and O / l at the end is exact whatever reference was used).  The rare
-                // half whose maximum does move is recomputed from the logits still in registers.
-                for (int h = 0; h < nb; ++h) {
-                    uint32_t sr[64];
-                    ptx::tmem_ld32(t_s + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
-                    ptx::tmem_ld32(t_s + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
-                    ptx::tmem_wait_ld();
-                    if (last_is_diag && 2 * tp + h == w.n - 1) {
+                uint32_t sr[64];
+                ptx::tmem_ld32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+                ptx::tmem_ld32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+                ptx::tmem_wait_ld();
+                if (last_is_diag && t == w.n - 1) {
 #pragma unroll
-                        for (int c = 0; c < 64; ++c)
-                            if (c > qrow) sr[c] = 0xff800000u;  // -inf
+                    for (int c = 0; c < 64; ++c)
+                        if (c > qrow) sr[c] = 0xff800000u;  // -inf
+                }
+                // Fast path: p = exp2(s * scale - m) against the reference maximum m carried from
+                // earlier steps (lazy rescaling: m moves only when the row maximum exceeds it by
+                // more than the threshold, so p stays below 2^threshold and O / l at the end is
+                // exact whatever reference was used).  Two-wide fp32 arithmetic; the row maximum
+                // is watched on the rounded bf16 values (p > 2^threshold <=> s - m > threshold;
+                // an overflow shows up as inf).
+                const uint64_t negm_2 = ptx::pack_f32x2(-m, -m);
+                uint64_t sum2[2] = {0ull, 0ull};
+                uint32_t pmax2[2] = {0u, 0u};
+                uint32_t pk[32];
+#pragma unroll
+                for (int c = 0; c < 64; c += 4) {
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const uint64_t y2 = ptx::fma_f32x2(
+                            ptx::pack_f32x2(__uint_as_float(sr[c + 2 * e]), __uint_as_float(sr[c + 2 * e + 1])), sl2_2,
+                            negm_2);
+                        float y0, y1;
+                        ptx::unpack_f32x2(y2, y0, y1);
+                        const float p0 = ptx::ex2(y0), p1 = ptx::ex2(y1);
+                        sum2[e] = ptx::add_f32x2(sum2[e], ptx::pack_f32x2(p0, p1));
+                        const uint32_t q = ptx::cvt_bf16x2(p0, p1);
+                        pk[(c >> 1) + e] = q;
+                        pmax2[e] = ptx::max_bf16x2(pmax2[e], q);
                     }
+                }
+                float sum;
+                {
+                    float s0, s1, s2, s3;
+                    ptx::unpack_f32x2(sum2[0], s0, s1);
+                    ptx::unpack_f32x2(sum2[1], s2, s3);
+                    sum = (s0 + s1) + (s2 + s3);
+                }
+                const uint32_t pm = ptx::max_bf16x2(pmax2[0], pmax2[1]);
+                const float pmaxf = fmaxf(__uint_as_float(pm << 16), __uint_as_float(pm & 0xffff0000u));
+                // !(x <= limit) also catches inf and NaN.
+                const bool suspect = t == 0 || !(pmaxf <= 256.0f);
+                if (__any_sync(0xffffffffu, suspect)) {
+                    // Rare path: exact row maximum, new reference for the rows that need it, what
+                    // was accumulated so far brought to the new reference, P recomputed from the
+                    // logits still in registers.
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                    for (int c = 0; c < 64; c += 4) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) mx4[e] = fmaxf(mx4[e], __uint_as_float(sr[c + e]));
+                    }
+                    const float mx2 = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
+                    const bool grow = t == 0 || mx2 > m + kRescaleThreshold;
+                    const float m_new = grow ? mx2 : m;
+                    const float alpha = grow ? ptx::ex2(m - m_new) : 1.0f;  // 0 on the first step
+                    l *= alpha;
+                    m = m_new;
+                    if (t > 0) {
+                        // O may be rescaled only once the previous step's P V has completed.
+                        ok = wait_bar(bar(BAR_O_DONE + s), (kc - 1) & 1, abort_flag, a.status, 11);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                        ptx::tc_fence_after_sync();
+#pragma unroll 1
+                        for (int ch = 0; ch < D / 32; ++ch) {
+                            uint32_t orr[32];
+                            ptx::tmem_ld32(t_o + ch * 32, orr);
+                            ptx::tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                            ptx::tmem_st32(t_o + ch * 32, orr);
+                        }
+                    }
                     float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-                    uint32_t pk[32];
-                    const float neg_m = -m;
 #pragma unroll
                     for (int c = 0; c < 64; c += 4) {
                         float pv[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const float x = __uint_as_float(sr[c + e]);
-                            mx4[e] = fmaxf(mx4[e], x);
-                            pv[e] = ptx::ex2(fmaf(x, sl2, neg_m));
+                            pv[e] = ptx::ex2(fmaf(__uint_as_float(sr[c + e]), sl2, -m));
                             sum4[e] += pv[e];
                         }
-                        const __nv_bfloat162 h01 = __floats2bfloat162_rn(pv[0], pv[1]);
-                        const __nv_bfloat162 h23 = __floats2bfloat162_rn(pv[2], pv[3]);
-                        pk[c >> 1] = *reinterpret_cast<const uint32_t *>(&h01);
-                        pk[(c >> 1) + 1] = *reinterpret_cast<const uint32_t *>(&h23);
+                        pk[c >> 1] = ptx::cvt_bf16x2(pv[0], pv[1]);
+                        pk[(c >> 1) + 1] = ptx::cvt_bf16x2(pv[2], pv[3]);
                     }
-                    const float mx2 = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
-                    const bool first = tp == 0 && h == 0;
-                    const bool grow = first || mx2 > m + kRescaleThreshold;
-                    if (__any_sync(0xffffffffu, grow)) {
-                        const float m_new = grow ? mx2 : m;
-                        const float alpha = grow ? ptx::ex2(m - m_new) : 1.0f;  // 0 on the first half
-                        l *= alpha;
-                        m = m_new;
-                        if (tp > 0) {
-                            // O_s is quiescent: the S just waited for was issued after the previous P V.
-#pragma unroll 1
-                            for (int ch = 0; ch < D / 32; ++ch) {
-                                uint32_t orr[32];
-                                ptx::tmem_ld32(t_o + ch * 32, orr);
-                                ptx::tmem_wait_ld();
-#pragma unroll
-                                for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-                                ptx::tmem_st32(t_o + ch * 32, orr);
-                            }
-                        }
-                        if (h == 1) {
-                            // The first half's P of this step is already stored: bring it to the new reference.
-                            uint32_t pr[32];
-                            ptx::tmem_ld32(t_s, pr);
-                            ptx::tmem_wait_ld();
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) {
-                                const float lo = __uint_as_float(pr[c] << 16) * alpha;
-                                const float hi = __uint_as_float(pr[c] & 0xffff0000u) * alpha;
-                                const __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
-                                pr[c] = *reinterpret_cast<const uint32_t *>(&h2);
-                            }
-                            ptx::tmem_st32(t_s, pr);
-                        }
-                        sum4[0] = sum4[1] = sum4[2] = sum4[3] = 0.f;
-#pragma unroll
-                        for (int c = 0; c < 64; c += 4) {
-                            float pv[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                pv[e] = ptx::ex2(fmaf(__uint_as_float(sr[c + e]), sl2, -m));
-                                sum4[e] += pv[e];
-                            }
-                            const __nv_bfloat162 h01 = __floats2bfloat162_rn(pv[0], pv[1]);
-                            const __nv_bfloat162 h23 = __floats2bfloat162_rn(pv[2], pv[3]);
-                            pk[c >> 1] = *reinterpret_cast<const uint32_t *>(&h01);
-                            pk[(c >> 1) + 1] = *reinterpret_cast<const uint32_t *>(&h23);
-                        }
-                    }
-                    l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-                    // P (bf16 pairs) goes to the first columns of the S region: half h -> [32 h, 32 h + 32).
-                    // Half 0 overwrites logits that were just read; half 1's logits sit at [64, 128).
-                    ptx::tmem_st32(t_s + h * 32, pk);
+                    sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                }
+                l += sum;
+                // P (bf16 pairs) overlays the first 32 columns of the S buffer just read.
+                ptx::tmem_st32(t_s, pk);
+                if (kc > 0) {
+                    // Observe every phase of the P V completion barrier (the previous step's P V
+                    // has normally finished long ago), so that its parity stays unambiguous.
+                    ok = wait_bar(bar(BAR_O_DONE + s), (kc - 1) & 1, abort_flag, a.status, 12);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
@@ -447,10 +447,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 continue;
             }
             // Epilogue: O / l and LSE = ln sum exp(s) = (m + log2 l) ln 2.
-            ok = wait_bar(bar(BAR_O_DONE + s), ul & 1, abort_flag, a.status, 10);
+            ok = wait_bar(bar(BAR_O_DONE + s), (kc - 1) & 1, abort_flag, a.status, 10);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            ++ul;
             ptx::tc_fence_after_sync();
             const float inv = 1.0f / l;
             const int64_t obase = w.b * a.o_sb + tok * a.o_ss + (int64_t)head * a.o_sh;
@@ -469,16 +468,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     } else {
                         uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(a.o) + obase + ch * 32);
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t h[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const __nv_bfloat162 h2 = __floats2bfloat162_rn(
-                                    __uint_as_float(orr[8 * c + 2 * e]) * inv, __uint_as_float(orr[8 * c + 2 * e + 1]) * inv);
-                                h[e] = *reinterpret_cast<const uint32_t *>(&h2);
-                            }
-                            dst[c] = make_uint4(h[0], h[1], h[2], h[3]);
-                        }
+                        for (int c = 0; c < 4; ++c)
+                            dst[c] = make_uint4(
+                                ptx::cvt_bf16x2(__uint_as_float(orr[8 * c]) * inv, __uint_as_float(orr[8 * c + 1]) * inv),
+                                ptx::cvt_bf16x2(__uint_as_float(orr[8 * c + 2]) * inv, __uint_as_float(orr[8 * c + 3]) * inv),
+                                ptx::cvt_bf16x2(__uint_as_float(orr[8 * c + 4]) * inv, __uint_as_float(orr[8 * c + 5]) * inv),
+                                ptx::cvt_bf16x2(__uint_as_float(orr[8 * c + 6]) * inv, __uint_as_float(orr[8 * c + 7]) * inv));
                     }
                 }
             }
