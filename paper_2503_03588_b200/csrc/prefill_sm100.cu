@@ -63,22 +63,25 @@ enum : uint32_t {
     BAR_Q_FULL = 0, BAR_Q_EMPTY = 1, BAR_K_FULL = 2, BAR_K_EMPTY = BAR_K_FULL + kKStages,
     BAR_V_FULL = BAR_K_EMPTY + kKStages, BAR_V_EMPTY = BAR_V_FULL + kVStages,
     BAR_S_FULL = BAR_V_EMPTY + kVStages,  // [slot][buffer]
-    BAR_P_FULL = BAR_S_FULL + 4, BAR_O_DONE = BAR_P_FULL + 2, BAR_COUNT = BAR_O_DONE + 2
+    BAR_P_FULL = BAR_S_FULL + 4,
+    BAR_O_DONE = BAR_P_FULL + 2,  // [slot][step parity]: P V of that step has completed
+    BAR_COUNT = BAR_O_DONE + 4
 };
 
 struct Unit {
     int32_t b, hk, i, sub, rs, n;
 };
 
-__device__ __forceinline__ Unit decode_unit(const PrefillArgs &a, int64_t u)
+// Unit index -> coordinates (the unit count fits in 30 bits; checked on the host).
+__device__ __forceinline__ Unit decode_unit(const PrefillArgs &a, uint32_t u)
 {
     Unit r;
-    r.sub = (int32_t)(u % a.nsub);
-    u /= a.nsub;
-    r.hk = (int32_t)(u % a.Hkv);
-    u /= a.Hkv;
-    r.i = a.nqb - 1 - (int32_t)(u % a.nqb);  // long rows first
-    r.b = (int32_t)(u / a.nqb);
+    r.sub = (int32_t)(u % (uint32_t)a.nsub);
+    u /= (uint32_t)a.nsub;
+    r.hk = (int32_t)(u % (uint32_t)a.Hkv);
+    u /= (uint32_t)a.Hkv;
+    r.i = a.nqb - 1 - (int32_t)(u % (uint32_t)a.nqb);  // long rows first
+    r.b = (int32_t)(u / (uint32_t)a.nqb);
     r.rs = __ldg(a.row_ptr + r.i);
     r.n = __ldg(a.row_ptr + r.i + 1) - r.rs;
     return r;
@@ -133,10 +136,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::mbar_init(bar(BAR_V_FULL + s), 1);
             ptx::mbar_init(bar(BAR_V_EMPTY + s), 1);
         }
-        for (int s = 0; s < 4; ++s) ptx::mbar_init(bar(BAR_S_FULL + s), 1);
+        for (int s = 0; s < 4; ++s) {
+            ptx::mbar_init(bar(BAR_S_FULL + s), 1);
+            ptx::mbar_init(bar(BAR_O_DONE + s), 1);
+        }
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(bar(BAR_P_FULL + s), 128);
-            ptx::mbar_init(bar(BAR_O_DONE + s), 1);
         }
         *abort_flag = 0;
         ptx::fence_barrier_init();
@@ -160,7 +165,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::prefetch_tensormap(&tmV);
             uint32_t kc = 0, ul = 0;  // key blocks and units issued so far by this CTA
             bool ok = true;
-            for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
+            for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
                 const Unit w = decode_unit(a, u);
                 if (w.n <= 0) continue;
                 if (ul > 0) ok = wait_bar(bar(BAR_Q_EMPTY), (ul - 1) & 1, abort_flag, a.status, 1);
@@ -241,7 +246,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             };
             uint32_t kc = 0, ul = 0;
             bool ok = true;
-            for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
+            for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
                 const Unit w = decode_unit(a, u);
                 if (w.n <= 0) continue;
                 ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 4));
@@ -280,7 +285,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         ptx::tc_fence_after_sync();
                         if (leader) {
                             issue_pv(s, c & 1, c % kVStages, t > 0);
-                            ptx::umma_commit(bar(BAR_O_DONE + s));
+                            ptx::umma_commit(bar(BAR_O_DONE + 2 * s + (c & 1)));
                             if (s == 1) ptx::umma_commit(bar(BAR_V_EMPTY + c % kVStages));
                             if (t + 2 < w.n) {
                                 issue_qk(s, c & 1, (c + 2) % kKStages);
@@ -312,15 +317,27 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const uint64_t sl2_2 = ptx::pack_f32x2(sl2, sl2);
         uint32_t kc = 0;
         bool ok = true;
-        for (int64_t u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
-            const Unit w = decode_unit(a, u);
+        Unit w_next = {};
+        int32_t lastcol_next = -1;
+        if (blockIdx.x < (uint32_t)a.n_units) {
+            w_next = decode_unit(a, blockIdx.x);
+            if (w_next.n > 0) lastcol_next = __ldg(a.col_idx + w_next.rs + w_next.n - 1);
+        }
+        for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
+            const Unit w = w_next;
+            const int32_t lastcol = lastcol_next;
+            if (u + gridDim.x < (uint32_t)a.n_units) {
+                // Metadata of the next unit: loaded now, used one unit later.
+                w_next = decode_unit(a, u + gridDim.x);
+                lastcol_next = w_next.n > 0 ? __ldg(a.col_idx + w_next.rs + w_next.n - 1) : -1;
+            }
             const int head_local = w.sub * 4 + 2 * s + (row >> 6);
             const int head = w.hk * a.G + head_local;
             const int64_t tok = (int64_t)w.i * kBlk + qrow;
             const bool valid = head_local < a.G && tok < a.N;
             // Algorithm 1's causal term acts inside the diagonal pair (col == row) only; rows end
             // with that block.
-            const bool last_is_diag = w.n > 0 && __ldg(a.col_idx + w.rs + w.n - 1) == w.i;
+            const bool last_is_diag = w.n > 0 && lastcol == w.i;
             float m = -INFINITY, l = 0.f;
             for (int t = 0; t < w.n; ++t, ++kc) {
                 const uint32_t t_s = t_s0 + (kc & 1) * 64;
@@ -391,8 +408,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     l *= alpha;
                     m = m_new;
                     if (t > 0) {
-                        // O may be rescaled only once the previous step's P V has completed.
-                        ok = wait_bar(bar(BAR_O_DONE + s), (kc - 1) & 1, abort_flag, a.status, 11);
+                        // O may be rescaled only once the previous step's P V has completed.  (The
+                        // completion barriers alternate by step parity; the S waited for above was issued
+                        // after the P V of step kc - 2, so a barrier is never more than one phase behind.)
+                        ok = wait_bar(bar(BAR_O_DONE + 2 * s + ((kc - 1) & 1)), ((kc - 1) >> 1) & 1, abort_flag, a.status, 11);
                         ok = __all_sync(0xffffffffu, ok);
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
@@ -423,13 +442,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 l += sum;
                 // P (bf16 pairs) overlays the first 32 columns of the S buffer just read.
                 ptx::tmem_st32(t_s, pk);
-                if (kc > 0) {
-                    // Observe every phase of the P V completion barrier (the previous step's P V
-                    // has normally finished long ago), so that its parity stays unambiguous.
-                    ok = wait_bar(bar(BAR_O_DONE + s), (kc - 1) & 1, abort_flag, a.status, 12);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(bar(BAR_P_FULL + s));
@@ -447,7 +459,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 continue;
             }
             // Epilogue: O / l and LSE = ln sum exp(s) = (m + log2 l) ln 2.
-            ok = wait_bar(bar(BAR_O_DONE + s), (kc - 1) & 1, abort_flag, a.status, 10);
+            ok = wait_bar(bar(BAR_O_DONE + 2 * s + ((kc - 1) & 1)), ((kc - 1) >> 1) & 1, abort_flag, a.status, 10);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             ptx::tc_fence_after_sync();
@@ -615,6 +627,7 @@ extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const
     a.G = p->n_q_heads / p->n_kv_heads;
     a.nsub = (a.G + 3) / 4;
     a.n_units = (int64_t)p->batch * nqb * a.Hkv * a.nsub;
+    if (a.n_units > (int64_t)0x3fffffff) return fail(PA_ERR_SHAPE, "too many work units (%lld)", (long long)a.n_units);
     a.o_is_f32 = p->o_dtype == PA_F32;
     const float scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.0f / sqrtf((float)D);
     a.scale_log2 = scale * 1.4426950408889634f;
