@@ -54,7 +54,7 @@ struct SmemMap {
     static constexpr uint32_t kK = kQ + 2 * kQSlot;
     static constexpr uint32_t kV = kK + kKStages * kBlkTile;
     static constexpr uint32_t kBars = kV + kVStages * kBlkTile;
-    static constexpr uint32_t kTotal = kBars + 256;
+    static constexpr uint32_t kTotal = kBars + 512;
     static constexpr uint32_t kAlloc = kTotal + 1024;         // slack for 1024-byte alignment
 };
 
@@ -442,6 +442,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 l += sum;
                 // P (bf16 pairs) overlays the first 32 columns of the S buffer just read.
                 ptx::tmem_st32(t_s, pk);
+                if (kc > 0) {
+                    // Do not run two P hand-overs ahead of the issuer: its parity wait on this slot's
+                    // P barrier can tell only one completed phase from none.  Once the previous
+                    // step's P V has completed (normally long ago) the issuer has consumed that phase.
+                    ok = wait_bar(bar(BAR_O_DONE + 2 * s + ((kc - 1) & 1)), ((kc - 1) >> 1) & 1, abort_flag, a.status, 12);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(bar(BAR_P_FULL + s));
