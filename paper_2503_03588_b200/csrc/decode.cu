@@ -2,10 +2,10 @@
 // its position (Section 4.1: same pattern in prefilling and decoding; Eq. (1) for the row).
 //
 // Split-K: one CTA per (sequence, KV head, chunk) where a chunk is one 64-key block of the
-// row's block list.  Each CTA stages its K and V block in shared memory with coalesced 16-byte
-// asynchronous copies, computes the logits of all query heads of the group, a chunk-local
-// softmax (warp-shuffle reductions) and the unnormalised partial output, and writes
-// (o[D], m, l) per head to the workspace.  A second kernel merges the chunks with the
+// row's block list.  Each CTA reads its K and V block with coalesced 16-byte loads, computes the
+// logits of all query heads of the group and the unnormalised partial output on the warp-level
+// tensor-core MMA, a chunk-local softmax (warp-shuffle reductions), and writes (o[D], m, l)
+// per head to the workspace.  A second kernel merges the chunks with the
 // log-sum-exp rule.  The second launch overlaps the first one's tail through programmatic
 // dependent launch; it waits for the partials with griddepcontrol.wait.
 #include <cuda_bf16.h>
@@ -32,42 +32,51 @@ struct DecodeArgs {
     float scale_log2;  // softmax_scale * log2(e)
 };
 
-__device__ __forceinline__ void cp_async16(void *smem, const void *gmem)
+// 16-byte read-only global load.
+__device__ __forceinline__ uint4 ldg16(const void *p)
 {
-    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem));
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait()
-{
-    asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+    uint4 r;
+    asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];\n"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
 }
 
-// Physical 16-byte chunk of logical chunk c in row r: XOR with the row keeps the eight rows a
-// quarter-warp reads at one logical column in different banks.
-template <int D>
-__device__ __forceinline__ int swz(int r, int c)
+// D(16x8, fp32) += A(16x16, bf16, row-major) * B(16x8, bf16, column-major), one warp.
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1)
 {
-    return r * (D / 8) + (c ^ (r & 7));
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};\n"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// Partial attention of one 64-key block for all query heads of a KV group.
+//
+// Each of the four warps takes 16 keys and runs the two small contractions on the warp-level
+// tensor-core MMA (16 x 8 x 16): the query heads of the group are the M rows (rows beyond the
+// group are zero), so one pass over K and V serves every head.  K, V and Q are read straight
+// from global memory with 16-byte loads, all issued before the first use.  A thread's 16-byte
+// piece holds eight consecutive features of one row; the dot product does not care in which
+// order features are paired, so the pieces are fed to the MMA fragments as they come (Q and K
+// use the same pairing), and for P V two rows are interleaved with byte permutes.  The four
+// warps' (o, m, l) are merged in shared memory and one partial per head goes to the workspace.
 template <int D>
 __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const DecodeArgs a)
 {
     // Let the combine kernel's CTAs be scheduled as soon as SM resources free up.
     asm volatile("griddepcontrol.launch_dependents;\n" ::);
 
-    constexpr int CPR = D / 8;  // 16-byte chunks per row
-    __shared__ __align__(16) uint4 sK[kDecBlock * CPR];
-    __shared__ __align__(16) uint4 sV[kDecBlock * CPR];
-    __shared__ __align__(16) float sQ[kMaxGroup * D];
-    __shared__ __align__(16) float sP[kMaxGroup * kDecBlock];
-    __shared__ float sRed[kMaxGroup * 4];
-    __shared__ float sM[kMaxGroup], sL[kMaxGroup];
+    constexpr int NJ = D / 32;  // 16-byte pieces per thread and row for Q and K
+    constexpr int NV = D / 64;  // 16-byte pieces per thread and row for V
+    __shared__ float sO[4][kMaxGroup][D];
+    __shared__ float sM[4][kMaxGroup], sL[4][kMaxGroup];
 
     const int chunk = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
     const int G = a.G;
 
     const int64_t len = a.lens[b];
@@ -80,108 +89,110 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const Decod
     });
     if (chunk >= n) return;
     const int n_keys = jblk == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
+    const int base = wid * 16;  // first key of this warp inside the block
 
-    // Stage K and V (rows beyond n_keys are not read from memory and are zero-filled).
+    // ---- loads (keys at or beyond n_keys do not exist: zeros instead of a read)
     const __nv_bfloat16 *kb = a.k + b * a.k_sb + (jblk * kDecBlock) * a.k_ss + hk * a.k_sh;
     const __nv_bfloat16 *vb = a.v + b * a.v_sb + (jblk * kDecBlock) * a.v_ss + hk * a.v_sh;
-    for (int idx = tid; idx < kDecBlock * CPR; idx += kDecThreads) {
-        const int r = idx / CPR, c = idx % CPR;
-        if (r < n_keys)
-            cp_async16(&sK[swz<D>(r, c)], kb + r * a.k_ss + c * 8);
-        else
-            sK[swz<D>(r, c)] = make_uint4(0, 0, 0, 0);
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    uint4 kr[2][NJ], vr[4][NV], qr[NJ];
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+        const int key = base + nt * 8 + g;
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) kr[nt][j] = key < n_keys ? ldg16(kb + key * a.k_ss + 8 * (4 * j + t)) : zero4;
     }
-    cp_async_commit();
-    for (int idx = tid; idx < kDecBlock * CPR; idx += kDecThreads) {
-        const int r = idx / CPR, c = idx % CPR;
-        if (r < n_keys)
-            cp_async16(&sV[r * CPR + c], vb + r * a.v_ss + c * 8);
-        else
-            sV[r * CPR + c] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int kx = 0; kx < 4; ++kx) {
+        const int key = base + 2 * t + (kx & 1) + (kx >> 1) * 8;
+#pragma unroll
+        for (int jj = 0; jj < NV; ++jj) vr[kx][jj] = key < n_keys ? ldg16(vb + key * a.v_ss + 8 * (g + 8 * jj)) : zero4;
     }
-    cp_async_commit();
-    // Query rows of the group, widened to fp32.
-    const __nv_bfloat16 *qb = a.q + ((int64_t)b * a.Hq + (int64_t)hk * G) * D;
-    for (int idx = tid; idx < G * D; idx += kDecThreads) sQ[idx] = __bfloat162float(qb[idx]);
-    cp_async_wait<1>();
-    __syncthreads();
+    const __nv_bfloat16 *qb = a.q + ((int64_t)b * a.Hq + (int64_t)hk * G + g) * D;
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) qr[j] = g < G ? ldg16(qb + 8 * (4 * j + t)) : zero4;
 
-    // Logits: thread -> (key = tid % 64, half = tid / 64); half 0 takes heads [0, 4), half 1 [4, 8).
+    // ---- S = Q K^T: rows = heads, columns = the warp's 16 keys (two 8-key tiles)
+    float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) {
+            mma_bf16(sc[nt], qr[j].x, 0u, qr[j].y, 0u, kr[nt][j].x, kr[nt][j].y);
+            mma_bf16(sc[nt], qr[j].z, 0u, qr[j].w, 0u, kr[nt][j].z, kr[nt][j].w);
+        }
+    }
+    // This thread holds head g, keys base + 8 nt + 2 t + {0, 1}.  Softmax over the warp's keys in
+    // the base-2 domain: s2 = s * scale * log2(e).
+    float s2[2][2];
+    float mw = -INFINITY;
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            const int key = base + nt * 8 + 2 * t + x;
+            s2[nt][x] = key < n_keys ? sc[nt][x] * a.scale_log2 : -INFINITY;
+            mw = fmaxf(mw, s2[nt][x]);
+        }
+    mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, 1));
+    mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, 2));
+    float pe[2][2], lw = 0.f;
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            pe[nt][x] = mw == -INFINITY ? 0.f : exp2f(s2[nt][x] - mw);
+            lw += pe[nt][x];
+        }
+    lw += __shfl_xor_sync(0xffffffffu, lw, 1);
+    lw += __shfl_xor_sync(0xffffffffu, lw, 2);
+    // P as the A operand of P V: columns 2t, 2t+1 (first key tile) and 2t+8, 2t+9 (second).
+    const __nv_bfloat162 p01 = __floats2bfloat162_rn(pe[0][0], pe[0][1]);
+    const __nv_bfloat162 p23 = __floats2bfloat162_rn(pe[1][0], pe[1][1]);
+    const uint32_t pa0 = *reinterpret_cast<const uint32_t *>(&p01), pa2 = *reinterpret_cast<const uint32_t *>(&p23);
+
+    // ---- O = P V: the B operand pairs two keys per register; feature tile (jj, e) of this
+    // thread's quad covers features 8 (n + 8 jj) + e, n = 0..7.
     {
-        const int key = tid & 63, h0 = (tid >> 6) * 4;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 4
-        for (int c = 0; c < CPR; ++c) {
-            const uint4 kk = sK[swz<D>(key, c)];
-            const uint32_t w[4] = {kk.x, kk.y, kk.z, kk.w};
-            float kf[8];
 #pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                kf[2 * t] = __uint_as_float(w[t] << 16);
-                kf[2 * t + 1] = __uint_as_float(w[t] & 0xffff0000u);
-            }
+        for (int jj = 0; jj < NV; ++jj) {
+            const uint32_t v0[4] = {vr[0][jj].x, vr[0][jj].y, vr[0][jj].z, vr[0][jj].w};
+            const uint32_t v1[4] = {vr[1][jj].x, vr[1][jj].y, vr[1][jj].z, vr[1][jj].w};
+            const uint32_t v2[4] = {vr[2][jj].x, vr[2][jj].y, vr[2][jj].z, vr[2][jj].w};
+            const uint32_t v3[4] = {vr[3][jj].x, vr[3][jj].y, vr[3][jj].z, vr[3][jj].w};
 #pragma unroll
-            for (int hh = 0; hh < 4; ++hh) {
-                if (h0 + hh < G) {
-                    const float4 q0 = *reinterpret_cast<const float4 *>(&sQ[(h0 + hh) * D + c * 8]);
-                    const float4 q1 = *reinterpret_cast<const float4 *>(&sQ[(h0 + hh) * D + c * 8 + 4]);
-                    acc[hh] += kf[0] * q0.x + kf[1] * q0.y + kf[2] * q0.z + kf[3] * q0.w +
-                               kf[4] * q1.x + kf[5] * q1.y + kf[6] * q1.z + kf[7] * q1.w;
+            for (int e = 0; e < 8; ++e) {
+                const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
+                const uint32_t b0 = __byte_perm(v0[e >> 1], v1[e >> 1], sel);
+                const uint32_t b1 = __byte_perm(v2[e >> 1], v3[e >> 1], sel);
+                float oc[4] = {0.f, 0.f, 0.f, 0.f};
+                mma_bf16(oc, pa0, 0u, pa2, 0u, b0, b1);
+                // oc[0], oc[1]: head g, features 8 (2t + x + 8 jj) + e
+                if (g < G) {
+                    sO[wid][g][8 * (2 * t + 8 * jj) + e] = oc[0];
+                    sO[wid][g][8 * (2 * t + 1 + 8 * jj) + e] = oc[1];
                 }
             }
         }
-        // Chunk-local softmax per head in the base-2 domain: s2 = s * scale * log2(e).
-#pragma unroll
-        for (int hh = 0; hh < 4; ++hh) {
-            const int h = h0 + hh;
-            const float s2 = key < n_keys ? acc[hh] * a.scale_log2 : -INFINITY;
-            float mx = s2;
-            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            if (lane == 0) sRed[h * 4 + (warp & 1)] = mx;
-            acc[hh] = s2;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int hh = 0; hh < 4; ++hh) {
-            const int h = h0 + hh;
-            const float m = fmaxf(sRed[h * 4 + 0], sRed[h * 4 + 1]);  // finite: key 0 is valid
-            const float pexp = exp2f(acc[hh] - m);                     // 0 for masked keys
-            sP[h * kDecBlock + key] = pexp;
-            float sum = pexp;
-            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            if (lane == 0) sRed[h * 4 + 2 + (warp & 1)] = sum;
-            if (key == 0) sM[h] = m;
-        }
     }
-    cp_async_wait<0>();
+    if (t == 0 && g < G) {
+        sM[wid][g] = mw;
+        sL[wid][g] = lw;
+    }
     __syncthreads();
-    if (tid < kMaxGroup) sL[tid] = sRed[tid * 4 + 2] + sRed[tid * 4 + 3];
 
-    // Partial output: thread -> feature d (D <= 128 threads), all heads of the group.
-    if (tid < D) {
-        float o[kMaxGroup];
-#pragma unroll
-        for (int h = 0; h < kMaxGroup; ++h) o[h] = 0.f;
-        const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(sV);
-#pragma unroll 4
-        for (int key = 0; key < kDecBlock; ++key) {
-            const float vv = __bfloat162float(vs[key * D + tid]);
-#pragma unroll
-            for (int h = 0; h < kMaxGroup; ++h)
-                if (h < G) o[h] += sP[h * kDecBlock + key] * vv;
+    // ---- merge the four warps and write one partial (o[D], m, l) per head
+    for (int idx = tid; idx < G * D; idx += kDecThreads) {
+        const int h = idx / D, d = idx % D;
+        const float m0 = sM[0][h], m1 = sM[1][h], m2 = sM[2][h], m3 = sM[3][h];
+        const float m = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));  // finite: key 0 of the block exists
+        const float w0 = exp2f(m0 - m), w1 = exp2f(m1 - m), w2 = exp2f(m2 - m), w3 = exp2f(m3 - m);
+        float *dst = a.partial + (((int64_t)b * a.Hq + hk * G + h) * a.chunks + chunk) * (D + 2);
+        dst[d] = sO[0][h][d] * w0 + sO[1][h][d] * w1 + sO[2][h][d] * w2 + sO[3][h][d] * w3;
+        if (d == 0) {
+            dst[D] = m;
+            dst[D + 1] = sL[0][h] * w0 + sL[1][h] * w1 + sL[2][h] * w2 + sL[3][h] * w3;
         }
-#pragma unroll
-        for (int h = 0; h < kMaxGroup; ++h)
-            if (h < G) {
-                float *dst = a.partial + (((int64_t)b * a.Hq + hk * G + h) * a.chunks + chunk) * (D + 2);
-                dst[tid] = o[h];
-            }
-    }
-    __syncthreads();
-    if (tid < G) {
-        float *dst = a.partial + (((int64_t)b * a.Hq + hk * G + tid) * a.chunks + chunk) * (D + 2);
-        dst[D] = sM[tid];      // base-2 running max of the chunk
-        dst[D + 1] = sL[tid];  // sum of 2^(s2 - m)
     }
 }
 
