@@ -201,6 +201,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const Decod
 template <int D>
 __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeArgs a)
 {
+    __shared__ float s_red[D / 32];
     const int h = blockIdx.x, b = blockIdx.y, d = threadIdx.x;
     const int64_t len = a.lens[b];
     const bool valid = len >= 1 && len <= a.max_len;
@@ -209,9 +210,18 @@ __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeArgs a)
     // The partial kernel's writes are visible only after this wait.
     asm volatile("griddepcontrol.wait;\n" ::: "memory");
     const float *src = a.partial + (((int64_t)b * a.Hq + h) * a.chunks) * (D + 2);
+    // Global maximum: the chunks are spread over the threads (independent loads), then reduced.
     float m = -INFINITY;
-    for (int c = 0; c < n; ++c) m = fmaxf(m, src[c * (D + 2) + D]);
+    for (int c = d; c < n; c += D) m = fmaxf(m, src[c * (D + 2) + D]);
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((d & 31) == 0) s_red[d >> 5] = m;
+    __syncthreads();
+    m = s_red[0];
+#pragma unroll
+    for (int w = 1; w < D / 32; ++w) m = fmaxf(m, s_red[w]);
+    // Weighted sums; the loop is unrolled so that the loads of several chunks are in flight.
     float l = 0.f, acc = 0.f;
+#pragma unroll 8
     for (int c = 0; c < n; ++c) {
         const float w = exp2f(src[c * (D + 2) + D] - m);
         l += src[c * (D + 2) + D + 1] * w;
