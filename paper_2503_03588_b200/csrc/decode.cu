@@ -2,12 +2,13 @@
 // its position (Section 4.1: same pattern in prefilling and decoding; Eq. (1) for the row).
 //
 // Split-K: one CTA per (sequence, KV head, chunk) where a chunk is one 64-key block of the
-// row's block list.  Each CTA reads its K and V block with coalesced 16-byte loads, computes the
-// logits of all query heads of the group and the unnormalised partial output on the warp-level
-// tensor-core MMA, a chunk-local softmax (warp-shuffle reductions), and writes (o[D], m, l)
-// per head to the workspace.  A second kernel merges the chunks with the
-// log-sum-exp rule.  The second launch overlaps the first one's tail through programmatic
-// dependent launch; it waits for the partials with griddepcontrol.wait.
+// row's block list.  Each CTA reads its K and V block with coalesced 16-byte loads and computes
+// the logits of all query heads of the group, a chunk-local softmax and the unnormalised partial
+// output on the warp-level tensor-core MMA.  The chunk partials (o[D], m, l) are then merged with
+// the log-sum-exp rule: when a row's block list fits one thread-block cluster (16 CTAs), inside
+// the same kernel through distributed shared memory; otherwise through the workspace and a
+// second kernel launched with programmatic dependent launch.
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -19,6 +20,7 @@ namespace pa {
 constexpr int kDecBlock = 64;     // keys per block (the only supported block size)
 constexpr int kDecThreads = 128;  // threads per CTA of the partial kernel
 constexpr int kMaxGroup = 8;      // query heads per KV head supported by the partial kernel
+constexpr int kDecCluster = 16;   // CTAs per cluster of the single-kernel path
 
 struct DecodeArgs {
     const __nv_bfloat16 *q, *k, *v;
@@ -53,26 +55,37 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Partial attention of one 64-key block for all query heads of a KV group.
-//
-// Each of the four warps takes 16 keys and runs the two small contractions on the warp-level
-// tensor-core MMA (16 x 8 x 16): the query heads of the group are the M rows (rows beyond the
-// group are zero), so one pass over K and V serves every head.  K, V and Q are read straight
-// from global memory with 16-byte loads, all issued before the first use.  A thread's 16-byte
-// piece holds eight consecutive features of one row; the dot product does not care in which
-// order features are paired, so the pieces are fed to the MMA fragments as they come (Q and K
-// use the same pairing), and for P V two rows are interleaved with byte permutes.  The four
-// warps' (o, m, l) are merged in shared memory and one partial per head goes to the workspace.
-template <int D>
-__global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const DecodeArgs a)
+__device__ __forceinline__ float ex2_approx(float x)
 {
-    // Let the combine kernel's CTAs be scheduled as soon as SM resources free up.
-    asm volatile("griddepcontrol.launch_dependents;\n" ::);
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
 
+// Attention of one 64-key block for all query heads of a KV group, and (CLUSTER) the merge of
+// the row's blocks.
+//
+// Logits: each of the four warps takes 16 keys; the query heads of the group are the M rows of
+// the 16 x 8 x 16 MMA (rows beyond the group are zero), so one pass over K serves every head.
+// K, V and Q are read straight from global memory with 16-byte loads, all issued before the
+// first use.  A thread's 16-byte piece holds eight consecutive features of one row; the dot
+// product does not care in which order features are paired, so the pieces are fed to the MMA
+// fragments as they come (Q and K use the same pairing).  The logits go through shared memory
+// once so that every warp sees the whole 64-key row and the block's softmax uses one maximum.
+// Output: each warp owns 32 of the features and runs P V over all 64 keys for them (two rows of
+// V are interleaved with byte permutes to form the B fragments), so no cross-warp merge is needed.
+template <int D, bool CLUSTER>
+__global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeArgs a)
+{
+    namespace cg = cooperative_groups;
+    if (!CLUSTER) {
+        // Let the combine kernel's CTAs be scheduled as soon as SM resources free up.
+        asm volatile("griddepcontrol.launch_dependents;\n" ::);
+    }
     constexpr int NJ = D / 32;  // 16-byte pieces per thread and row for Q and K
-    constexpr int NV = D / 64;  // 16-byte pieces per thread and row for V
-    __shared__ float sO[4][kMaxGroup][D];
-    __shared__ float sM[4][kMaxGroup], sL[4][kMaxGroup];
+    __shared__ float sS[kMaxGroup][kDecBlock + 8];  // base-2 logits of the block
+    __shared__ float sPart[CLUSTER ? kMaxGroup * D : 1];  // this block's unnormalised output
+    __shared__ float sMl[2][kMaxGroup];                    // its maximum and sum per head
 
     const int chunk = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -80,119 +93,174 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(const Decod
     const int G = a.G;
 
     const int64_t len = a.lens[b];
-    if (len < 1 || len > a.max_len) return;
-    const int64_t p = len - 1, row = p / kDecBlock;
+    const bool valid = len >= 1 && len <= a.max_len;
+    const int64_t p = len - 1, row = valid ? p / kDecBlock : 0;
     // Every thread walks the (short) list; the chunk-th entry is this CTA's key block.
     int64_t jblk = -1;
-    const int n = for_each_key_block(row, a.W, a.S, [&](int pos, int64_t j) {
-        if (pos == chunk) jblk = j;
-    });
-    if (chunk >= n) return;
-    const int n_keys = jblk == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
-    const int base = wid * 16;  // first key of this warp inside the block
+    int n = 0;
+    if (valid)
+        n = for_each_key_block(row, a.W, a.S, [&](int pos, int64_t j) {
+            if (pos == chunk) jblk = j;
+        });
+    const bool active = chunk < n;
+    if (!CLUSTER && !active) return;
 
-    // ---- loads (keys at or beyond n_keys do not exist: zeros instead of a read)
-    const __nv_bfloat16 *kb = a.k + b * a.k_sb + (jblk * kDecBlock) * a.k_ss + hk * a.k_sh;
-    const __nv_bfloat16 *vb = a.v + b * a.v_sb + (jblk * kDecBlock) * a.v_ss + hk * a.v_sh;
-    const uint4 zero4 = make_uint4(0, 0, 0, 0);
-    uint4 kr[2][NJ], vr[4][NV], qr[NJ];
-#pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
-        const int key = base + nt * 8 + g;
-#pragma unroll
-        for (int j = 0; j < NJ; ++j) kr[nt][j] = key < n_keys ? ldg16(kb + key * a.k_ss + 8 * (4 * j + t)) : zero4;
-    }
-#pragma unroll
-    for (int kx = 0; kx < 4; ++kx) {
-        const int key = base + 2 * t + (kx & 1) + (kx >> 1) * 8;
-#pragma unroll
-        for (int jj = 0; jj < NV; ++jj) vr[kx][jj] = key < n_keys ? ldg16(vb + key * a.v_ss + 8 * (g + 8 * jj)) : zero4;
-    }
-    const __nv_bfloat16 *qb = a.q + ((int64_t)b * a.Hq + (int64_t)hk * G + g) * D;
-#pragma unroll
-    for (int j = 0; j < NJ; ++j) qr[j] = g < G ? ldg16(qb + 8 * (4 * j + t)) : zero4;
+    if (active) {
+        const int n_keys = jblk == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
+        const int base = wid * 16;            // first key of this warp's logit tile
+        const int vchunk = (g & 3) + 4 * wid;  // this thread's 8-feature piece of V rows
+        const bool pv_warp = 4 * wid < D / 8;  // warps that own output features
 
-    // ---- S = Q K^T: rows = heads, columns = the warp's 16 keys (two 8-key tiles)
-    float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        // ---- loads (keys at or beyond n_keys do not exist: zeros instead of a read)
+        const __nv_bfloat16 *kb = a.k + b * a.k_sb + (jblk * kDecBlock) * a.k_ss + hk * a.k_sh;
+        const __nv_bfloat16 *vb = a.v + b * a.v_sb + (jblk * kDecBlock) * a.v_ss + hk * a.v_sh;
+        const uint4 zero4 = make_uint4(0, 0, 0, 0);
+        uint4 kr[2][NJ], vr[4][4], qr[NJ];
 #pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
+        for (int nt = 0; nt < 2; ++nt) {
+            const int key = base + nt * 8 + g;
 #pragma unroll
-        for (int j = 0; j < NJ; ++j) {
-            mma_bf16(sc[nt], qr[j].x, 0u, qr[j].y, 0u, kr[nt][j].x, kr[nt][j].y);
-            mma_bf16(sc[nt], qr[j].z, 0u, qr[j].w, 0u, kr[nt][j].z, kr[nt][j].w);
+            for (int j = 0; j < NJ; ++j)
+                kr[nt][j] = key < n_keys ? ldg16(kb + key * a.k_ss + 8 * (4 * j + t)) : zero4;
         }
-    }
-    // This thread holds head g, keys base + 8 nt + 2 t + {0, 1}.  Softmax over the warp's keys in
-    // the base-2 domain: s2 = s * scale * log2(e).
-    float s2[2][2];
-    float mw = -INFINITY;
+        const __nv_bfloat16 *qb = a.q + ((int64_t)b * a.Hq + (int64_t)hk * G + g) * D;
 #pragma unroll
-    for (int nt = 0; nt < 2; ++nt)
+        for (int j = 0; j < NJ; ++j) qr[j] = g < G ? ldg16(qb + 8 * (4 * j + t)) : zero4;
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
-            const int key = base + nt * 8 + 2 * t + x;
-            s2[nt][x] = key < n_keys ? sc[nt][x] * a.scale_log2 : -INFINITY;
-            mw = fmaxf(mw, s2[nt][x]);
-        }
-    mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, 1));
-    mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, 2));
-    float pe[2][2], lw = 0.f;
+        for (int ks = 0; ks < 4; ++ks)
 #pragma unroll
-    for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-            pe[nt][x] = mw == -INFINITY ? 0.f : exp2f(s2[nt][x] - mw);
-            lw += pe[nt][x];
-        }
-    lw += __shfl_xor_sync(0xffffffffu, lw, 1);
-    lw += __shfl_xor_sync(0xffffffffu, lw, 2);
-    // P as the A operand of P V: columns 2t, 2t+1 (first key tile) and 2t+8, 2t+9 (second).
-    const __nv_bfloat162 p01 = __floats2bfloat162_rn(pe[0][0], pe[0][1]);
-    const __nv_bfloat162 p23 = __floats2bfloat162_rn(pe[1][0], pe[1][1]);
-    const uint32_t pa0 = *reinterpret_cast<const uint32_t *>(&p01), pa2 = *reinterpret_cast<const uint32_t *>(&p23);
+            for (int kx = 0; kx < 4; ++kx) {
+                const int key = 16 * ks + 2 * t + (kx & 1) + (kx >> 1) * 8;
+                vr[ks][kx] = (pv_warp && key < n_keys) ? ldg16(vb + key * a.v_ss + 8 * vchunk) : zero4;
+            }
 
-    // ---- O = P V: the B operand pairs two keys per register; feature tile (jj, e) of this
-    // thread's quad covers features 8 (n + 8 jj) + e, n = 0..7.
-    {
+        // ---- S = Q K^T: rows = heads, columns = the warp's 16 keys (two 8-key tiles)
+        float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
-        for (int jj = 0; jj < NV; ++jj) {
-            const uint32_t v0[4] = {vr[0][jj].x, vr[0][jj].y, vr[0][jj].z, vr[0][jj].w};
-            const uint32_t v1[4] = {vr[1][jj].x, vr[1][jj].y, vr[1][jj].z, vr[1][jj].w};
-            const uint32_t v2[4] = {vr[2][jj].x, vr[2][jj].y, vr[2][jj].z, vr[2][jj].w};
-            const uint32_t v3[4] = {vr[3][jj].x, vr[3][jj].y, vr[3][jj].z, vr[3][jj].w};
+        for (int nt = 0; nt < 2; ++nt) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
-                const uint32_t b0 = __byte_perm(v0[e >> 1], v1[e >> 1], sel);
-                const uint32_t b1 = __byte_perm(v2[e >> 1], v3[e >> 1], sel);
-                float oc[4] = {0.f, 0.f, 0.f, 0.f};
-                mma_bf16(oc, pa0, 0u, pa2, 0u, b0, b1);
-                // oc[0], oc[1]: head g, features 8 (2t + x + 8 jj) + e
-                if (g < G) {
-                    sO[wid][g][8 * (2 * t + 8 * jj) + e] = oc[0];
-                    sO[wid][g][8 * (2 * t + 1 + 8 * jj) + e] = oc[1];
+            for (int j = 0; j < NJ; ++j) {
+                mma_bf16(sc[nt], qr[j].x, 0u, qr[j].y, 0u, kr[nt][j].x, kr[nt][j].y);
+                mma_bf16(sc[nt], qr[j].z, 0u, qr[j].w, 0u, kr[nt][j].z, kr[nt][j].w);
+            }
+        }
+        // This thread holds head g, keys base + 8 nt + 2 t + {0, 1}: to shared memory in the
+        // base-2 domain (s * scale * log2(e)); keys that do not exist become -inf.
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+            const int key = base + nt * 8 + 2 * t;
+            float2 v2;
+            v2.x = key < n_keys ? sc[nt][0] * a.scale_log2 : -INFINITY;
+            v2.y = key + 1 < n_keys ? sc[nt][1] * a.scale_log2 : -INFINITY;
+            *reinterpret_cast<float2 *>(&sS[g][key]) = v2;
+        }
+        __syncthreads();
+
+        // ---- block softmax: thread (g, t) takes keys 16 ks + {2t, 2t+1, 2t+8, 2t+9}, ks = 0..3
+        // (exactly the positions of its P fragments); the four t lanes cover the row.
+        float2 sv[4][2];
+        float mrow = -INFINITY;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                sv[ks][hh] = *reinterpret_cast<const float2 *>(&sS[g][16 * ks + 8 * hh + 2 * t]);
+                mrow = fmaxf(mrow, fmaxf(sv[ks][hh].x, sv[ks][hh].y));
+            }
+        mrow = fmaxf(mrow, __shfl_xor_sync(0xffffffffu, mrow, 1));
+        mrow = fmaxf(mrow, __shfl_xor_sync(0xffffffffu, mrow, 2));  // finite: key 0 of the block exists
+        uint32_t pa[4][2];
+        float lrow = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const float p0 = ex2_approx(sv[ks][hh].x - mrow), p1 = ex2_approx(sv[ks][hh].y - mrow);
+                lrow += p0 + p1;
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+                pa[ks][hh] = *reinterpret_cast<const uint32_t *>(&h2);
+            }
+        lrow += __shfl_xor_sync(0xffffffffu, lrow, 1);
+        lrow += __shfl_xor_sync(0xffffffffu, lrow, 2);
+        if (wid == 0 && t == 0 && g < G) {
+            sMl[0][g] = mrow;
+            sMl[1][g] = lrow;
+            if (!CLUSTER) {
+                float *dst = a.partial + (((int64_t)b * a.Hq + hk * G + g) * a.chunks + chunk) * (D + 2);
+                dst[D] = mrow;      // base-2 maximum of the block
+                dst[D + 1] = lrow;  // sum of 2^(s2 - m)
+            }
+        }
+
+        // ---- O = P V for this warp's 32 features.  Lanes g and g + 4 read the same 16-byte piece
+        // and take its low / high half: feature tile e covers features 8 vchunk(n) + e + 4 (n >> 2)
+        // for n = 0..7.
+        if (pv_warp) {
+            const bool hi = (g >> 2) != 0;
+            float acc[4][4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[e][0] = acc[e][1] = acc[e][2] = acc[e][3] = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                uint32_t w0[2], w1[2], w2[2], w3[2];  // the two 32-bit words this lane uses, per key
+                w0[0] = hi ? vr[ks][0].z : vr[ks][0].x; w0[1] = hi ? vr[ks][0].w : vr[ks][0].y;
+                w1[0] = hi ? vr[ks][1].z : vr[ks][1].x; w1[1] = hi ? vr[ks][1].w : vr[ks][1].y;
+                w2[0] = hi ? vr[ks][2].z : vr[ks][2].x; w2[1] = hi ? vr[ks][2].w : vr[ks][2].y;
+                w3[0] = hi ? vr[ks][3].z : vr[ks][3].x; w3[1] = hi ? vr[ks][3].w : vr[ks][3].y;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
+                    const uint32_t b0 = __byte_perm(w0[e >> 1], w1[e >> 1], sel);
+                    const uint32_t b1 = __byte_perm(w2[e >> 1], w3[e >> 1], sel);
+                    mma_bf16(acc[e], pa[ks][0], 0u, pa[ks][1], 0u, b0, b1);
                 }
+            }
+            // acc[e][x]: head g, column n = 2t + x of the tile -> feature below.
+            if (g < G) {
+                float *dst = CLUSTER ? &sPart[g * D]
+                                     : a.partial + (((int64_t)b * a.Hq + hk * G + g) * a.chunks + chunk) * (D + 2);
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+#pragma unroll
+                    for (int x = 0; x < 2; ++x) {
+                        const int nn = 2 * t + x;
+                        dst[8 * ((nn & 3) + 4 * wid) + e + 4 * (nn >> 2)] = acc[e][x];
+                    }
             }
         }
     }
-    if (t == 0 && g < G) {
-        sM[wid][g] = mw;
-        sL[wid][g] = lw;
-    }
-    __syncthreads();
 
-    // ---- merge the four warps and write one partial (o[D], m, l) per head
-    for (int idx = tid; idx < G * D; idx += kDecThreads) {
-        const int h = idx / D, d = idx % D;
-        const float m0 = sM[0][h], m1 = sM[1][h], m2 = sM[2][h], m3 = sM[3][h];
-        const float m = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));  // finite: key 0 of the block exists
-        const float w0 = exp2f(m0 - m), w1 = exp2f(m1 - m), w2 = exp2f(m2 - m), w3 = exp2f(m3 - m);
-        float *dst = a.partial + (((int64_t)b * a.Hq + hk * G + h) * a.chunks + chunk) * (D + 2);
-        dst[d] = sO[0][h][d] * w0 + sO[1][h][d] * w1 + sO[2][h][d] * w2 + sO[3][h][d] * w3;
-        if (d == 0) {
-            dst[D] = m;
-            dst[D + 1] = sL[0][h] * w0 + sL[1][h] * w1 + sL[2][h] * w2 + sL[3][h] * w3;
+    if (CLUSTER) {
+        // ---- merge the row's blocks across the cluster (rank = chunk): every CTA, busy or not,
+        // takes a slice of the (head, feature) outputs and reads the partials of the n active
+        // CTAs from their shared memory:  m = max m_c,  l = sum l_c 2^(m_c - m),
+        // o = sum o_c 2^(m_c - m) / l,  LSE = (m + log2 l) ln 2.
+        cg::cluster_group cluster = cg::this_cluster();
+        cluster.sync();
+        const int per = (G * D + kDecCluster - 1) / kDecCluster;
+        const int elem = chunk * per + tid;
+        if (tid < per && elem < G * D) {
+            const int h = elem / D, d = elem % D;
+            float m = -INFINITY;
+#pragma unroll 4
+            for (int c = 0; c < n; ++c) m = fmaxf(m, cluster.map_shared_rank(&sMl[0][0], c)[h]);
+            float l = 0.f, acc = 0.f;
+#pragma unroll 4
+            for (int c = 0; c < n; ++c) {
+                const float w = ex2_approx(cluster.map_shared_rank(&sMl[0][0], c)[h] - m);
+                l += cluster.map_shared_rank(&sMl[1][0], c)[h] * w;
+                acc += cluster.map_shared_rank(&sPart[0], c)[h * D + d] * w;
+            }
+            const float out = n > 0 ? acc / l : 0.f;
+            const int64_t oi = ((int64_t)b * a.Hq + hk * G + h) * D + d;
+            if (a.o_is_f32)
+                reinterpret_cast<float *>(a.o)[oi] = out;
+            else
+                reinterpret_cast<__nv_bfloat16 *>(a.o)[oi] = __float2bfloat16_rn(out);
+            if (d == 0)
+                a.lse[(int64_t)b * a.Hq + hk * G + h] = n > 0 ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
         }
+        cluster.sync();  // peers' shared memory stays alive until every read is done
     }
 }
 
@@ -249,9 +317,12 @@ __global__ void decode_block_list_kernel(int64_t len, int32_t W, int32_t S, int3
 // Upper bound on the number of listed blocks of any row below n_rows.
 static int max_row_blocks(int64_t n_rows, int32_t W, int32_t S)
 {
-    int bits = 0;
-    for (int64_t x = n_rows > 0 ? n_rows - 1 : 0; x > 0; x >>= 1) ++bits;
-    int64_t bound = (int64_t)(W > 1 ? W : 1) + S + bits;
+    // window distances 0 .. w-1, every power of two 2^k >= w with 2^k <= n_rows - 1, sink blocks
+    const int64_t w = W > 1 ? W : 1;
+    int powers = 0;
+    for (int64_t pw = 1; pw <= n_rows - 1; pw *= 2)
+        if (pw >= w) ++powers;
+    const int64_t bound = w + S + powers;
     return (int)(bound < n_rows ? bound : n_rows);
 }
 
@@ -331,11 +402,34 @@ extern "C" pa_status pa_decode(const pa_decode_params *p, const void *q, const v
     a.scale_log2 = scale * 1.4426950408889634f;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (a.chunks <= kDecCluster) {
+        // One kernel: the row's blocks form one cluster and merge through distributed shared memory.
+        cudaLaunchConfig_t ccfg = {};
+        ccfg.gridDim = dim3(kDecCluster, (unsigned)a.Hkv, (unsigned)a.batch);
+        ccfg.blockDim = dim3(kDecThreads, 1, 1);
+        ccfg.dynamicSmemBytes = 0;
+        ccfg.stream = st;
+        cudaLaunchAttribute cattr[1];
+        cattr[0].id = cudaLaunchAttributeClusterDimension;
+        cattr[0].val.clusterDim.x = kDecCluster;
+        cattr[0].val.clusterDim.y = 1;
+        cattr[0].val.clusterDim.z = 1;
+        ccfg.attrs = cattr;
+        ccfg.numAttrs = 1;
+        if (p->head_dim == 128) {
+            PA_CUDA_OK(cudaFuncSetAttribute(decode_block_kernel<128, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+            PA_CUDA_OK(cudaLaunchKernelEx(&ccfg, decode_block_kernel<128, true>, a));
+        } else {
+            PA_CUDA_OK(cudaFuncSetAttribute(decode_block_kernel<64, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+            PA_CUDA_OK(cudaLaunchKernelEx(&ccfg, decode_block_kernel<64, true>, a));
+        }
+        return PA_OK;
+    }
     const dim3 grid1((unsigned)a.chunks, (unsigned)a.Hkv, (unsigned)a.batch);
     if (p->head_dim == 128)
-        decode_partial_kernel<128><<<grid1, kDecThreads, 0, st>>>(a);
+        decode_block_kernel<128, false><<<grid1, kDecThreads, 0, st>>>(a);
     else
-        decode_partial_kernel<64><<<grid1, kDecThreads, 0, st>>>(a);
+        decode_block_kernel<64, false><<<grid1, kDecThreads, 0, st>>>(a);
     PA_CUDA_OK(cudaGetLastError());
 
     cudaLaunchConfig_t cfg = {};
