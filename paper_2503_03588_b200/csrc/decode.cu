@@ -21,6 +21,7 @@ constexpr int kDecBlock = 64;     // keys per block (the only supported block si
 constexpr int kDecThreads = 128;  // threads per CTA of the partial kernel
 constexpr int kMaxGroup = 8;      // query heads per KV head supported by the partial kernel
 constexpr int kDecCluster = 16;   // CTAs per cluster of the single-kernel path
+constexpr int kRecvStride = 80;   // floats per sender in a CTA's receive buffer: 64 outputs, 8 m, 8 l
 
 struct DecodeArgs {
     const __nv_bfloat16 *q, *k, *v;
@@ -84,7 +85,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
     }
     constexpr int NJ = D / 32;  // 16-byte pieces per thread and row for Q and K
     __shared__ float sS[kMaxGroup][kDecBlock + 8];  // base-2 logits of the block
-    __shared__ float sPart[CLUSTER ? kMaxGroup * D : 1];  // this block's unnormalised output
+    __shared__ float sRecv[CLUSTER ? kDecCluster * kRecvStride : 1];  // slices sent by the row's blocks
     __shared__ float sMl[2][kMaxGroup];                    // its maximum and sum per head
 
     const int chunk = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
@@ -94,12 +95,14 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
 
     const int64_t len = a.lens[b];
     const bool valid = len >= 1 && len <= a.max_len;
-    const int64_t p = len - 1, row = valid ? p / kDecBlock : 0;
+    if (CLUSTER) asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");  // "I have started"
+    const int64_t p = len - 1;
+    const int32_t row = valid ? (int32_t)(p / kDecBlock) : 0;  // max_len / 64 fits in 31 bits (host check)
     // Every thread walks the (short) list; the chunk-th entry is this CTA's key block.
-    int64_t jblk = -1;
+    int32_t jblk = -1;
     int n = 0;
     if (valid)
-        n = for_each_key_block(row, a.W, a.S, [&](int pos, int64_t j) {
+        n = for_each_key_block_t<int32_t>(row, a.W, a.S, [&](int pos, int32_t j) {
             if (pos == chunk) jblk = j;
         });
     const bool active = chunk < n;
@@ -112,8 +115,8 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
         const bool pv_warp = 4 * wid < D / 8;  // warps that own output features
 
         // ---- loads (keys at or beyond n_keys do not exist: zeros instead of a read)
-        const __nv_bfloat16 *kb = a.k + b * a.k_sb + (jblk * kDecBlock) * a.k_ss + hk * a.k_sh;
-        const __nv_bfloat16 *vb = a.v + b * a.v_sb + (jblk * kDecBlock) * a.v_ss + hk * a.v_sh;
+        const __nv_bfloat16 *kb = a.k + b * a.k_sb + ((int64_t)jblk * kDecBlock) * a.k_ss + hk * a.k_sh;
+        const __nv_bfloat16 *vb = a.v + b * a.v_sb + ((int64_t)jblk * kDecBlock) * a.v_ss + hk * a.v_sh;
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
         uint4 kr[2][NJ], vr[4][4], qr[NJ];
 #pragma unroll
@@ -182,10 +185,10 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
             }
         lrow += __shfl_xor_sync(0xffffffffu, lrow, 1);
         lrow += __shfl_xor_sync(0xffffffffu, lrow, 2);
-        if (wid == 0 && t == 0 && g < G) {
+        if (wid == 0 && t == 0 && g < kMaxGroup) {
             sMl[0][g] = mrow;
             sMl[1][g] = lrow;
-            if (!CLUSTER) {
+            if (!CLUSTER && g < G) {
                 float *dst = a.partial + (((int64_t)b * a.Hq + hk * G + g) * a.chunks + chunk) * (D + 2);
                 dst[D] = mrow;      // base-2 maximum of the block
                 dst[D + 1] = lrow;  // sum of 2^(s2 - m)
@@ -216,9 +219,26 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
                 }
             }
             // acc[e][x]: head g, column n = 2t + x of the tile -> feature below.
-            if (g < G) {
-                float *dst = CLUSTER ? &sPart[g * D]
-                                     : a.partial + (((int64_t)b * a.Hq + hk * G + g) * a.chunks + chunk) * (D + 2);
+            if (CLUSTER) {
+                // Every CTA of the cluster has started (it arrived at the barrier on entry), so its
+                // shared memory may be written.  Output element (head, feature) belongs to the CTA
+                // that will finish it: slices of `per` consecutive elements in cluster-rank order.
+                asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+                if (g < G) {
+                    cg::cluster_group cluster = cg::this_cluster();
+                    const int per = (G * D + kDecCluster - 1) / kDecCluster;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+#pragma unroll
+                        for (int x = 0; x < 2; ++x) {
+                            const int nn = 2 * t + x;
+                            const int elem = g * D + 8 * ((nn & 3) + 4 * wid) + e + 4 * (nn >> 2);
+                            const int owner = elem / per;
+                            cluster.map_shared_rank(&sRecv[0], owner)[chunk * kRecvStride + (elem - owner * per)] = acc[e][x];
+                        }
+                }
+            } else if (g < G) {
+                float *dst = a.partial + (((int64_t)b * a.Hq + hk * G + g) * a.chunks + chunk) * (D + 2);
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
 #pragma unroll
@@ -227,14 +247,28 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
                         dst[8 * ((nn & 3) + 4 * wid) + e + 4 * (nn >> 2)] = acc[e][x];
                     }
             }
+        } else if (CLUSTER) {
+            asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
         }
+        if (CLUSTER) {
+            // This block's maximum and sum per head, to every CTA of the cluster.
+            __syncthreads();
+            cg::cluster_group cluster = cg::this_cluster();
+            const int owner = tid & (kDecCluster - 1), h = tid >> 4;
+            float *dst = cluster.map_shared_rank(&sRecv[0], owner) + chunk * kRecvStride;
+            dst[64 + h] = sMl[0][h];
+            dst[72 + h] = sMl[1][h];
+        }
+    } else if (CLUSTER) {
+        asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
     }
 
     if (CLUSTER) {
-        // ---- merge the row's blocks across the cluster (rank = chunk): every CTA, busy or not,
-        // takes a slice of the (head, feature) outputs and reads the partials of the n active
-        // CTAs from their shared memory:  m = max m_c,  l = sum l_c 2^(m_c - m),
-        // o = sum o_c 2^(m_c - m) / l,  LSE = (m + log2 l) ln 2.
+        // ---- merge the row's blocks (cluster rank = chunk).  Every CTA, busy or not, finishes a
+        // slice of the (head, feature) outputs from what the n active CTAs sent to its shared
+        // memory:  m = max m_c,  l = sum l_c 2^(m_c - m),  o = sum o_c 2^(m_c - m) / l,
+        // LSE = (m + log2 l) ln 2.  Nothing is read remotely after this barrier, so a CTA may
+        // exit as soon as its slice is written.
         cg::cluster_group cluster = cg::this_cluster();
         cluster.sync();
         const int per = (G * D + kDecCluster - 1) / kDecCluster;
@@ -242,14 +276,12 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
         if (tid < per && elem < G * D) {
             const int h = elem / D, d = elem % D;
             float m = -INFINITY;
-#pragma unroll 4
-            for (int c = 0; c < n; ++c) m = fmaxf(m, cluster.map_shared_rank(&sMl[0][0], c)[h]);
+            for (int c = 0; c < n; ++c) m = fmaxf(m, sRecv[c * kRecvStride + 64 + h]);
             float l = 0.f, acc = 0.f;
-#pragma unroll 4
             for (int c = 0; c < n; ++c) {
-                const float w = ex2_approx(cluster.map_shared_rank(&sMl[0][0], c)[h] - m);
-                l += cluster.map_shared_rank(&sMl[1][0], c)[h] * w;
-                acc += cluster.map_shared_rank(&sPart[0], c)[h * D + d] * w;
+                const float w = ex2_approx(sRecv[c * kRecvStride + 64 + h] - m);
+                l += sRecv[c * kRecvStride + 72 + h] * w;
+                acc += sRecv[c * kRecvStride + tid] * w;
             }
             const float out = n > 0 ? acc / l : 0.f;
             const int64_t oi = ((int64_t)b * a.Hq + hk * G + h) * D + d;
@@ -260,7 +292,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
             if (d == 0)
                 a.lse[(int64_t)b * a.Hq + hk * G + h] = n > 0 ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
         }
-        cluster.sync();  // peers' shared memory stays alive until every read is done
     }
 }
 
@@ -339,6 +370,7 @@ static pa_status check_decode(const pa_decode_params *p)
     if (p->n_q_heads % p->n_kv_heads) return fail(PA_ERR_SHAPE, "n_q_heads must be a multiple of n_kv_heads");
     if (p->n_q_heads / p->n_kv_heads > kMaxGroup)
         return fail(PA_ERR_SHAPE, "at most %d query heads per KV head", kMaxGroup);
+    if (p->max_len > ((int64_t)1 << 36)) return fail(PA_ERR_SHAPE, "max_len too large");
     if (p->batch > 65535 || p->n_kv_heads > 65535 || p->n_q_heads > 65535)
         return fail(PA_ERR_SHAPE, "batch and head counts must be <= 65535");
     if (p->window_blocks > 4096 || p->sink_blocks > 4096)

@@ -12,26 +12,27 @@
 namespace pa {
 
 // Calls emit(pos, j) for every listed key block j of query block i in ascending order and
-// returns the row length.  i >= 0, W >= 0, S >= 0.
-template <typename Emit>
-__host__ __device__ inline int for_each_key_block(int64_t i, int32_t W, int32_t S, Emit emit)
+// returns the row length.  i >= 0, W >= 0, S >= 0.  Index is int64_t, or int32_t where the block
+// indices are known to fit (the decode kernel: a cheaper walk on its critical path).
+template <typename Index, typename Emit>
+__host__ __device__ inline int for_each_key_block_t(Index i, int32_t W, int32_t S, Emit emit)
 {
-    const int64_t w_eff = W > 1 ? W : 1;
-    const int64_t sink_end = (int64_t)S < i + 1 ? (int64_t)S : i + 1;  // sink run [0, sink_end)
-    int64_t js = 0;                                                    // sink cursor
-    int64_t jw = i - w_eff + 1 > 0 ? i - w_eff + 1 : 0;                // window cursor .. i
-    int64_t pw = 0;                                                    // current power distance
+    const Index w_eff = W > 1 ? (Index)W : (Index)1;
+    const Index sink_end = (Index)S < i + 1 ? (Index)S : i + 1;  // sink run [0, sink_end)
+    Index js = 0;                                                // sink cursor
+    Index jw = i - w_eff + 1 > 0 ? i - w_eff + 1 : 0;            // window cursor .. i
+    Index pw = 0;                                                // current power distance
     if (i >= 1) {
         pw = 1;
-        while (pw * 2 <= i) pw *= 2;                                   // largest 2^k <= i
+        while (pw <= i / 2) pw *= 2;                             // largest 2^k <= i
     }
-    const int64_t kNone = INT64_MAX;
+    const Index kNone = sizeof(Index) == 8 ? (Index)INT64_MAX : (Index)INT32_MAX;
     int n = 0;
     while (true) {
-        const int64_t a = js < sink_end ? js : kNone;
-        const int64_t b = pw >= 1 ? i - pw : kNone;
-        const int64_t c = jw <= i ? jw : kNone;
-        int64_t j = a < b ? a : b;
+        const Index a = js < sink_end ? js : kNone;
+        const Index b = pw >= 1 ? i - pw : kNone;
+        const Index c = jw <= i ? jw : kNone;
+        Index j = a < b ? a : b;
         j = j < c ? j : c;
         if (j == kNone) break;
         emit(n, j);
@@ -41,6 +42,12 @@ __host__ __device__ inline int for_each_key_block(int64_t i, int32_t W, int32_t 
         if (c == j) ++jw;
     }
     return n;
+}
+
+template <typename Emit>
+__host__ __device__ inline int for_each_key_block(int64_t i, int32_t W, int32_t S, Emit emit)
+{
+    return for_each_key_block_t<int64_t>(i, W, S, emit);
 }
 
 struct NoEmit {
