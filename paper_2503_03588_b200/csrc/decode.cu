@@ -5,10 +5,8 @@
 // row's block list.  Each CTA reads its K and V block with coalesced 16-byte loads and computes
 // the logits of all query heads of the group, a chunk-local softmax and the unnormalised partial
 // output on the warp-level tensor-core MMA.  The chunk partials (o[D], m, l) are then merged with
-// the log-sum-exp rule: when a row's block list fits one thread-block cluster (16 CTAs), inside
-// the same kernel through distributed shared memory; otherwise through the workspace and a
-// second kernel launched with programmatic dependent launch.
-#include <cooperative_groups.h>
+// the log-sum-exp rule by a second kernel, launched with programmatic dependent launch so that
+// its start-up overlaps the first kernel's tail; it waits for the partials with griddepcontrol.wait.
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -20,8 +18,6 @@ namespace pa {
 constexpr int kDecBlock = 64;     // keys per block (the only supported block size)
 constexpr int kDecThreads = 128;  // threads per CTA of the partial kernel
 constexpr int kMaxGroup = 8;      // query heads per KV head supported by the partial kernel
-constexpr int kDecCluster = 16;   // CTAs per cluster of the single-kernel path
-constexpr int kRecvStride = 80;   // floats per sender in a CTA's receive buffer: 64 outputs, 8 m, 8 l
 
 struct DecodeArgs {
     const __nv_bfloat16 *q, *k, *v;
@@ -63,8 +59,7 @@ __device__ __forceinline__ float ex2_approx(float x)
     return y;
 }
 
-// Attention of one 64-key block for all query heads of a KV group, and (CLUSTER) the merge of
-// the row's blocks.
+// Attention of one 64-key block for all query heads of a KV group.
 //
 // Logits: each of the four warps takes 16 keys; the query heads of the group are the M rows of
 // the 16 x 8 x 16 MMA (rows beyond the group are zero), so one pass over K serves every head.
@@ -75,18 +70,13 @@ __device__ __forceinline__ float ex2_approx(float x)
 // once so that every warp sees the whole 64-key row and the block's softmax uses one maximum.
 // Output: each warp owns 32 of the features and runs P V over all 64 keys for them (two rows of
 // V are interleaved with byte permutes to form the B fragments), so no cross-warp merge is needed.
-template <int D, bool CLUSTER>
+template <int D>
 __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeArgs a)
 {
-    namespace cg = cooperative_groups;
-    if (!CLUSTER) {
-        // Let the combine kernel's CTAs be scheduled as soon as SM resources free up.
-        asm volatile("griddepcontrol.launch_dependents;\n" ::);
-    }
+    // Let the combine kernel's CTAs be scheduled as soon as SM resources free up.
+    asm volatile("griddepcontrol.launch_dependents;\n" ::);
     constexpr int NJ = D / 32;  // 16-byte pieces per thread and row for Q and K
     __shared__ float sS[kMaxGroup][kDecBlock + 8];  // base-2 logits of the block
-    __shared__ float sRecv[CLUSTER ? kDecCluster * kRecvStride : 1];  // slices sent by the row's blocks
-    __shared__ float sMl[2][kMaxGroup];                    // its maximum and sum per head
 
     const int chunk = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -95,7 +85,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
 
     const int64_t len = a.lens[b];
     const bool valid = len >= 1 && len <= a.max_len;
-    if (CLUSTER) asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");  // "I have started"
     const int64_t p = len - 1;
     const int32_t row = valid ? (int32_t)(p / kDecBlock) : 0;  // max_len / 64 fits in 31 bits (host check)
     // Every thread walks the (short) list; the chunk-th entry is this CTA's key block.
@@ -105,10 +94,9 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
         n = for_each_key_block_t<int32_t>(row, a.W, a.S, [&](int pos, int32_t j) {
             if (pos == chunk) jblk = j;
         });
-    const bool active = chunk < n;
-    if (!CLUSTER && !active) return;
+    if (chunk >= n) return;
 
-    if (active) {
+    {
         const int n_keys = jblk == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
         const int base = wid * 16;            // first key of this warp's logit tile
         const int vchunk = (g & 3) + 4 * wid;  // this thread's 8-feature piece of V rows
@@ -185,14 +173,10 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
             }
         lrow += __shfl_xor_sync(0xffffffffu, lrow, 1);
         lrow += __shfl_xor_sync(0xffffffffu, lrow, 2);
-        if (wid == 0 && t == 0 && g < kMaxGroup) {
-            sMl[0][g] = mrow;
-            sMl[1][g] = lrow;
-            if (!CLUSTER && g < G) {
-                float *dst = a.partial + (((int64_t)b * a.Hq + hk * G + g) * a.chunks + chunk) * (D + 2);
-                dst[D] = mrow;      // base-2 maximum of the block
-                dst[D + 1] = lrow;  // sum of 2^(s2 - m)
-            }
+        if (wid == 0 && t == 0 && g < G) {
+            float *dst = a.partial + (((int64_t)b * a.Hq + hk * G + g) * a.chunks + chunk) * (D + 2);
+            dst[D] = mrow;      // base-2 maximum of the block
+            dst[D + 1] = lrow;  // sum of 2^(s2 - m)
         }
 
         // ---- O = P V for this warp's 32 features.  Lanes g and g + 4 read the same 16-byte piece
@@ -219,25 +203,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
                 }
             }
             // acc[e][x]: head g, column n = 2t + x of the tile -> feature below.
-            if (CLUSTER) {
-                // Every CTA of the cluster has started (it arrived at the barrier on entry), so its
-                // shared memory may be written.  Output element (head, feature) belongs to the CTA
-                // that will finish it: slices of `per` consecutive elements in cluster-rank order.
-                asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
-                if (g < G) {
-                    cg::cluster_group cluster = cg::this_cluster();
-                    const int per = (G * D + kDecCluster - 1) / kDecCluster;
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-#pragma unroll
-                        for (int x = 0; x < 2; ++x) {
-                            const int nn = 2 * t + x;
-                            const int elem = g * D + 8 * ((nn & 3) + 4 * wid) + e + 4 * (nn >> 2);
-                            const int owner = elem / per;
-                            cluster.map_shared_rank(&sRecv[0], owner)[chunk * kRecvStride + (elem - owner * per)] = acc[e][x];
-                        }
-                }
-            } else if (g < G) {
+            if (g < G) {
                 float *dst = a.partial + (((int64_t)b * a.Hq + hk * G + g) * a.chunks + chunk) * (D + 2);
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
@@ -247,50 +213,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_block_kernel(const DecodeA
                         dst[8 * ((nn & 3) + 4 * wid) + e + 4 * (nn >> 2)] = acc[e][x];
                     }
             }
-        } else if (CLUSTER) {
-            asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
-        }
-        if (CLUSTER) {
-            // This block's maximum and sum per head, to every CTA of the cluster.
-            __syncthreads();
-            cg::cluster_group cluster = cg::this_cluster();
-            const int owner = tid & (kDecCluster - 1), h = tid >> 4;
-            float *dst = cluster.map_shared_rank(&sRecv[0], owner) + chunk * kRecvStride;
-            dst[64 + h] = sMl[0][h];
-            dst[72 + h] = sMl[1][h];
-        }
-    } else if (CLUSTER) {
-        asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
-    }
-
-    if (CLUSTER) {
-        // ---- merge the row's blocks (cluster rank = chunk).  Every CTA, busy or not, finishes a
-        // slice of the (head, feature) outputs from what the n active CTAs sent to its shared
-        // memory:  m = max m_c,  l = sum l_c 2^(m_c - m),  o = sum o_c 2^(m_c - m) / l,
-        // LSE = (m + log2 l) ln 2.  Nothing is read remotely after this barrier, so a CTA may
-        // exit as soon as its slice is written.
-        cg::cluster_group cluster = cg::this_cluster();
-        cluster.sync();
-        const int per = (G * D + kDecCluster - 1) / kDecCluster;
-        const int elem = chunk * per + tid;
-        if (tid < per && elem < G * D) {
-            const int h = elem / D, d = elem % D;
-            float m = -INFINITY;
-            for (int c = 0; c < n; ++c) m = fmaxf(m, sRecv[c * kRecvStride + 64 + h]);
-            float l = 0.f, acc = 0.f;
-            for (int c = 0; c < n; ++c) {
-                const float w = ex2_approx(sRecv[c * kRecvStride + 64 + h] - m);
-                l += sRecv[c * kRecvStride + 72 + h] * w;
-                acc += sRecv[c * kRecvStride + tid] * w;
-            }
-            const float out = n > 0 ? acc / l : 0.f;
-            const int64_t oi = ((int64_t)b * a.Hq + hk * G + h) * D + d;
-            if (a.o_is_f32)
-                reinterpret_cast<float *>(a.o)[oi] = out;
-            else
-                reinterpret_cast<__nv_bfloat16 *>(a.o)[oi] = __float2bfloat16_rn(out);
-            if (d == 0)
-                a.lse[(int64_t)b * a.Hq + hk * G + h] = n > 0 ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
         }
     }
 }
@@ -434,34 +356,11 @@ extern "C" pa_status pa_decode(const pa_decode_params *p, const void *q, const v
     a.scale_log2 = scale * 1.4426950408889634f;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (a.chunks <= kDecCluster) {
-        // One kernel: the row's blocks form one cluster and merge through distributed shared memory.
-        cudaLaunchConfig_t ccfg = {};
-        ccfg.gridDim = dim3(kDecCluster, (unsigned)a.Hkv, (unsigned)a.batch);
-        ccfg.blockDim = dim3(kDecThreads, 1, 1);
-        ccfg.dynamicSmemBytes = 0;
-        ccfg.stream = st;
-        cudaLaunchAttribute cattr[1];
-        cattr[0].id = cudaLaunchAttributeClusterDimension;
-        cattr[0].val.clusterDim.x = kDecCluster;
-        cattr[0].val.clusterDim.y = 1;
-        cattr[0].val.clusterDim.z = 1;
-        ccfg.attrs = cattr;
-        ccfg.numAttrs = 1;
-        if (p->head_dim == 128) {
-            PA_CUDA_OK(cudaFuncSetAttribute(decode_block_kernel<128, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-            PA_CUDA_OK(cudaLaunchKernelEx(&ccfg, decode_block_kernel<128, true>, a));
-        } else {
-            PA_CUDA_OK(cudaFuncSetAttribute(decode_block_kernel<64, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-            PA_CUDA_OK(cudaLaunchKernelEx(&ccfg, decode_block_kernel<64, true>, a));
-        }
-        return PA_OK;
-    }
     const dim3 grid1((unsigned)a.chunks, (unsigned)a.Hkv, (unsigned)a.batch);
     if (p->head_dim == 128)
-        decode_block_kernel<128, false><<<grid1, kDecThreads, 0, st>>>(a);
+        decode_block_kernel<128><<<grid1, kDecThreads, 0, st>>>(a);
     else
-        decode_block_kernel<64, false><<<grid1, kDecThreads, 0, st>>>(a);
+        decode_block_kernel<64><<<grid1, kDecThreads, 0, st>>>(a);
     PA_CUDA_OK(cudaGetLastError());
 
     cudaLaunchConfig_t cfg = {};
