@@ -58,7 +58,7 @@ def test_active_block_counts_of_the_workloads(pa):
     assert pa.pa_layout_size(2048, 64, 1, 1) == (32, 187)
 
 
-def test_argument_validation_happens_before_any_launch(pa):
+def test_argument_validation_happens_before_any_launch(pa, oracle):
     """These calls must fail on the host (no GPU is present in the CPU test run)."""
     with pytest.raises(pa.PaError, match="PA_ERR_INVALID_ARG"):
         pa.pa_layout_size(0, 64, 5, 1)
@@ -94,7 +94,11 @@ def test_argument_validation_happens_before_any_launch(pa):
     assert prefill_status(good, ws_bytes=8) == "PA_ERR_WORKSPACE"
 
     dgood = pa.pa_decode_params(2, 4, 2, 128, 64, 5, 1, 4096, 0.0, s, s, pa.PA_BF16)
-    assert pa.pa_decode_workspace_bytes(dgood) == 2 * 4 * (5 + 1 + 6) * 130 * 4
+    # one (o[128], m, l) slot per query head and chunk; chunks = the longest block list of any row
+    rp_ref, _ = oracle.block_layout(4096, 64, 5, 1)
+    chunks = pa.pa_decode_workspace_bytes(dgood) // (2 * 4 * 130 * 4)
+    assert pa.pa_decode_workspace_bytes(dgood) == 2 * 4 * chunks * 130 * 4
+    assert chunks == int(np.diff(rp_ref).max()) == 9
     dbad = pa.pa_decode_params.from_buffer_copy(dgood); dbad.n_q_heads = 40
     assert pa.pa_decode_workspace_bytes(dbad) == 0
     st = pa.lib.pa_decode(ctypes.byref(dbad), p, p, p, p, p, p, p, 10**6, null)
