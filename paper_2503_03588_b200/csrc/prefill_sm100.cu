@@ -339,11 +339,16 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             // with that block.
             const bool last_is_diag = w.n > 0 && lastcol == w.i;
             float m = -INFINITY, l = 0.f;
-            // One step on the logits in `sr`; meanwhile the next step's logits are fetched into
-            // `sn` (S is double-buffered, so they are normally complete by the time this step's
-            // exponentials are done) and waited for only after P has been handed over.
-            auto step = [&](uint32_t (&sr)[64], uint32_t (&sn)[64], int t) -> bool {
+            for (int t = 0; t < w.n; ++t, ++kc) {
                 const uint32_t t_s = t_s0 + (kc & 1) * 64;
+                ok = wait_bar(bar(BAR_S_FULL + 2 * s + (kc & 1)), (kc >> 1) & 1, abort_flag, a.status, 9);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                uint32_t sr[64];
+                ptx::tmem_ld32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+                ptx::tmem_ld32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+                ptx::tmem_wait_ld();
                 if (last_is_diag && t == w.n - 1) {
 #pragma unroll
                     for (int c = 0; c < 64; ++c)
@@ -408,7 +413,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         // after the P V of step kc - 2, so a barrier is never more than one phase behind.)
                         ok = wait_bar(bar(BAR_O_DONE + 2 * s + ((kc - 1) & 1)), ((kc - 1) >> 1) & 1, abort_flag, a.status, 11);
                         ok = __all_sync(0xffffffffu, ok);
-                        if (!ok) return false;
+                        if (!ok) break;
                         ptx::tc_fence_after_sync();
 #pragma unroll 1
                         for (int ch = 0; ch < D / 32; ++ch) {
@@ -436,16 +441,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 }
                 l += sum;
                 // P (bf16 pairs) overlays the first 32 columns of the S buffer just read.
-                if (t + 1 < w.n) {
-                    const uint32_t k1 = kc + 1;
-                    ok = wait_bar(bar(BAR_S_FULL + 2 * s + (k1 & 1)), (k1 >> 1) & 1, abort_flag, a.status, 9);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) return false;
-                    ptx::tc_fence_after_sync();
-                    ptx::tmem_ld32(t_s0 + (k1 & 1) * 64, *reinterpret_cast<uint32_t(*)[32]>(&sn[0]));
-                    ptx::tmem_ld32(t_s0 + (k1 & 1) * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sn[32]));
-                }
-                // P (bf16 pairs) overlays the first 32 columns of the S buffer just read.
                 ptx::tmem_st32(t_s, pk);
                 if (kc > 0) {
                     // Do not run two P hand-overs ahead of the issuer: its parity wait on this slot's
@@ -453,29 +448,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     // step's P V has completed (normally long ago) the issuer has consumed that phase.
                     ok = wait_bar(bar(BAR_O_DONE + 2 * s + ((kc - 1) & 1)), ((kc - 1) >> 1) & 1, abort_flag, a.status, 12);
                     ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) return false;
+                    if (!ok) break;
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(bar(BAR_P_FULL + s));
-                if (t + 1 < w.n) ptx::tmem_wait_ld_into(sn);
-                ++kc;
-                return true;
-            };
-            if (w.n > 0) {
-                uint32_t sa[64], sb[64];
-                ok = wait_bar(bar(BAR_S_FULL + 2 * s + (kc & 1)), (kc >> 1) & 1, abort_flag, a.status, 9);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                ptx::tc_fence_after_sync();
-                ptx::tmem_ld32(t_s0 + (kc & 1) * 64, *reinterpret_cast<uint32_t(*)[32]>(&sa[0]));
-                ptx::tmem_ld32(t_s0 + (kc & 1) * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sa[32]));
-                ptx::tmem_wait_ld_into(sa);
-                for (int t = 0; t < w.n && ok; t += 2) {
-                    ok = step(sa, sb, t);
-                    if (ok && t + 1 < w.n) ok = step(sb, sa, t + 1);
-                }
             }
             if (!ok) break;
             if (w.n <= 0) {  // empty row: defined outputs, no barrier traffic
