@@ -394,6 +394,78 @@ def run_case(args):
     print(json.dumps(dict(case=args.case, launches=args.steps + 1)))
 
 
+def causal_csr(nqb: int):
+    """Dense causal block layout: row i lists blocks 0..i."""
+    lens = np.arange(1, nqb + 1, dtype=np.int64)
+    row_ptr = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    col_idx = np.concatenate([np.arange(n, dtype=np.int32) for n in lens])
+    return row_ptr, col_idx
+
+
+def row_matched_window_csr(row_ptr_pa: np.ndarray):
+    """Sliding window with the same number of blocks per row as the given layout: block 0 (sink)
+    plus the most recent blocks, so both layouts have identical active-block counts."""
+    nqb = len(row_ptr_pa) - 1
+    cols = []
+    for i in range(nqb):
+        cnt = int(row_ptr_pa[i + 1] - row_ptr_pa[i])
+        recent = np.arange(i - (cnt - 1) + 1, i + 1, dtype=np.int32) if cnt > 1 else np.zeros(0, np.int32)
+        row = np.concatenate([[0], recent]).astype(np.int32) if cnt > 1 else np.array([i], np.int32)
+        row = np.unique(np.clip(row, 0, i))
+        while len(row) < cnt:  # early rows where the sink falls inside the window
+            row = np.unique(np.concatenate([row, [max(0, int(row[1] if len(row) > 1 else row[0]) - 1)]])).astype(np.int32)
+            if len(row) == i + 1:
+                break
+        cols.append(row.astype(np.int32))
+    rp = np.concatenate([[0], np.cumsum([len(c) for c in cols])]).astype(np.int32)
+    return rp, np.concatenate(cols)
+
+
+def run_sweep(args):
+    """Sequence-length sweep of the prefill kernel: the PowerAttention layout, dense causal and a
+    row-matched sliding window (same active-block count) through the same pa_prefill call.
+    Prints one JSON object per (length, layout)."""
+    import paper_2503_03588_b200 as pa
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks = read_peaks()
+    for N in si.SWEEP_SEQ_LENS:
+        if N > args.sweep_max_len:
+            continue
+        w = si.sweep_workload(N)
+        Q, K, V = (t.to(dev) for t in si.prefill_inputs(w))
+        rp_pa, ci_pa = pa.pa_build_layout(N, w.block, w.window_blocks, w.sink_blocks)
+        rp_host = rp_pa.cpu().numpy()
+        nqb = len(rp_host) - 1
+        layouts = {"powerattention": (rp_pa, ci_pa)}
+        rw, cw = row_matched_window_csr(rp_host)
+        layouts["sliding_window_row_matched"] = (torch.as_tensor(rw).to(dev), torch.as_tensor(cw).to(dev))
+        if N <= args.sweep_dense_max_len:
+            rc, cc = causal_csr(nqb)
+            layouts["dense_causal"] = (torch.as_tensor(rc).to(dev), torch.as_tensor(cc).to(dev))
+        o = lse = ws = None
+        for name, (rp, ci) in layouts.items():
+            nnz = int(ci.numel())
+            o, lse, ws = pa.pa_prefill(Q, K, V, rp, ci, o=o, lse=lse, workspace=ws)
+            reps = 3 if name == "dense_causal" else 10
+            for _ in range(2):
+                pa.pa_prefill(Q, K, V, rp, ci, o=o, lse=lse, workspace=ws)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                pa.pa_prefill(Q, K, V, rp, ci, o=o, lse=lse, workspace=ws)
+            e1.record()
+            torch.cuda.synchronize()
+            pa.pa_prefill_status(ws)
+            ms = e0.elapsed_time(e1) / reps
+            tf = block_pair_flops(nnz, w) / (ms * 1e-3) / 1e12
+            print(json.dumps(dict(sweep=True, seq_len=N, layout=name, active_block_pairs=nnz, ms=ms, tflops=tf,
+                                  frac_of_bf16_peak=tf / peaks["bf16_tflops"], peak_source=peaks["source"])), flush=True)
+        del Q, K, V, o, lse
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -403,7 +475,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--case", default=None, choices=["prefill32k", "decode"],
                     help="run only a small single-kernel case (for profiler captures)")
+    ap.add_argument("--sweep", action="store_true", help="sequence-length sweep with comparison layouts")
+    ap.add_argument("--sweep-max-len", type=int, default=262144)
+    ap.add_argument("--sweep-dense-max-len", type=int, default=131072)
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.case:
         run_case(args)
         return
