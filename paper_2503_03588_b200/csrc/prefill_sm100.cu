@@ -484,7 +484,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         // O / l and LSE = ln sum exp(s) = (m + log2 l) ln 2 for both slots, off the softmax warps'
         // critical path: O is read out of tensor memory (which frees it for the next unit), then
         // written to global memory from registers.
-        ptx::setmaxnreg_inc<120>();
+        ptx::setmaxnreg_dec<120>();
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const int qrow = row & 63;
