@@ -14,6 +14,7 @@
 //   warps 4-7   online softmax of slot 0 (thread = tile row = TMEM lane)
 //   warps 8-11  online softmax of slot 1
 //   warps 12-15 epilogue: O / l and LSE out of tensor memory to global memory
+// Warps 0-3 and 12-15 give registers back (setmaxnreg) and the softmax warpgroups take them.
 // Every barrier wait is bounded; a wait that runs out records PA_ERR_TIMEOUT in the status
 // block, raises a CTA-wide abort flag and the CTA drains and exits (no trap, no endless spin).
 #include <cuda.h>
@@ -163,6 +164,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
+    if (warp < 4) ptx::setmaxnreg_dec<40>();
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -317,8 +319,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
         }
         __syncwarp();
-    } else if (warp < 12) {
+    } else if (warp >= 4 && warp < 12) {
         // ------------------------------------------------------------------ online softmax
+        ptx::setmaxnreg_inc<176>();  // 4 x 40 + 8 x 176 + 4 x 120 = 16 x 128, the CTA's registers
         const int s = (warp - 4) >> 2;          // slot
         const int quad = warp & 3;              // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;       // tile row = TMEM lane
@@ -481,6 +484,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         // O / l and LSE = ln sum exp(s) = (m + log2 l) ln 2 for both slots, off the softmax warps'
         // critical path: O is read out of tensor memory (which frees it for the next unit), then
         // written to global memory from registers.
+        ptx::setmaxnreg_dec<120>();
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const int qrow = row & 63;
