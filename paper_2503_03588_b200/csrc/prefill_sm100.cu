@@ -7,7 +7,8 @@
 // and the K/V tiles).  The key list is walked one 64-key block per step.  Warp roles:
 //   warp 0      TMA producer: Q tiles once per unit, then the listed K and V blocks, gathered by
 //               block index, into two rings of shared-memory tiles (128-byte swizzle)
-//   warp 1      tcgen05 issuer: S = Q K^T into tensor memory (two S buffers per slot, so the
+//   warp 1      tcgen05 issuer, serving the two slots independently as their inputs become
+//               ready: S = Q K^T into tensor memory (two S buffers per slot, so the
 //               logits of step t+1 are ready while the softmax works on step t); O += P V with
 //               P read from tensor memory (it overlays the S buffer it was computed from)
 //   warp 2      tensor-memory allocation
@@ -132,14 +133,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
     if (threadIdx.x == 0) {
         ptx::mbar_init(bar(BAR_Q_FULL), 1);
-        ptx::mbar_init(bar(BAR_Q_EMPTY), 1);
+        ptx::mbar_init(bar(BAR_Q_EMPTY), 2);  // one commit per slot
         for (int s = 0; s < kKStages; ++s) {
             ptx::mbar_init(bar(BAR_K_FULL + s), 1);
-            ptx::mbar_init(bar(BAR_K_EMPTY + s), 1);
+            ptx::mbar_init(bar(BAR_K_EMPTY + s), 2);
         }
         for (int s = 0; s < kVStages; ++s) {
             ptx::mbar_init(bar(BAR_V_FULL + s), 1);
-            ptx::mbar_init(bar(BAR_V_EMPTY + s), 1);
+            ptx::mbar_init(bar(BAR_V_EMPTY + s), 2);
         }
         for (int s = 0; s < 4; ++s) {
             ptx::mbar_init(bar(BAR_S_FULL + s), 1);
@@ -252,70 +253,108 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     ptx::umma_ts_lohi(dst, pa_ + kk * 8, vb + ((kk * 2048) >> 4), desc_hi, idesc_pv,
                                       (acc || kk > 0) ? 1u : 0u);
             };
-            uint32_t kc = 0, ul = 0;
-            bool ok = true;
-            for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
-                const Unit w = decode_unit(a, u);
-                if (w.n <= 0) continue;
-                ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 4));
-                if (!ok) break;
-                // Prologue: S of the first two steps.
-                for (int t0 = 0; t0 < 2 && t0 < w.n && ok; ++t0) {
-                    const uint32_t c0 = kc + t0;
-                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + c0 % kKStages), (c0 / kKStages) & 1,
-                                                          abort_flag, a.status, 5));
-                    if (!ok) break;
-                    ptx::tc_fence_after_sync();
-                    if (leader) {
-                        for (int s = 0; s < 2; ++s) {
-                            issue_qk(s, c0 & 1, c0 % kKStages);
-                            ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c0 & 1)));
-                        }
-                        ptx::umma_commit(bar(BAR_K_EMPTY + c0 % kKStages));
+            // The two slots advance independently: each has its own cursor over (unit, step), and
+            // the issuer serves whichever slot has its inputs ready (non-blocking barrier tests), so
+            // a slot whose softmax is late never holds up the other.  A slot's sequence per unit is
+            // S(0), S(1), then for every step t: O += P(t) V(t), S(t + 2).  Shared stages (Q, K, V)
+            // are released by a commit from each slot (their "empty" barriers count two arrivals).
+            struct Cursor {
+                uint32_t u, kc, ul;  // unit index; key blocks and units completed before this unit
+                Unit w;
+                int t;               // next step whose P V is to be issued
+                bool prologue_done, finished;
+            };
+            Cursor cur[2];
+            auto load_unit = [&](Cursor &c) {
+                c.finished = true;
+                while (c.u < (uint32_t)a.n_units) {
+                    c.w = decode_unit(a, c.u);
+                    if (c.w.n > 0) {
+                        c.finished = false;
+                        break;
                     }
-                    __syncwarp();
+                    c.u += gridDim.x;
                 }
-                if (!ok) break;
-                if (w.n <= 2 && leader) ptx::umma_commit(bar(BAR_Q_EMPTY));
-                for (int t = 0; t < w.n && ok; ++t) {
-                    const uint32_t c = kc + t;
-                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_V_FULL + c % kVStages), (c / kVStages) & 1,
-                                                          abort_flag, a.status, 6));
-                    if (!ok) break;
-                    if (t + 2 < w.n) {
-                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + (c + 2) % kKStages),
-                                                              ((c + 2) / kKStages) & 1, abort_flag, a.status, 8));
-                        if (!ok) break;
-                    }
-                    for (int s = 0; s < 2; ++s) {
-                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + s), c & 1, abort_flag, a.status, 7));
-                        if (!ok) break;
+                c.t = 0;
+                c.prologue_done = false;
+            };
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+                cur[s].u = blockIdx.x;
+                cur[s].kc = 0;
+                cur[s].ul = 0;
+                load_unit(cur[s]);
+            }
+            long long t_last = clock64();
+            bool ok = true;
+            while (ok && !(cur[0].finished && cur[1].finished)) {
+                bool progressed = false;
+#pragma unroll
+                for (int s = 0; s < 2; ++s) {
+                    Cursor &c = cur[s];
+                    if (c.finished) continue;
+                    const int n = c.w.n;
+                    if (!c.prologue_done) {
+                        bool r = ptx::mbar_test_wait(bar(BAR_Q_FULL), c.ul & 1) &&
+                                 ptx::mbar_test_wait(bar(BAR_K_FULL + c.kc % kKStages), (c.kc / kKStages) & 1);
+                        if (n >= 2)
+                            r = r && ptx::mbar_test_wait(bar(BAR_K_FULL + (c.kc + 1) % kKStages), ((c.kc + 1) / kKStages) & 1);
+                        if (!__all_sync(0xffffffffu, r)) continue;
                         ptx::tc_fence_after_sync();
-                        if (t == 0 && ul > 0) {
-                            // The previous unit's O must have left tensor memory.
-                            ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_O_FREE + s), (ul - 1) & 1, abort_flag, a.status, 14));
-                            if (!ok) break;
-                            ptx::tc_fence_after_sync();
-                        }
                         if (leader) {
-                            issue_pv(s, c & 1, c % kVStages, t > 0);
-                            ptx::umma_commit(bar(BAR_O_DONE + 2 * s + (c & 1)));
-                            if (t + 1 == w.n) ptx::umma_commit(bar(BAR_O_FINAL + s));
-                            if (s == 1) ptx::umma_commit(bar(BAR_V_EMPTY + c % kVStages));
-                            if (t + 2 < w.n) {
-                                issue_qk(s, c & 1, (c + 2) % kKStages);
-                                ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c & 1)));
-                                if (s == 1) {
-                                    ptx::umma_commit(bar(BAR_K_EMPTY + (c + 2) % kKStages));
-                                    if (t + 3 == w.n) ptx::umma_commit(bar(BAR_Q_EMPTY));
-                                }
+                            for (int t0 = 0; t0 < 2 && t0 < n; ++t0) {
+                                const uint32_t c0 = c.kc + t0;
+                                issue_qk(s, c0 & 1, c0 % kKStages);
+                                ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c0 & 1)));
+                                ptx::umma_commit(bar(BAR_K_EMPTY + c0 % kKStages));
                             }
+                            if (n <= 2) ptx::umma_commit(bar(BAR_Q_EMPTY));
                         }
                         __syncwarp();
+                        c.prologue_done = true;
+                        progressed = true;
+                        continue;
+                    }
+                    const uint32_t cc = c.kc + c.t;
+                    bool r = ptx::mbar_test_wait(bar(BAR_P_FULL + s), cc & 1) &&
+                             ptx::mbar_test_wait(bar(BAR_V_FULL + cc % kVStages), (cc / kVStages) & 1);
+                    if (c.t + 2 < n)
+                        r = r && ptx::mbar_test_wait(bar(BAR_K_FULL + (cc + 2) % kKStages), ((cc + 2) / kKStages) & 1);
+                    if (c.t == 0 && c.ul > 0)  // the previous unit's O must have left tensor memory
+                        r = r && ptx::mbar_test_wait(bar(BAR_O_FREE + s), (c.ul - 1) & 1);
+                    if (!__all_sync(0xffffffffu, r)) continue;
+                    ptx::tc_fence_after_sync();
+                    if (leader) {
+                        issue_pv(s, cc & 1, cc % kVStages, c.t > 0);
+                        ptx::umma_commit(bar(BAR_O_DONE + 2 * s + (cc & 1)));
+                        if (c.t + 1 == n) ptx::umma_commit(bar(BAR_O_FINAL + s));
+                        ptx::umma_commit(bar(BAR_V_EMPTY + cc % kVStages));
+                        if (c.t + 2 < n) {
+                            issue_qk(s, cc & 1, (cc + 2) % kKStages);
+                            ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (cc & 1)));
+                            ptx::umma_commit(bar(BAR_K_EMPTY + (cc + 2) % kKStages));
+                            if (c.t + 3 == n) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                        }
+                    }
+                    __syncwarp();
+                    progressed = true;
+                    if (++c.t == n) {
+                        c.kc += n;
+                        ++c.ul;
+                        c.u += gridDim.x;
+                        load_unit(c);
                     }
                 }
-                kc += w.n;
-                ++ul;
+                if (progressed) {
+                    t_last = clock64();
+                } else if (*abort_flag) {
+                    ok = false;
+                } else if (clock64() - t_last > kWaitCycles) {
+                    if (atomicCAS(a.status, 0, (int)PA_ERR_TIMEOUT) == 0) a.status[1] = 4;
+                    *abort_flag = 1;
+                    __threadfence_block();
+                    ok = false;
+                }
             }
         }
         __syncwarp();
