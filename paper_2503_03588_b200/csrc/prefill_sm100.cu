@@ -350,7 +350,32 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 } else if (*abort_flag) {
                     ok = false;
                 } else if (clock64() - t_last > kWaitCycles) {
-                    if (atomicCAS(a.status, 0, (int)PA_ERR_TIMEOUT) == 0) a.status[1] = 4;
+                    if (atomicCAS(a.status, 0, (int)PA_ERR_TIMEOUT) == 0) {
+                        a.status[1] = 4;
+                        // Where each slot stood: words 2.. = block, then per slot (unit, step, row length,
+                        // units done, prologue done, readiness bits P/V/K/Ofree or Q/K0/K1).
+                        if (leader) {
+                            a.status[2] = (int)blockIdx.x;
+                            for (int s = 0; s < 2; ++s) {
+                                const Cursor &c = cur[s];
+                                int32_t *d = a.status + 4 + 8 * s;
+                                d[0] = (int)c.u; d[1] = c.t; d[2] = c.w.n; d[3] = (int)c.ul; d[4] = c.prologue_done; d[5] = c.finished;
+                                const uint32_t cc = c.kc + c.t;
+                                int bits = 0;
+                                if (!c.prologue_done) {
+                                    bits |= ptx::mbar_test_wait(bar(BAR_Q_FULL), c.ul & 1) ? 1 : 0;
+                                    bits |= ptx::mbar_test_wait(bar(BAR_K_FULL + c.kc % kKStages), (c.kc / kKStages) & 1) ? 2 : 0;
+                                    bits |= ptx::mbar_test_wait(bar(BAR_K_FULL + (c.kc + 1) % kKStages), ((c.kc + 1) / kKStages) & 1) ? 4 : 0;
+                                } else {
+                                    bits |= ptx::mbar_test_wait(bar(BAR_P_FULL + s), cc & 1) ? 1 : 0;
+                                    bits |= ptx::mbar_test_wait(bar(BAR_V_FULL + cc % kVStages), (cc / kVStages) & 1) ? 2 : 0;
+                                    bits |= ptx::mbar_test_wait(bar(BAR_K_FULL + (cc + 2) % kKStages), ((cc + 2) / kKStages) & 1) ? 4 : 0;
+                                    bits |= (c.ul == 0 || ptx::mbar_test_wait(bar(BAR_O_FREE + s), (c.ul - 1) & 1)) ? 8 : 0;
+                                }
+                                d[6] = bits; d[7] = (int)c.kc;
+                            }
+                        }
+                    }
                     *abort_flag = 1;
                     __threadfence_block();
                     ok = false;
