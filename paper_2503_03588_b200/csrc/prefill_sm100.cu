@@ -394,7 +394,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const uint32_t t_o = tmem_base + ((uint32_t)(quad * 32) << 16) + 256 + s * D;
         const float sl2 = a.scale_log2;
         const uint64_t sl2_2 = ptx::pack_f32x2(sl2, sl2);
-        uint32_t kc = 0;
+        uint32_t kc = 0, units_done = 0;
         bool ok = true;
         Unit w_next = {};
         int32_t lastcol_next = -1;
@@ -532,7 +532,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 if (t + 1 == w.n) {
-                    // Row statistics for the epilogue warps (they finish O / l and the LSE).
+                    // Row statistics for the epilogue warps (they finish O / l and the LSE).  The
+                    // epilogue must be done with the previous unit's statistics first (already the
+                    // case unless this unit has a single step).
+                    if (units_done > 0) {
+                        ok = wait_bar(bar(BAR_O_FREE + s), (units_done - 1) & 1, abort_flag, a.status, 16);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                    }
                     reinterpret_cast<float2 *>(smem + SM::kStats)[s * 128 + row] = make_float2(m, l);
                     __threadfence_block();
                 }
@@ -542,6 +549,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     if (t + 1 == w.n) ptx::mbar_arrive(bar(BAR_ML_READY + s));
                 }
             }
+            if (w.n > 0) ++units_done;
         }
     } else if (warp >= 12) {
         // ------------------------------------------------------------------ epilogue
