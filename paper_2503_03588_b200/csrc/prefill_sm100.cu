@@ -7,15 +7,13 @@
 // and the K/V tiles).  The key list is walked one 64-key block per step.  Warp roles:
 //   warp 0      TMA producer: Q tiles once per unit, then the listed K and V blocks, gathered by
 //               block index, into two rings of shared-memory tiles (128-byte swizzle)
-//   warp 1      tcgen05 issuer, serving the two slots independently as their inputs become
-//               ready: S = Q K^T into tensor memory (two S buffers per slot, so the
+//   warp 1      tcgen05 issuer: S = Q K^T into tensor memory (two S buffers per slot, so the
 //               logits of step t+1 are ready while the softmax works on step t); O += P V with
 //               P read from tensor memory (it overlays the S buffer it was computed from)
 //   warp 2      tensor-memory allocation
 //   warps 4-7   online softmax of slot 0 (thread = tile row = TMEM lane)
 //   warps 8-11  online softmax of slot 1
-//   warps 12-15 epilogue: O / l and LSE out of tensor memory to global memory
-// Warps 0-3 and 12-15 give registers back (setmaxnreg) and the softmax warpgroups take them.
+// Warps 0-3 give registers back (setmaxnreg) and the softmax warpgroups take them.
 // Every barrier wait is bounded; a wait that runs out records PA_ERR_TIMEOUT in the status
 // block, raises a CTA-wide abort flag and the CTA drains and exits (no trap, no endless spin).
 #include <cuda.h>
@@ -28,9 +26,9 @@
 namespace pa {
 
 constexpr int kBlk = 64;               // tokens per query / key block
-constexpr int kThreads = 512;          // 16 warps: control, two softmax warpgroups, epilogue
+constexpr int kThreads = 384;          // 12 warps: one control warpgroup, two softmax warpgroups
 constexpr int kKStages = 5;            // K block ring depth
-constexpr int kVStages = 4;            // V block ring depth
+constexpr int kVStages = 5;            // V block ring depth
 constexpr uint32_t kTmemCols = 512;    // slot s: S/P buffers at columns 128 s + 64 b, O at 256 + s D
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logits: rescale O only when the row max grows by more
 constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
@@ -55,8 +53,7 @@ struct SmemMap {
     static constexpr uint32_t kBlkTile = kBlkSub * (D / 64);  // one K or V block
     static constexpr uint32_t kK = kQ + 2 * kQSlot;
     static constexpr uint32_t kV = kK + kKStages * kBlkTile;
-    static constexpr uint32_t kStats = kV + kVStages * kBlkTile;  // [slot][row] (m, l) for the epilogue
-    static constexpr uint32_t kBars = kStats + 2 * 128 * 8;
+    static constexpr uint32_t kBars = kV + kVStages * kBlkTile;
     static constexpr uint32_t kTotal = kBars + 512;
     static constexpr uint32_t kAlloc = kTotal + 1024;         // slack for 1024-byte alignment
 };
@@ -68,10 +65,7 @@ enum : uint32_t {
     BAR_S_FULL = BAR_V_EMPTY + kVStages,  // [slot][buffer]
     BAR_P_FULL = BAR_S_FULL + 4,
     BAR_O_DONE = BAR_P_FULL + 2,  // [slot][step parity]: P V of that step has completed
-    BAR_O_FINAL = BAR_O_DONE + 4,   // [slot]: the unit's last P V has completed
-    BAR_ML_READY = BAR_O_FINAL + 2,  // [slot]: the unit's row statistics are in shared memory
-    BAR_O_FREE = BAR_ML_READY + 2,   // [slot]: the epilogue has read O out of tensor memory
-    BAR_COUNT = BAR_O_FREE + 2
+    BAR_COUNT = BAR_O_DONE + 4
 };
 
 struct Unit {
@@ -133,14 +127,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
     if (threadIdx.x == 0) {
         ptx::mbar_init(bar(BAR_Q_FULL), 1);
-        ptx::mbar_init(bar(BAR_Q_EMPTY), 2);  // one commit per slot
+        ptx::mbar_init(bar(BAR_Q_EMPTY), 1);
         for (int s = 0; s < kKStages; ++s) {
             ptx::mbar_init(bar(BAR_K_FULL + s), 1);
-            ptx::mbar_init(bar(BAR_K_EMPTY + s), 2);
+            ptx::mbar_init(bar(BAR_K_EMPTY + s), 1);
         }
         for (int s = 0; s < kVStages; ++s) {
             ptx::mbar_init(bar(BAR_V_FULL + s), 1);
-            ptx::mbar_init(bar(BAR_V_EMPTY + s), 2);
+            ptx::mbar_init(bar(BAR_V_EMPTY + s), 1);
         }
         for (int s = 0; s < 4; ++s) {
             ptx::mbar_init(bar(BAR_S_FULL + s), 1);
@@ -148,9 +142,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(bar(BAR_P_FULL + s), 4);  // one arrival per softmax warp of the slot
-            ptx::mbar_init(bar(BAR_O_FINAL + s), 1);
-            ptx::mbar_init(bar(BAR_ML_READY + s), 4);
-            ptx::mbar_init(bar(BAR_O_FREE + s), 4);
         }
         *abort_flag = 0;
         ptx::fence_barrier_init();
@@ -253,139 +244,69 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     ptx::umma_ts_lohi(dst, pa_ + kk * 8, vb + ((kk * 2048) >> 4), desc_hi, idesc_pv,
                                       (acc || kk > 0) ? 1u : 0u);
             };
-            // The two slots advance independently: each has its own cursor over (unit, step), and
-            // the issuer serves whichever slot has its inputs ready (non-blocking barrier tests), so
-            // a slot whose softmax is late never holds up the other.  A slot's sequence per unit is
-            // S(0), S(1), then for every step t: O += P(t) V(t), S(t + 2).  Shared stages (Q, K, V)
-            // are released by a commit from each slot (their "empty" barriers count two arrivals).
-            struct Cursor {
-                uint32_t u, kc, ul;  // unit index; key blocks and units completed before this unit
-                Unit w;
-                int t;               // next step whose P V is to be issued
-                bool prologue_done, finished;
-            };
-            Cursor cur[2];
-            auto load_unit = [&](Cursor &c) {
-                c.finished = true;
-                while (c.u < (uint32_t)a.n_units) {
-                    c.w = decode_unit(a, c.u);
-                    if (c.w.n > 0) {
-                        c.finished = false;
-                        break;
-                    }
-                    c.u += gridDim.x;
-                }
-                c.t = 0;
-                c.prologue_done = false;
-            };
-#pragma unroll
-            for (int s = 0; s < 2; ++s) {
-                cur[s].u = blockIdx.x;
-                cur[s].kc = 0;
-                cur[s].ul = 0;
-                load_unit(cur[s]);
-            }
-            long long t_last = clock64();
+            uint32_t kc = 0, ul = 0;
             bool ok = true;
-            while (ok && !(cur[0].finished && cur[1].finished)) {
-                bool progressed = false;
-#pragma unroll
-                for (int s = 0; s < 2; ++s) {
-                    Cursor &c = cur[s];
-                    if (c.finished) continue;
-                    const int n = c.w.n;
-                    if (!c.prologue_done) {
-                        bool r = ptx::mbar_test_wait(bar(BAR_Q_FULL), c.ul & 1) &&
-                                 ptx::mbar_test_wait(bar(BAR_K_FULL + c.kc % kKStages), (c.kc / kKStages) & 1);
-                        if (n >= 2)
-                            r = r && ptx::mbar_test_wait(bar(BAR_K_FULL + (c.kc + 1) % kKStages), ((c.kc + 1) / kKStages) & 1);
-                        if (!__all_sync(0xffffffffu, r)) continue;
-                        ptx::tc_fence_after_sync();
-                        if (leader) {
-                            for (int t0 = 0; t0 < 2 && t0 < n; ++t0) {
-                                const uint32_t c0 = c.kc + t0;
-                                issue_qk(s, c0 & 1, c0 % kKStages);
-                                ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c0 & 1)));
-                                ptx::umma_commit(bar(BAR_K_EMPTY + c0 % kKStages));
-                            }
-                            if (n <= 2) ptx::umma_commit(bar(BAR_Q_EMPTY));
-                        }
-                        __syncwarp();
-                        c.prologue_done = true;
-                        progressed = true;
-                        continue;
-                    }
-                    const uint32_t cc = c.kc + c.t;
-                    bool r = ptx::mbar_test_wait(bar(BAR_P_FULL + s), cc & 1) &&
-                             ptx::mbar_test_wait(bar(BAR_V_FULL + cc % kVStages), (cc / kVStages) & 1);
-                    if (c.t + 2 < n)
-                        r = r && ptx::mbar_test_wait(bar(BAR_K_FULL + (cc + 2) % kKStages), ((cc + 2) / kKStages) & 1);
-                    if (c.t == 0 && c.ul > 0)  // the previous unit's O must have left tensor memory
-                        r = r && ptx::mbar_test_wait(bar(BAR_O_FREE + s), (c.ul - 1) & 1);
-                    if (!__all_sync(0xffffffffu, r)) continue;
+            for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
+                const Unit w = decode_unit(a, u);
+                if (w.n <= 0) continue;
+                ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 4));
+                if (!ok) break;
+                // Prologue: S of the first two steps.
+                for (int t0 = 0; t0 < 2 && t0 < w.n && ok; ++t0) {
+                    const uint32_t c0 = kc + t0;
+                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + c0 % kKStages), (c0 / kKStages) & 1,
+                                                          abort_flag, a.status, 5));
+                    if (!ok) break;
                     ptx::tc_fence_after_sync();
                     if (leader) {
-                        issue_pv(s, cc & 1, cc % kVStages, c.t > 0);
-                        ptx::umma_commit(bar(BAR_O_DONE + 2 * s + (cc & 1)));
-                        if (c.t + 1 == n) ptx::umma_commit(bar(BAR_O_FINAL + s));
-                        ptx::umma_commit(bar(BAR_V_EMPTY + cc % kVStages));
-                        if (c.t + 2 < n) {
-                            issue_qk(s, cc & 1, (cc + 2) % kKStages);
-                            ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (cc & 1)));
-                            ptx::umma_commit(bar(BAR_K_EMPTY + (cc + 2) % kKStages));
-                            if (c.t + 3 == n) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                        for (int s = 0; s < 2; ++s) {
+                            issue_qk(s, c0 & 1, c0 % kKStages);
+                            ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c0 & 1)));
                         }
+                        ptx::umma_commit(bar(BAR_K_EMPTY + c0 % kKStages));
                     }
                     __syncwarp();
-                    progressed = true;
-                    if (++c.t == n) {
-                        c.kc += n;
-                        ++c.ul;
-                        c.u += gridDim.x;
-                        load_unit(c);
-                    }
                 }
-                if (progressed) {
-                    t_last = clock64();
-                } else if (*abort_flag) {
-                    ok = false;
-                } else if (clock64() - t_last > kWaitCycles) {
-                    if (atomicCAS(a.status, 0, (int)PA_ERR_TIMEOUT) == 0) {
-                        a.status[1] = 4;
-                        // Where each slot stood: words 2.. = block, then per slot (unit, step, row length,
-                        // units done, prologue done, readiness bits P/V/K/Ofree or Q/K0/K1).
+                if (!ok) break;
+                if (w.n <= 2 && leader) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                for (int t = 0; t < w.n && ok; ++t) {
+                    const uint32_t c = kc + t;
+                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_V_FULL + c % kVStages), (c / kVStages) & 1,
+                                                          abort_flag, a.status, 6));
+                    if (!ok) break;
+                    if (t + 2 < w.n) {
+                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + (c + 2) % kKStages),
+                                                              ((c + 2) / kKStages) & 1, abort_flag, a.status, 8));
+                        if (!ok) break;
+                    }
+                    for (int s = 0; s < 2; ++s) {
+                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + s), c & 1, abort_flag, a.status, 7));
+                        if (!ok) break;
+                        ptx::tc_fence_after_sync();
                         if (leader) {
-                            a.status[2] = (int)blockIdx.x;
-                            for (int s = 0; s < 2; ++s) {
-                                const Cursor &c = cur[s];
-                                int32_t *d = a.status + 4 + 8 * s;
-                                d[0] = (int)c.u; d[1] = c.t; d[2] = c.w.n; d[3] = (int)c.ul; d[4] = c.prologue_done; d[5] = c.finished;
-                                const uint32_t cc = c.kc + c.t;
-                                int bits = 0;
-                                if (!c.prologue_done) {
-                                    bits |= ptx::mbar_test_wait(bar(BAR_Q_FULL), c.ul & 1) ? 1 : 0;
-                                    bits |= ptx::mbar_test_wait(bar(BAR_K_FULL + c.kc % kKStages), (c.kc / kKStages) & 1) ? 2 : 0;
-                                    bits |= ptx::mbar_test_wait(bar(BAR_K_FULL + (c.kc + 1) % kKStages), ((c.kc + 1) / kKStages) & 1) ? 4 : 0;
-                                } else {
-                                    bits |= ptx::mbar_test_wait(bar(BAR_P_FULL + s), cc & 1) ? 1 : 0;
-                                    bits |= ptx::mbar_test_wait(bar(BAR_V_FULL + cc % kVStages), (cc / kVStages) & 1) ? 2 : 0;
-                                    bits |= ptx::mbar_test_wait(bar(BAR_K_FULL + (cc + 2) % kKStages), ((cc + 2) / kKStages) & 1) ? 4 : 0;
-                                    bits |= (c.ul == 0 || ptx::mbar_test_wait(bar(BAR_O_FREE + s), (c.ul - 1) & 1)) ? 8 : 0;
+                            issue_pv(s, c & 1, c % kVStages, t > 0);
+                            ptx::umma_commit(bar(BAR_O_DONE + 2 * s + (c & 1)));
+                            if (s == 1) ptx::umma_commit(bar(BAR_V_EMPTY + c % kVStages));
+                            if (t + 2 < w.n) {
+                                issue_qk(s, c & 1, (c + 2) % kKStages);
+                                ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c & 1)));
+                                if (s == 1) {
+                                    ptx::umma_commit(bar(BAR_K_EMPTY + (c + 2) % kKStages));
+                                    if (t + 3 == w.n) ptx::umma_commit(bar(BAR_Q_EMPTY));
                                 }
-                                d[6] = bits; d[7] = (int)c.kc;
                             }
                         }
+                        __syncwarp();
                     }
-                    *abort_flag = 1;
-                    __threadfence_block();
-                    ok = false;
                 }
+                kc += w.n;
+                ++ul;
             }
         }
         __syncwarp();
-    } else if (warp >= 4 && warp < 12) {
+    } else if (warp >= 4) {
         // ------------------------------------------------------------------ online softmax
-        ptx::setmaxnreg_inc<176>();  // 4 x 40 + 8 x 176 + 4 x 120 = 16 x 128, the CTA's registers
+        ptx::setmaxnreg_inc<232>();
         const int s = (warp - 4) >> 2;          // slot
         const int quad = warp & 3;              // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;       // tile row = TMEM lane
@@ -394,7 +315,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const uint32_t t_o = tmem_base + ((uint32_t)(quad * 32) << 16) + 256 + s * D;
         const float sl2 = a.scale_log2;
         const uint64_t sl2_2 = ptx::pack_f32x2(sl2, sl2);
-        uint32_t kc = 0, units_done = 0;
+        uint32_t kc = 0;
         bool ok = true;
         Unit w_next = {};
         int32_t lastcol_next = -1;
@@ -531,108 +452,54 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
-                if (t + 1 == w.n) {
-                    // Row statistics for the epilogue warps (they finish O / l and the LSE).  The
-                    // epilogue must be done with the previous unit's statistics first (already the
-                    // case unless this unit has a single step).
-                    if (units_done > 0) {
-                        ok = wait_bar(bar(BAR_O_FREE + s), (units_done - 1) & 1, abort_flag, a.status, 16);
-                        ok = __all_sync(0xffffffffu, ok);
-                        if (!ok) break;
-                    }
-                    reinterpret_cast<float2 *>(smem + SM::kStats)[s * 128 + row] = make_float2(m, l);
-                    __threadfence_block();
-                }
                 __syncwarp();
-                if (lane == 0) {
-                    ptx::mbar_arrive(bar(BAR_P_FULL + s));
-                    if (t + 1 == w.n) ptx::mbar_arrive(bar(BAR_ML_READY + s));
+                if (lane == 0) ptx::mbar_arrive(bar(BAR_P_FULL + s));
+            }
+            if (!ok) break;
+            if (w.n <= 0) {  // empty row: defined outputs, no barrier traffic
+                if (valid) {
+                    for (int c = 0; c < D; ++c) {
+                        const int64_t oi = w.b * a.o_sb + tok * a.o_ss + head * a.o_sh + c;
+                        if (a.o_is_f32) reinterpret_cast<float *>(a.o)[oi] = 0.f;
+                        else reinterpret_cast<__nv_bfloat16 *>(a.o)[oi] = __float2bfloat16_rn(0.f);
+                    }
+                    a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = -INFINITY;
+                }
+                continue;
+            }
+            // Epilogue: O / l and LSE = ln sum exp(s) = (m + log2 l) ln 2.
+            ok = wait_bar(bar(BAR_O_DONE + 2 * s + ((kc - 1) & 1)), ((kc - 1) >> 1) & 1, abort_flag, a.status, 10);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            const float inv = 1.0f / l;
+            const int64_t obase = w.b * a.o_sb + tok * a.o_ss + (int64_t)head * a.o_sh;
+#pragma unroll
+            for (int ch = 0; ch < D / 32; ++ch) {
+                uint32_t orr[32];
+                ptx::tmem_ld32(t_o + ch * 32, orr);
+                ptx::tmem_wait_ld();
+                if (valid) {
+                    if (a.o_is_f32) {
+                        float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(a.o) + obase + ch * 32);
+#pragma unroll
+                        for (int c = 0; c < 8; ++c)
+                            dst[c] = make_float4(__uint_as_float(orr[4 * c]) * inv, __uint_as_float(orr[4 * c + 1]) * inv,
+                                                 __uint_as_float(orr[4 * c + 2]) * inv, __uint_as_float(orr[4 * c + 3]) * inv);
+                    } else {
+                        uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(a.o) + obase + ch * 32);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            dst[c] = make_uint4(
+                                ptx::cvt_bf16x2(__uint_as_float(orr[8 * c]) * inv, __uint_as_float(orr[8 * c + 1]) * inv),
+                                ptx::cvt_bf16x2(__uint_as_float(orr[8 * c + 2]) * inv, __uint_as_float(orr[8 * c + 3]) * inv),
+                                ptx::cvt_bf16x2(__uint_as_float(orr[8 * c + 4]) * inv, __uint_as_float(orr[8 * c + 5]) * inv),
+                                ptx::cvt_bf16x2(__uint_as_float(orr[8 * c + 6]) * inv, __uint_as_float(orr[8 * c + 7]) * inv));
+                    }
                 }
             }
-            if (w.n > 0) ++units_done;
-        }
-    } else if (warp >= 12) {
-        // ------------------------------------------------------------------ epilogue
-        // O / l and LSE = ln sum exp(s) = (m + log2 l) ln 2 for both slots, off the softmax warps'
-        // critical path: O is read out of tensor memory (which frees it for the next unit), then
-        // written to global memory from registers.
-        ptx::setmaxnreg_dec<120>();
-        const int quad = warp & 3;
-        const int row = quad * 32 + lane;
-        const int qrow = row & 63;
-        uint32_t ul = 0;
-        bool ok = true;
-        for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
-            const Unit w = decode_unit(a, u);
-            const int64_t tok = (int64_t)w.i * kBlk + qrow;
-#pragma unroll 1
-            for (int s = 0; s < 2; ++s) {
-                const int head_local = w.sub * 4 + 2 * s + (row >> 6);
-                const int head = w.hk * a.G + head_local;
-                const bool valid = head_local < a.G && tok < a.N;
-                const int64_t obase = w.b * a.o_sb + tok * a.o_ss + (int64_t)head * a.o_sh;
-                if (w.n <= 0) {  // empty row: defined outputs, no barrier traffic
-                    if (valid) {
-                        for (int c = 0; c < D; ++c) {
-                            if (a.o_is_f32) reinterpret_cast<float *>(a.o)[obase + c] = 0.f;
-                            else reinterpret_cast<__nv_bfloat16 *>(a.o)[obase + c] = __float2bfloat16_rn(0.f);
-                        }
-                        a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = -INFINITY;
-                    }
-                    continue;
-                }
-                ok = wait_bar(bar(BAR_ML_READY + s), ul & 1, abort_flag, a.status, 15);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                const float2 ml = reinterpret_cast<const float2 *>(smem + SM::kStats)[s * 128 + row];
-                ok = wait_bar(bar(BAR_O_FINAL + s), ul & 1, abort_flag, a.status, 10);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                ptx::tc_fence_after_sync();
-                const uint32_t t_o = tmem_base + ((uint32_t)(quad * 32) << 16) + 256 + s * D;
-                const float inv = 1.0f / ml.y;
-                if (a.o_is_f32) {
-#pragma unroll
-                    for (int ch = 0; ch < D / 32; ++ch) {
-                        uint32_t orr[32];
-                        ptx::tmem_ld32(t_o + ch * 32, orr);
-                        ptx::tmem_wait_ld();
-                        if (ch == D / 32 - 1) {
-                            ptx::tc_fence_before_sync();
-                            __syncwarp();
-                            if (lane == 0) ptx::mbar_arrive(bar(BAR_O_FREE + s));
-                        }
-                        if (valid) {
-                            float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(a.o) + obase + ch * 32);
-#pragma unroll
-                            for (int c = 0; c < 8; ++c)
-                                dst[c] = make_float4(__uint_as_float(orr[4 * c]) * inv, __uint_as_float(orr[4 * c + 1]) * inv,
-                                                     __uint_as_float(orr[4 * c + 2]) * inv, __uint_as_float(orr[4 * c + 3]) * inv);
-                        }
-                    }
-                } else {
-                    uint32_t pk[D / 2];
-#pragma unroll
-                    for (int ch = 0; ch < D / 32; ++ch) {
-                        uint32_t orr[32];
-                        ptx::tmem_ld32(t_o + ch * 32, orr);
-                        ptx::tmem_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 16; ++c)
-                            pk[ch * 16 + c] = ptx::cvt_bf16x2(__uint_as_float(orr[2 * c]) * inv, __uint_as_float(orr[2 * c + 1]) * inv);
-                    }
-                    ptx::tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(bar(BAR_O_FREE + s));
-                    if (valid) {
-                        uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(a.o) + obase);
-#pragma unroll
-                        for (int c = 0; c < D / 8; ++c) dst[c] = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-                    }
-                }
-                if (valid) a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = (ml.x + log2f(ml.y)) * 0.6931471805599453f;
-            }
-            if (w.n > 0) ++ul;
+            if (valid) a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = (m + log2f(l)) * 0.6931471805599453f;
+            ptx::tc_fence_before_sync();
         }
     }
 
