@@ -364,6 +364,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 uint64_t sum2[2] = {0ull, 0ull};
                 uint32_t pmax2[2] = {0u, 0u};
                 uint32_t pk[32];
+                if (t > 0) {  // the first step of a unit has no reference yet: straight to the exact path
 #pragma unroll
                 for (int c = 0; c < 64; c += 4) {
 #pragma unroll
@@ -379,6 +380,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         pk[(c >> 1) + e] = q;
                         pmax2[e] = ptx::max_bf16x2(pmax2[e], q);
                     }
+                }
                 }
                 float sum;
                 {
