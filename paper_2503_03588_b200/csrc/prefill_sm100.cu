@@ -13,7 +13,8 @@
 //   warp 2      tensor-memory allocation
 //   warps 4-7   online softmax of slot 0 (thread = tile row = TMEM lane)
 //   warps 8-11  online softmax of slot 1
-// Warps 0-3 give registers back (setmaxnreg) and the softmax warpgroups take them.
+//   warps 12-15 epilogue: O / l and LSE out of tensor memory to global memory
+// Warps 0-3 and 12-15 give registers back (setmaxnreg) and the softmax warpgroups take them.
 // Every barrier wait is bounded; a wait that runs out records PA_ERR_TIMEOUT in the status
 // block, raises a CTA-wide abort flag and the CTA drains and exits (no trap, no endless spin).
 #include <cuda.h>
@@ -26,9 +27,9 @@
 namespace pa {
 
 constexpr int kBlk = 64;               // tokens per query / key block
-constexpr int kThreads = 384;          // 12 warps: one control warpgroup, two softmax warpgroups
+constexpr int kThreads = 512;          // 16 warps: control, two softmax warpgroups, epilogue
 constexpr int kKStages = 5;            // K block ring depth
-constexpr int kVStages = 5;            // V block ring depth
+constexpr int kVStages = 4;            // V block ring depth
 constexpr uint32_t kTmemCols = 512;    // slot s: S/P buffers at columns 128 s + 64 b, O at 256 + s D
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logits: rescale O only when the row max grows by more
 constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
@@ -53,7 +54,8 @@ struct SmemMap {
     static constexpr uint32_t kBlkTile = kBlkSub * (D / 64);  // one K or V block
     static constexpr uint32_t kK = kQ + 2 * kQSlot;
     static constexpr uint32_t kV = kK + kKStages * kBlkTile;
-    static constexpr uint32_t kBars = kV + kVStages * kBlkTile;
+    static constexpr uint32_t kStats = kV + kVStages * kBlkTile;  // [slot][row] (m, l) for the epilogue
+    static constexpr uint32_t kBars = kStats + 2 * 128 * 8;
     static constexpr uint32_t kTotal = kBars + 512;
     static constexpr uint32_t kAlloc = kTotal + 1024;         // slack for 1024-byte alignment
 };
@@ -65,7 +67,10 @@ enum : uint32_t {
     BAR_S_FULL = BAR_V_EMPTY + kVStages,  // [slot][buffer]
     BAR_P_FULL = BAR_S_FULL + 4,
     BAR_O_DONE = BAR_P_FULL + 2,  // [slot][step parity]: P V of that step has completed
-    BAR_COUNT = BAR_O_DONE + 4
+    BAR_O_FINAL = BAR_O_DONE + 4,   // [slot]: the unit's last P V has completed
+    BAR_ML_READY = BAR_O_FINAL + 2,  // [slot]: the unit's row statistics are in shared memory
+    BAR_O_FREE = BAR_ML_READY + 2,   // [slot]: the epilogue has read O out of tensor memory
+    BAR_COUNT = BAR_O_FREE + 2
 };
 
 struct Unit {
@@ -142,6 +147,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(bar(BAR_P_FULL + s), 4);  // one arrival per softmax warp of the slot
+            ptx::mbar_init(bar(BAR_O_FINAL + s), 1);
+            ptx::mbar_init(bar(BAR_ML_READY + s), 4);
+            ptx::mbar_init(bar(BAR_O_FREE + s), 4);
         }
         *abort_flag = 0;
         ptx::fence_barrier_init();
@@ -244,37 +252,63 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     ptx::umma_ts_lohi(dst, pa_ + kk * 8, vb + ((kk * 2048) >> 4), desc_hi, idesc_pv,
                                       (acc || kk > 0) ? 1u : 0u);
             };
-            uint32_t kc = 0, ul = 0;
-            bool ok = true;
-            for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
-                const Unit w = decode_unit(a, u);
-                if (w.n <= 0) continue;
-                ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 4));
-                if (!ok) break;
-                // Prologue: S of the first two steps.
-                for (int t0 = 0; t0 < 2 && t0 < w.n && ok; ++t0) {
-                    const uint32_t c0 = kc + t0;
+            // First non-empty unit at or after u (stride: the grid), or n_units.
+            auto next_unit = [&](uint32_t u, int &n) {
+                for (; u < (uint32_t)a.n_units; u += gridDim.x) {
+                    n = decode_unit(a, u).n;
+                    if (n > 0) break;
+                }
+                return u;
+            };
+            // S of the first two steps of a unit, for one slot.  Steps are numbered through the
+            // CTA's whole run (kc0 = number of the unit's first step), so the buffer and ring
+            // arithmetic does not care about unit boundaries.
+            auto issue_head = [&](int s, uint32_t kc0, int n) {
+                for (int t0 = 0; t0 < 2 && t0 < n; ++t0) {
+                    const uint32_t c0 = kc0 + t0;
+                    issue_qk(s, c0 & 1, c0 % kKStages);
+                    ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c0 & 1)));
+                    if (s == 1) ptx::umma_commit(bar(BAR_K_EMPTY + c0 % kKStages));
+                }
+                if (s == 1 && n <= 2) ptx::umma_commit(bar(BAR_Q_EMPTY));
+            };
+            // Q of unit number ul and the K blocks of its first two steps have landed.
+            auto wait_head = [&](uint32_t ul, uint32_t kc0, int n) {
+                bool ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 4));
+                for (int t0 = 0; t0 < 2 && t0 < n && ok; ++t0) {
+                    const uint32_t c0 = kc0 + t0;
                     ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + c0 % kKStages), (c0 / kKStages) & 1,
                                                           abort_flag, a.status, 5));
-                    if (!ok) break;
-                    ptx::tc_fence_after_sync();
-                    if (leader) {
-                        for (int s = 0; s < 2; ++s) {
-                            issue_qk(s, c0 & 1, c0 % kKStages);
-                            ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c0 & 1)));
-                        }
-                        ptx::umma_commit(bar(BAR_K_EMPTY + c0 % kKStages));
-                    }
-                    __syncwarp();
                 }
-                if (!ok) break;
-                if (w.n <= 2 && leader) ptx::umma_commit(bar(BAR_Q_EMPTY));
-                for (int t = 0; t < w.n && ok; ++t) {
+                ptx::tc_fence_after_sync();
+                return ok;
+            };
+            uint32_t kc = 0, ul = 0;
+            bool ok = true;
+            int n = 0, nn = 0;  // key blocks of this unit and of the next
+            uint32_t u = next_unit(blockIdx.x, n);
+            if (u < (uint32_t)a.n_units) {
+                ok = wait_head(0, 0, n);
+                if (ok && leader) {
+                    issue_head(0, 0, n);
+                    issue_head(1, 0, n);
+                }
+                __syncwarp();
+            }
+            while (u < (uint32_t)a.n_units && ok) {
+                // The next unit's coordinates are fetched now and used at this unit's last step,
+                // where the S of its first two steps is issued right behind each slot's last P V:
+                // the softmax warps then find their next logits ready while the epilogue warps
+                // are still writing this unit's O.
+                const uint32_t un = next_unit(u + gridDim.x, nn);
+                const bool has_next = un < (uint32_t)a.n_units;
+                for (int t = 0; t < n && ok; ++t) {
                     const uint32_t c = kc + t;
+                    const bool last = t + 1 == n;
                     ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_V_FULL + c % kVStages), (c / kVStages) & 1,
                                                           abort_flag, a.status, 6));
                     if (!ok) break;
-                    if (t + 2 < w.n) {
+                    if (t + 2 < n) {
                         ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + (c + 2) % kKStages),
                                                               ((c + 2) / kKStages) & 1, abort_flag, a.status, 8));
                         if (!ok) break;
@@ -283,30 +317,47 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + s), c & 1, abort_flag, a.status, 7));
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
+                        if (t == 0 && ul > 0) {
+                            // The previous unit's O must have left tensor memory.
+                            ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_O_FREE + s), (ul - 1) & 1, abort_flag, a.status, 14));
+                            if (!ok) break;
+                            ptx::tc_fence_after_sync();
+                        }
                         if (leader) {
                             issue_pv(s, c & 1, c % kVStages, t > 0);
                             ptx::umma_commit(bar(BAR_O_DONE + 2 * s + (c & 1)));
+                            if (last) ptx::umma_commit(bar(BAR_O_FINAL + s));
                             if (s == 1) ptx::umma_commit(bar(BAR_V_EMPTY + c % kVStages));
-                            if (t + 2 < w.n) {
+                            if (t + 2 < n) {
                                 issue_qk(s, c & 1, (c + 2) % kKStages);
                                 ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c & 1)));
                                 if (s == 1) {
                                     ptx::umma_commit(bar(BAR_K_EMPTY + (c + 2) % kKStages));
-                                    if (t + 3 == w.n) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                                    if (t + 3 == n) ptx::umma_commit(bar(BAR_Q_EMPTY));
                                 }
                             }
                         }
                         __syncwarp();
+                        if (last && has_next) {
+                            if (s == 0) {
+                                ok = wait_head(ul + 1, kc + n, nn);
+                                if (!ok) break;
+                            }
+                            if (leader) issue_head(s, kc + n, nn);
+                            __syncwarp();
+                        }
                     }
                 }
-                kc += w.n;
+                kc += n;
                 ++ul;
+                u = un;
+                n = nn;
             }
         }
         __syncwarp();
-    } else if (warp >= 4) {
+    } else if (warp >= 4 && warp < 12) {
         // ------------------------------------------------------------------ online softmax
-        ptx::setmaxnreg_inc<232>();
+        ptx::setmaxnreg_inc<176>();  // 4 x 40 + 8 x 176 + 4 x 120 = 16 x 128, the CTA's registers
         const int s = (warp - 4) >> 2;          // slot
         const int quad = warp & 3;              // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;       // tile row = TMEM lane
@@ -315,7 +366,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const uint32_t t_o = tmem_base + ((uint32_t)(quad * 32) << 16) + 256 + s * D;
         const float sl2 = a.scale_log2;
         const uint64_t sl2_2 = ptx::pack_f32x2(sl2, sl2);
-        uint32_t kc = 0;
+        uint32_t kc = 0, ul = 0;
         bool ok = true;
         Unit w_next = {};
         int32_t lastcol_next = -1;
@@ -454,54 +505,108 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
+                if (t + 1 == w.n) {
+                    // Row statistics for the epilogue warps (they finish O / l and the LSE).  The
+                    // previous unit's must have been read: that also keeps this slot's statistics
+                    // barrier at most one phase ahead of the epilogue.
+                    if (ul > 0) {
+                        ok = wait_bar(bar(BAR_O_FREE + s), (ul - 1) & 1, abort_flag, a.status, 13);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                    }
+                    reinterpret_cast<float2 *>(smem + SM::kStats)[s * 128 + row] = make_float2(m, l);
+                    __threadfence_block();
+                }
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(bar(BAR_P_FULL + s));
-            }
-            if (!ok) break;
-            if (w.n <= 0) {  // empty row: defined outputs, no barrier traffic
-                if (valid) {
-                    for (int c = 0; c < D; ++c) {
-                        const int64_t oi = w.b * a.o_sb + tok * a.o_ss + head * a.o_sh + c;
-                        if (a.o_is_f32) reinterpret_cast<float *>(a.o)[oi] = 0.f;
-                        else reinterpret_cast<__nv_bfloat16 *>(a.o)[oi] = __float2bfloat16_rn(0.f);
-                    }
-                    a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = -INFINITY;
-                }
-                continue;
-            }
-            // Epilogue: O / l and LSE = ln sum exp(s) = (m + log2 l) ln 2.
-            ok = wait_bar(bar(BAR_O_DONE + 2 * s + ((kc - 1) & 1)), ((kc - 1) >> 1) & 1, abort_flag, a.status, 10);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            ptx::tc_fence_after_sync();
-            const float inv = 1.0f / l;
-            const int64_t obase = w.b * a.o_sb + tok * a.o_ss + (int64_t)head * a.o_sh;
-#pragma unroll
-            for (int ch = 0; ch < D / 32; ++ch) {
-                uint32_t orr[32];
-                ptx::tmem_ld32(t_o + ch * 32, orr);
-                ptx::tmem_wait_ld();
-                if (valid) {
-                    if (a.o_is_f32) {
-                        float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(a.o) + obase + ch * 32);
-#pragma unroll
-                        for (int c = 0; c < 8; ++c)
-                            dst[c] = make_float4(__uint_as_float(orr[4 * c]) * inv, __uint_as_float(orr[4 * c + 1]) * inv,
-                                                 __uint_as_float(orr[4 * c + 2]) * inv, __uint_as_float(orr[4 * c + 3]) * inv);
-                    } else {
-                        uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(a.o) + obase + ch * 32);
-#pragma unroll
-                        for (int c = 0; c < 4; ++c)
-                            dst[c] = make_uint4(
-                                ptx::cvt_bf16x2(__uint_as_float(orr[8 * c]) * inv, __uint_as_float(orr[8 * c + 1]) * inv),
-                                ptx::cvt_bf16x2(__uint_as_float(orr[8 * c + 2]) * inv, __uint_as_float(orr[8 * c + 3]) * inv),
-                                ptx::cvt_bf16x2(__uint_as_float(orr[8 * c + 4]) * inv, __uint_as_float(orr[8 * c + 5]) * inv),
-                                ptx::cvt_bf16x2(__uint_as_float(orr[8 * c + 6]) * inv, __uint_as_float(orr[8 * c + 7]) * inv));
-                    }
+                if (lane == 0) {
+                    ptx::mbar_arrive(bar(BAR_P_FULL + s));
+                    if (t + 1 == w.n) ptx::mbar_arrive(bar(BAR_ML_READY + s));
                 }
             }
-            if (valid) a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = (m + log2f(l)) * 0.6931471805599453f;
-            ptx::tc_fence_before_sync();
+            if (w.n > 0) ++ul;
+        }
+    } else if (warp >= 12) {
+        // ------------------------------------------------------------------ epilogue
+        // O / l and LSE = ln sum exp(s) = (m + log2 l) ln 2 for both slots, off the softmax warps'
+        // critical path: O is read out of tensor memory (which frees it for the next unit), then
+        // written to global memory from registers.
+        ptx::setmaxnreg_dec<120>();
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const int qrow = row & 63;
+        uint32_t ul = 0;
+        bool ok = true;
+        for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
+            const Unit w = decode_unit(a, u);
+            const int64_t tok = (int64_t)w.i * kBlk + qrow;
+#pragma unroll 1
+            for (int s = 0; s < 2; ++s) {
+                const int head_local = w.sub * 4 + 2 * s + (row >> 6);
+                const int head = w.hk * a.G + head_local;
+                const bool valid = head_local < a.G && tok < a.N;
+                const int64_t obase = w.b * a.o_sb + tok * a.o_ss + (int64_t)head * a.o_sh;
+                if (w.n <= 0) {  // empty row: defined outputs, no barrier traffic
+                    if (valid) {
+                        for (int c = 0; c < D; ++c) {
+                            if (a.o_is_f32) reinterpret_cast<float *>(a.o)[obase + c] = 0.f;
+                            else reinterpret_cast<__nv_bfloat16 *>(a.o)[obase + c] = __float2bfloat16_rn(0.f);
+                        }
+                        a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = -INFINITY;
+                    }
+                    continue;
+                }
+                ok = wait_bar(bar(BAR_ML_READY + s), ul & 1, abort_flag, a.status, 15);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const float2 ml = reinterpret_cast<const float2 *>(smem + SM::kStats)[s * 128 + row];
+                ok = wait_bar(bar(BAR_O_FINAL + s), ul & 1, abort_flag, a.status, 10);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t t_o = tmem_base + ((uint32_t)(quad * 32) << 16) + 256 + s * D;
+                const float inv = 1.0f / ml.y;
+                if (a.o_is_f32) {
+#pragma unroll
+                    for (int ch = 0; ch < D / 32; ++ch) {
+                        uint32_t orr[32];
+                        ptx::tmem_ld32(t_o + ch * 32, orr);
+                        ptx::tmem_wait_ld();
+                        if (ch == D / 32 - 1) {
+                            ptx::tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive(bar(BAR_O_FREE + s));
+                        }
+                        if (valid) {
+                            float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(a.o) + obase + ch * 32);
+#pragma unroll
+                            for (int c = 0; c < 8; ++c)
+                                dst[c] = make_float4(__uint_as_float(orr[4 * c]) * inv, __uint_as_float(orr[4 * c + 1]) * inv,
+                                                     __uint_as_float(orr[4 * c + 2]) * inv, __uint_as_float(orr[4 * c + 3]) * inv);
+                        }
+                    }
+                } else {
+                    uint32_t pk[D / 2];
+#pragma unroll
+                    for (int ch = 0; ch < D / 32; ++ch) {
+                        uint32_t orr[32];
+                        ptx::tmem_ld32(t_o + ch * 32, orr);
+                        ptx::tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 16; ++c)
+                            pk[ch * 16 + c] = ptx::cvt_bf16x2(__uint_as_float(orr[2 * c]) * inv, __uint_as_float(orr[2 * c + 1]) * inv);
+                    }
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(bar(BAR_O_FREE + s));
+                    if (valid) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(a.o) + obase);
+#pragma unroll
+                        for (int c = 0; c < D / 8; ++c) dst[c] = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                    }
+                }
+                if (valid) a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = (ml.x + log2f(ml.y)) * 0.6931471805599453f;
+            }
+            if (w.n > 0) ++ul;
         }
     }
 
