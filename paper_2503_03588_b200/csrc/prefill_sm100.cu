@@ -28,7 +28,7 @@ namespace pa {
 
 constexpr int kBlk = 64;               // tokens per query / key block
 constexpr int kThreads = 512;          // 16 warps: control, two softmax warpgroups, epilogue
-constexpr int kKStages = 5;            // K block ring depth
+constexpr int kKStages = 4;            // K block ring depth
 constexpr int kVStages = 4;            // V block ring depth
 constexpr uint32_t kTmemCols = 512;    // slot s: S/P buffers at columns 128 s + 64 b, O at 256 + s D
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logits: rescale O only when the row max grows by more
@@ -54,10 +54,13 @@ struct SmemMap {
     static constexpr uint32_t kBlkTile = kBlkSub * (D / 64);  // one K or V block
     static constexpr uint32_t kK = kQ + 2 * kQSlot;
     static constexpr uint32_t kV = kK + kKStages * kBlkTile;
-    static constexpr uint32_t kStats = kV + kVStages * kBlkTile;  // [slot][row] (m, l) for the epilogue
-    static constexpr uint32_t kBars = kStats + 2 * 128 * 8;
+    static constexpr uint32_t kOStage = kV + kVStages * kBlkTile;  // one slot's O tile on its way out
+    static constexpr uint32_t kOStageBytes = 128 * D * 2;
+    static constexpr uint32_t kStats = kOStage + kOStageBytes;    // [slot][row] softmax denominators
+    static constexpr uint32_t kBars = kStats + 2 * 128 * 4;
     static constexpr uint32_t kTotal = kBars + 512;
     static constexpr uint32_t kAlloc = kTotal + 1024;         // slack for 1024-byte alignment
+    static_assert(kAlloc <= 227 * 1024, "shared memory budget");
 };
 
 // Barrier slots inside the barrier area (8 bytes each).
@@ -70,7 +73,9 @@ enum : uint32_t {
     BAR_O_FINAL = BAR_O_DONE + 4,   // [slot]: the unit's last P V has completed
     BAR_ML_READY = BAR_O_FINAL + 2,  // [slot]: the unit's row statistics are in shared memory
     BAR_O_FREE = BAR_ML_READY + 2,   // [slot]: the epilogue has read O out of tensor memory
-    BAR_COUNT = BAR_O_FREE + 2
+    BAR_STAGE_FREE = BAR_O_FREE + 2,  // the output staging tile has been read by its bulk stores
+    BAR_STAGE_FULL = BAR_STAGE_FREE + 1,  // ... has been written by the four epilogue warps
+    BAR_COUNT = BAR_STAGE_FULL + 1
 };
 
 struct Unit {
@@ -116,7 +121,8 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-               const __grid_constant__ CUtensorMap tmV, const PrefillArgs a)
+               const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+               const PrefillArgs a)
 {
     using SM = SmemMap<D>;
     constexpr int DH = D / 64;  // 64-feature (128-byte) sub-tiles per row
@@ -151,6 +157,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::mbar_init(bar(BAR_ML_READY + s), 4);
             ptx::mbar_init(bar(BAR_O_FREE + s), 4);
         }
+        ptx::mbar_init(bar(BAR_STAGE_FREE), 1);
+        ptx::mbar_init(bar(BAR_STAGE_FULL), 4);
         *abort_flag = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
@@ -173,9 +181,22 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::prefetch_tensormap(&tmV);
             uint32_t kc = 0, ul = 0;  // key blocks and units issued so far by this CTA
             bool ok = true;
-            for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
-                const Unit w = decode_unit(a, u);
-                if (w.n <= 0) continue;
+            // A unit's coordinates and its first block index are fetched while the previous unit's
+            // loads are still waiting for ring space, the other block indices one block ahead.
+            auto next_unit = [&](uint32_t u, Unit &w, int32_t &j0) {
+                for (; u < (uint32_t)a.n_units; u += gridDim.x) {
+                    w = decode_unit(a, u);
+                    if (w.n > 0) {
+                        j0 = __ldg(a.col_idx + w.rs);
+                        break;
+                    }
+                }
+                return u;
+            };
+            Unit w;
+            int32_t j = 0;
+            uint32_t u = next_unit(blockIdx.x, w, j);
+            while (u < (uint32_t)a.n_units && ok) {
                 if (ul > 0) ok = wait_bar(bar(BAR_Q_EMPTY), (ul - 1) & 1, abort_flag, a.status, 1);
                 if (!ok) break;
                 ptx::mbar_expect_tx(bar(BAR_Q_FULL), 2 * SM::kQSlot);
@@ -185,7 +206,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                                          bar(BAR_Q_FULL), dh * 64, w.i * kBlk,
                                          w.hk * a.G + w.sub * 4 + 2 * s, w.b);
                 for (int t = 0; t < w.n; ++t, ++kc) {
-                    const int32_t j = __ldg(a.col_idx + w.rs + t);
+                    const int32_t jn = t + 1 < w.n ? __ldg(a.col_idx + w.rs + t + 1) : 0;
                     const uint32_t ks = kc % kKStages, vs = kc % kVStages;
                     if (kc >= (uint32_t)kKStages) {
                         ok = wait_bar(bar(BAR_K_EMPTY + ks), (kc / kKStages - 1) & 1, abort_flag, a.status, 2);
@@ -203,8 +224,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     for (int dh = 0; dh < DH; ++dh)
                         ptx::tma_load_4d(smem_base + SM::kV + vs * SM::kBlkTile + dh * SM::kBlkSub, &tmV,
                                          bar(BAR_V_FULL + vs), dh * 64, j * kBlk, w.hk, w.b);
+                    j = jn;
                 }
                 ++ul;
+                u = next_unit(u + gridDim.x, w, j);
             }
             if (!ok) {
                 // Drain: give copies already in flight a bounded chance to land before exit.
@@ -253,11 +276,17 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                                       (acc || kk > 0) ? 1u : 0u);
             };
             // First non-empty unit at or after u (stride: the grid), or n_units.
-            auto next_unit = [&](uint32_t u, int &n) {
-                for (; u < (uint32_t)a.n_units; u += gridDim.x) {
-                    n = decode_unit(a, u).n;
-                    if (n > 0) break;
-                }
+            auto unit_blocks = [&](uint32_t u) {
+                return u < (uint32_t)a.n_units ? decode_unit(a, u).n : 0;
+            };
+            // Block count `n` of the candidate after u is already loaded (`ahead`); the count
+            // after that is requested now, so no unit boundary waits for a load.
+            auto next_unit = [&](uint32_t u, int &n, int &ahead) {
+                do {
+                    u += gridDim.x;
+                    n = ahead;
+                    ahead = unit_blocks(u + gridDim.x);
+                } while (u < (uint32_t)a.n_units && n <= 0);
                 return u;
             };
             // S of the first two steps of a unit, for one slot.  Steps are numbered through the
@@ -286,7 +315,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             uint32_t kc = 0, ul = 0;
             bool ok = true;
             int n = 0, nn = 0;  // key blocks of this unit and of the next
-            uint32_t u = next_unit(blockIdx.x, n);
+            int ahead = unit_blocks(blockIdx.x);
+            uint32_t u = next_unit(blockIdx.x - gridDim.x, n, ahead);  // (the sum wraps back to blockIdx.x)
             if (u < (uint32_t)a.n_units) {
                 ok = wait_head(0, 0, n);
                 if (ok && leader) {
@@ -300,7 +330,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 // where the S of its first two steps is issued right behind each slot's last P V:
                 // the softmax warps then find their next logits ready while the epilogue warps
                 // are still writing this unit's O.
-                const uint32_t un = next_unit(u + gridDim.x, nn);
+                const uint32_t un = next_unit(u, nn, ahead);
                 const bool has_next = un < (uint32_t)a.n_units;
                 for (int t = 0; t < n && ok; ++t) {
                     const uint32_t c = kc + t;
@@ -368,20 +398,23 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const uint64_t sl2_2 = ptx::pack_f32x2(sl2, sl2);
         uint32_t kc = 0, ul = 0;
         bool ok = true;
-        Unit w_next = {};
-        int32_t lastcol_next = -1;
-        if (blockIdx.x < (uint32_t)a.n_units) {
-            w_next = decode_unit(a, blockIdx.x);
-            if (w_next.n > 0) lastcol_next = __ldg(a.col_idx + w_next.rs + w_next.n - 1);
-        }
+        // Unit metadata runs ahead of its use so that no load sits between two units: the row
+        // extent two units ahead, the row's last block index (needs the extent) one unit ahead.
+        auto fetch_unit = [&](uint32_t u) {
+            Unit r = {};
+            if (u < (uint32_t)a.n_units) r = decode_unit(a, u);
+            return r;
+        };
+        auto fetch_lastcol = [&](const Unit &r) { return r.n > 0 ? __ldg(a.col_idx + r.rs + r.n - 1) : -1; };
+        Unit w_next = fetch_unit(blockIdx.x);
+        Unit w_next2 = fetch_unit(blockIdx.x + gridDim.x);
+        int32_t lastcol_next = fetch_lastcol(w_next);
         for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
             const Unit w = w_next;
             const int32_t lastcol = lastcol_next;
-            if (u + gridDim.x < (uint32_t)a.n_units) {
-                // Metadata of the next unit: loaded now, used one unit later.
-                w_next = decode_unit(a, u + gridDim.x);
-                lastcol_next = w_next.n > 0 ? __ldg(a.col_idx + w_next.rs + w_next.n - 1) : -1;
-            }
+            w_next = w_next2;
+            lastcol_next = fetch_lastcol(w_next);
+            w_next2 = fetch_unit(u + 2 * gridDim.x);
             const int head_local = w.sub * 4 + 2 * s + (row >> 6);
             const int head = w.hk * a.G + head_local;
             const int64_t tok = (int64_t)w.i * kBlk + qrow;
@@ -506,16 +539,18 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 if (t + 1 == w.n) {
-                    // Row statistics for the epilogue warps (they finish O / l and the LSE).  The
-                    // previous unit's must have been read: that also keeps this slot's statistics
-                    // barrier at most one phase ahead of the epilogue.
+                    // Softmax denominators for the epilogue warps (they finish O / l).  The previous
+                    // unit's must have been read: that also keeps this slot's statistics barrier at
+                    // most one phase ahead of the epilogue.
                     if (ul > 0) {
                         ok = wait_bar(bar(BAR_O_FREE + s), (ul - 1) & 1, abort_flag, a.status, 13);
                         ok = __all_sync(0xffffffffu, ok);
                         if (!ok) break;
                     }
-                    reinterpret_cast<float2 *>(smem + SM::kStats)[s * 128 + row] = make_float2(m, l);
+                    reinterpret_cast<float *>(smem + SM::kStats)[s * 128 + row] = l;
                     __threadfence_block();
+                    // LSE = ln sum exp(s) = (m + log2 l) ln 2.
+                    if (valid) a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = (m + log2f(l)) * 0.6931471805599453f;
                 }
                 __syncwarp();
                 if (lane == 0) {
@@ -527,14 +562,18 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
     } else if (warp >= 12) {
         // ------------------------------------------------------------------ epilogue
-        // O / l and LSE = ln sum exp(s) = (m + log2 l) ln 2 for both slots, off the softmax warps'
-        // critical path: O is read out of tensor memory (which frees it for the next unit), then
-        // written to global memory from registers.
+        // O / l for both slots, off the softmax warps' critical path.  O is read out of tensor
+        // memory (which frees it for the next unit); bf16 output is staged in shared memory in
+        // the 128-byte-swizzled box layout and leaves as bulk tensor stores, one per head and
+        // 64-feature half (rows beyond the sequence end are clipped by the tensor map), fp32
+        // output is written from registers.
         ptx::setmaxnreg_dec<120>();
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const int qrow = row & 63;
-        uint32_t ul = 0;
+        const bool store_thread = threadIdx.x == 12 * 32;
+        const uint32_t stage = smem_base + SM::kOStage;
+        uint32_t ul = 0, ns = 0;  // units and staged tiles so far
         bool ok = true;
         for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
             const Unit w = decode_unit(a, u);
@@ -558,13 +597,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 ok = wait_bar(bar(BAR_ML_READY + s), ul & 1, abort_flag, a.status, 15);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                const float2 ml = reinterpret_cast<const float2 *>(smem + SM::kStats)[s * 128 + row];
+                const float inv = 1.0f / reinterpret_cast<const float *>(smem + SM::kStats)[s * 128 + row];
                 ok = wait_bar(bar(BAR_O_FINAL + s), ul & 1, abort_flag, a.status, 10);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t t_o = tmem_base + ((uint32_t)(quad * 32) << 16) + 256 + s * D;
-                const float inv = 1.0f / ml.y;
                 if (a.o_is_f32) {
 #pragma unroll
                     for (int ch = 0; ch < D / 32; ++ch) {
@@ -598,16 +636,46 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     ptx::tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(bar(BAR_O_FREE + s));
-                    if (valid) {
-                        uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(a.o) + obase);
+                    // The staging tile is free once the previous bulk stores have read it.
+                    if (store_thread) {
+                        ptx::bulk_wait_read_all();
+                        ptx::mbar_arrive(bar(BAR_STAGE_FREE));
+                    }
+                    ok = wait_bar(bar(BAR_STAGE_FREE), ns & 1, abort_flag, a.status, 16);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    // Box (row >> 6, half): 64 tokens x 128 bytes; 16-byte chunk j of token t sits at
+                    // chunk position j ^ (t & 7).
+                    const uint32_t rbase = stage + (uint32_t)(row >> 6) * (uint32_t)(DH * 8192) + (uint32_t)qrow * 128u;
 #pragma unroll
-                        for (int c = 0; c < D / 8; ++c) dst[c] = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                    for (int c = 0; c < D / 8; ++c) {
+                        const uint32_t dst = rbase + (uint32_t)(c >> 3) * 8192u + ((uint32_t)((c & 7) ^ (qrow & 7)) << 4);
+                        ptx::st_shared_v4(dst, pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                    }
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(bar(BAR_STAGE_FULL));
+                    if (warp == 12) {
+                        ok = wait_bar(bar(BAR_STAGE_FULL), ns & 1, abort_flag, a.status, 17);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                    }
+                    ++ns;
+                    if (store_thread) {
+                        for (int hh = 0; hh < 2; ++hh) {
+                            const int hl = w.sub * 4 + 2 * s + hh;
+                            if (hl >= a.G) continue;
+                            for (int dh = 0; dh < DH; ++dh)
+                                ptx::tma_store_4d(&tmO, stage + (uint32_t)(hh * DH + dh) * 8192u, dh * 64, w.i * kBlk,
+                                                  w.hk * a.G + hl, w.b);
+                        }
+                        ptx::bulk_commit_group();
                     }
                 }
-                if (valid) a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = (ml.x + log2f(ml.y)) * 0.6931471805599453f;
             }
             if (w.n > 0) ++ul;
         }
+        if (store_thread) ptx::bulk_wait_all();
     }
 
     ptx::tc_fence_before_sync();
@@ -724,11 +792,16 @@ extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const
 
     EncodeTiledFn enc = nullptr;
     if (pa_status s = get_encode_fn(&enc)) return s;
-    CUtensorMap tmQ, tmK, tmV;
+    CUtensorMap tmQ, tmK, tmV, tmO;
     const int D = p->head_dim;
     if (pa_status s = make_map(enc, &tmQ, q, D, p->seq_len, p->n_q_heads, p->batch, p->q, 2, "q")) return s;
     if (pa_status s = make_map(enc, &tmK, k, D, p->seq_len, p->n_kv_heads, p->batch, p->k, 1, "k")) return s;
     if (pa_status s = make_map(enc, &tmV, v, D, p->seq_len, p->n_kv_heads, p->batch, p->v, 1, "v")) return s;
+    if (p->o_dtype == PA_BF16) {
+        if (pa_status s = make_map(enc, &tmO, o, D, p->seq_len, p->n_q_heads, p->batch, p->o, 1, "o")) return s;
+    } else {
+        tmO = tmQ;  // fp32 output is written from registers; the map is not used
+    }
 
     PrefillArgs a;
     a.row_ptr = row_ptr;
@@ -757,11 +830,11 @@ extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const
     if (D == 128) {
         PA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)SmemMap<128>::kAlloc));
-        prefill_kernel<128><<<grid, kThreads, SmemMap<128>::kAlloc, st>>>(tmQ, tmK, tmV, a);
+        prefill_kernel<128><<<grid, kThreads, SmemMap<128>::kAlloc, st>>>(tmQ, tmK, tmV, tmO, a);
     } else {
         PA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)SmemMap<64>::kAlloc));
-        prefill_kernel<64><<<grid, kThreads, SmemMap<64>::kAlloc, st>>>(tmQ, tmK, tmV, a);
+        prefill_kernel<64><<<grid, kThreads, SmemMap<64>::kAlloc, st>>>(tmQ, tmK, tmV, tmO, a);
     }
     PA_CUDA_OK(cudaGetLastError());
     return PA_OK;
