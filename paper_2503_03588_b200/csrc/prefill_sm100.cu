@@ -24,6 +24,20 @@
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
+// Registers per thread by role: 4 control warps, 8 softmax warps, 4 epilogue warps share the
+// CTA's 16 x 128.
+#ifndef PA_REG_CTRL
+#define PA_REG_CTRL 56
+#define PA_REG_SOFT 168
+#define PA_REG_EPI 120
+#endif
+// A warpgroup asking for more than the pool holds would wait for ever.
+static_assert(4 * PA_REG_CTRL + 8 * PA_REG_SOFT + 4 * PA_REG_EPI <= 16 * 128, "register split exceeds the CTA's registers");
+static_assert(PA_REG_CTRL % 8 == 0 && PA_REG_SOFT % 8 == 0 && PA_REG_EPI % 8 == 0, "setmaxnreg takes multiples of 8");
+#ifndef PA_WAIT_HINT_NS
+#define PA_WAIT_HINT_NS 0
+#endif
+
 namespace pa {
 
 constexpr int kBlk = 64;               // tokens per query / key block
@@ -106,7 +120,11 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     const long long t0 = clock64();
     uint32_t it = 0;
     while (true) {
+#if PA_WAIT_HINT_NS > 0
+        if (ptx::mbar_try_wait_hint(bar, parity, PA_WAIT_HINT_NS)) return true;
+#else
         if (ptx::mbar_try_wait(bar, parity)) return true;
+#endif
         if ((++it & 63u) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitCycles) break;
@@ -172,7 +190,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp < 4) ptx::setmaxnreg_dec<40>();
+    if (warp < 4) ptx::setmaxnreg_dec<PA_REG_CTRL>();
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -387,7 +405,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         __syncwarp();
     } else if (warp >= 4 && warp < 12) {
         // ------------------------------------------------------------------ online softmax
-        ptx::setmaxnreg_inc<176>();  // 4 x 40 + 8 x 176 + 4 x 120 = 16 x 128, the CTA's registers
+        ptx::setmaxnreg_inc<PA_REG_SOFT>();
         const int s = (warp - 4) >> 2;          // slot
         const int quad = warp & 3;              // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;       // tile row = TMEM lane
@@ -567,7 +585,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         // the 128-byte-swizzled box layout and leaves as bulk tensor stores, one per head and
         // 64-feature half (rows beyond the sequence end are clipped by the tensor map), fp32
         // output is written from registers.
-        ptx::setmaxnreg_dec<120>();
+        ptx::setmaxnreg_dec<PA_REG_EPI>();
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const int qrow = row & 63;
