@@ -34,6 +34,9 @@
 // A warpgroup asking for more than the pool holds would wait for ever.
 static_assert(4 * PA_REG_CTRL + 8 * PA_REG_SOFT + 4 * PA_REG_EPI <= 16 * 128, "register split exceeds the CTA's registers");
 static_assert(PA_REG_CTRL % 8 == 0 && PA_REG_SOFT % 8 == 0 && PA_REG_EPI % 8 == 0, "setmaxnreg takes multiples of 8");
+#ifndef PA_UNIFORM
+#define PA_UNIFORM 1
+#endif
 #ifndef PA_WAIT_HINT_NS
 #define PA_WAIT_HINT_NS 0
 #endif
@@ -188,7 +191,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_base_any = *tmem_slot;
+    const uint32_t tmem_base = tmem_base_any;
 
     if (warp < 4) ptx::setmaxnreg_dec<PA_REG_CTRL>();
     if (warp == 0) {
@@ -265,6 +269,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         // the leading-dimension offset for the MN-major V operand).
         {
             const bool leader = ptx::elect_one();
+#if PA_UNIFORM
+            const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_any, 0);
+#else
+            const uint32_t tmem_base = tmem_base_any;
+#endif
             constexpr uint32_t idesc_qk = ptx::idesc_bf16_f32(128, 64, 0);
             constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(128, D, 1);
             constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
@@ -294,9 +303,17 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                                       (acc || kk > 0) ? 1u : 0u);
             };
             // First non-empty unit at or after u (stride: the grid), or n_units.
+#if PA_UNIFORM
+            // Every lane loads the same words; the shuffle tells the compiler so, which lets the
+            // loop bounds, ring positions and descriptors live in uniform registers.
+            auto unit_blocks = [&](uint32_t u) {
+                return __shfl_sync(0xffffffffu, u < (uint32_t)a.n_units ? decode_unit(a, u).n : 0, 0);
+            };
+#else
             auto unit_blocks = [&](uint32_t u) {
                 return u < (uint32_t)a.n_units ? decode_unit(a, u).n : 0;
             };
+#endif
             // Block count `n` of the candidate after u is already loaded (`ahead`); the count
             // after that is requested now, so no unit boundary waits for a load.
             auto next_unit = [&](uint32_t u, int &n, int &ahead) {
