@@ -48,6 +48,13 @@ constexpr int kThreads = 512;          // 16 warps: control, two softmax warpgro
 constexpr int kKStages = 4;            // K block ring depth
 constexpr int kVStages = 4;            // V block ring depth
 constexpr uint32_t kTmemCols = 512;    // slot s: S/P buffers at columns 128 s + 64 b, O at 256 + s D
+// P is packed to bf16 by keeping the high halves of two fp32 values (one permute, no conversion
+// instruction: conversions share the exponential unit's issue rate).  Truncation alone would
+// bias P low, so every exponent carries +log2(1 + 2^-9): truncating p (1 + 2^-9) is centred on
+// p like rounding to nearest.  The row sums l carry the same factor; it is divided out of
+// O / l and subtracted from the LSE at the end.
+constexpr float kPackShiftLog2 = 0.0028150156070540f;  // log2(1 + 2^-9)
+constexpr float kPackScale = 1.001953125f;             // 1 + 2^-9
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logits: rescale O only when the row max grows by more
 constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
 
@@ -479,7 +486,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 // exact whatever reference was used).  Two-wide fp32 arithmetic; the row maximum
                 // is watched on the rounded bf16 values (p > 2^threshold <=> s - m > threshold;
                 // an overflow shows up as inf).
-                const uint64_t negm_2 = ptx::pack_f32x2(-m, -m);
+                const float negm = kPackShiftLog2 - m;
+                const uint64_t negm_2 = ptx::pack_f32x2(negm, negm);
                 uint64_t sum2[2] = {0ull, 0ull};
                 uint32_t pmax2[2] = {0u, 0u};
                 uint32_t pk[32];
@@ -495,7 +503,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         ptx::unpack_f32x2(y2, y0, y1);
                         const float p0 = ptx::ex2(y0), p1 = ptx::ex2(y1);
                         sum2[e] = ptx::add_f32x2(sum2[e], ptx::pack_f32x2(p0, p1));
-                        const uint32_t q = ptx::cvt_bf16x2(p0, p1);
+                        const uint32_t q = ptx::pack_bf16x2_trunc(p0, p1);
                         pk[(c >> 1) + e] = q;
                         pmax2[e] = ptx::max_bf16x2(pmax2[e], q);
                     }
@@ -552,11 +560,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         float pv[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            pv[e] = ptx::ex2(fmaf(__uint_as_float(sr[c + e]), sl2, -m));
+                            pv[e] = ptx::ex2(fmaf(__uint_as_float(sr[c + e]), sl2, kPackShiftLog2 - m));
                             sum4[e] += pv[e];
                         }
-                        pk[c >> 1] = ptx::cvt_bf16x2(pv[0], pv[1]);
-                        pk[(c >> 1) + 1] = ptx::cvt_bf16x2(pv[2], pv[3]);
+                        pk[c >> 1] = ptx::pack_bf16x2_trunc(pv[0], pv[1]);
+                        pk[(c >> 1) + 1] = ptx::pack_bf16x2_trunc(pv[2], pv[3]);
                     }
                     sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
                 }
@@ -585,7 +593,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     reinterpret_cast<float *>(smem + SM::kStats)[s * 128 + row] = l;
                     __threadfence_block();
                     // LSE = ln sum exp(s) = (m + log2 l) ln 2.
-                    if (valid) a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = (m + log2f(l)) * 0.6931471805599453f;
+                    if (valid) a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = (m + log2f(l) - kPackShiftLog2) * 0.6931471805599453f;
                 }
                 __syncwarp();
                 if (lane == 0) {
@@ -632,7 +640,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 ok = wait_bar(bar(BAR_ML_READY + s), ul & 1, abort_flag, a.status, 15);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                const float inv = 1.0f / reinterpret_cast<const float *>(smem + SM::kStats)[s * 128 + row];
+                const float inv = kPackScale / reinterpret_cast<const float *>(smem + SM::kStats)[s * 128 + row];
                 ok = wait_bar(bar(BAR_O_FINAL + s), ul & 1, abort_flag, a.status, 10);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
