@@ -48,13 +48,8 @@ constexpr int kThreads = 512;          // 16 warps: control, two softmax warpgro
 constexpr int kKStages = 4;            // K block ring depth
 constexpr int kVStages = 4;            // V block ring depth
 constexpr uint32_t kTmemCols = 512;    // slot s: S/P buffers at columns 128 s + 64 b, O at 256 + s D
-// P is packed to bf16 by keeping the high halves of two fp32 values (one permute, no conversion
-// instruction: conversions share the exponential unit's issue rate).  Truncation alone would
-// bias P low, so every exponent carries +log2(1 + 2^-9): truncating p (1 + 2^-9) is centred on
-// p like rounding to nearest.  The row sums l carry the same factor; it is divided out of
-// O / l and subtracted from the LSE at the end.
-constexpr float kPackShiftLog2 = 0.0028150156070540f;  // log2(1 + 2^-9)
-constexpr float kPackScale = 1.001953125f;             // 1 + 2^-9
+// A step's row sum above this limit sends the step through the exact path (new reference).
+constexpr float kSumLimit = 1048576.0f;  // 2^20
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logits: rescale O only when the row max grows by more
 constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
 
@@ -451,12 +446,16 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         Unit w_next = fetch_unit(blockIdx.x);
         Unit w_next2 = fetch_unit(blockIdx.x + gridDim.x);
         int32_t lastcol_next = fetch_lastcol(w_next);
-        for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
-            const Unit w = w_next;
-            const int32_t lastcol = lastcol_next;
+        // Called once per unit, after the first step's hand-over (the issuer is busy with it then),
+        // not between two units where the next logits are already waiting.
+        auto advance_metadata = [&](uint32_t u) {
             w_next = w_next2;
             lastcol_next = fetch_lastcol(w_next);
             w_next2 = fetch_unit(u + 2 * gridDim.x);
+        };
+        for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
+            const Unit w = w_next;
+            const int32_t lastcol = lastcol_next;
             const int head_local = w.sub * 4 + 2 * s + (row >> 6);
             const int head = w.hk * a.G + head_local;
             const int64_t tok = (int64_t)w.i * kBlk + qrow;
@@ -481,15 +480,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         if (c > qrow) sr[c] = 0xff800000u;  // -inf
                 }
                 // Fast path: p = exp2(s * scale - m) against the reference maximum m carried from
-                // earlier steps (lazy rescaling: m moves only when the row maximum exceeds it by
-                // more than the threshold, so p stays below 2^threshold and O / l at the end is
-                // exact whatever reference was used).  Two-wide fp32 arithmetic; the row maximum
-                // is watched on the rounded bf16 values (p > 2^threshold <=> s - m > threshold;
-                // an overflow shows up as inf).
-                const float negm = kPackShiftLog2 - m;
-                const uint64_t negm_2 = ptx::pack_f32x2(negm, negm);
+                // earlier steps (lazy rescaling: O / l at the end is exact whatever reference was
+                // used, as long as nothing overflows).  Two-wide fp32 arithmetic.  The watch is the
+                // step's row sum, which is needed anyway: it bounds every p of the row from above,
+                // so a sum within the limit means no p came near the fp32 / bf16 range, and an
+                // overflow shows up as inf.
+                const uint64_t negm_2 = ptx::pack_f32x2(-m, -m);
                 uint64_t sum2[2] = {0ull, 0ull};
-                uint32_t pmax2[2] = {0u, 0u};
                 uint32_t pk[32];
                 if (t > 0) {  // the first step of a unit has no reference yet: straight to the exact path
 #pragma unroll
@@ -503,9 +500,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         ptx::unpack_f32x2(y2, y0, y1);
                         const float p0 = ptx::ex2(y0), p1 = ptx::ex2(y1);
                         sum2[e] = ptx::add_f32x2(sum2[e], ptx::pack_f32x2(p0, p1));
-                        const uint32_t q = ptx::pack_bf16x2_trunc(p0, p1);
-                        pk[(c >> 1) + e] = q;
-                        pmax2[e] = ptx::max_bf16x2(pmax2[e], q);
+                        pk[(c >> 1) + e] = ptx::cvt_bf16x2(p0, p1);
                     }
                 }
                 }
@@ -516,10 +511,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     ptx::unpack_f32x2(sum2[1], s2, s3);
                     sum = (s0 + s1) + (s2 + s3);
                 }
-                const uint32_t pm = ptx::max_bf16x2(pmax2[0], pmax2[1]);
-                const float pmaxf = fmaxf(__uint_as_float(pm << 16), __uint_as_float(pm & 0xffff0000u));
                 // !(x <= limit) also catches inf and NaN.
-                const bool suspect = t == 0 || !(pmaxf <= 256.0f);
+                const bool suspect = t == 0 || !(sum <= kSumLimit);
                 if (__any_sync(0xffffffffu, suspect)) {
                     // Rare path: exact row maximum, new reference for the rows that need it, what
                     // was accumulated so far brought to the new reference, P recomputed from the
@@ -560,11 +553,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         float pv[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            pv[e] = ptx::ex2(fmaf(__uint_as_float(sr[c + e]), sl2, kPackShiftLog2 - m));
+                            pv[e] = ptx::ex2(fmaf(__uint_as_float(sr[c + e]), sl2, -m));
                             sum4[e] += pv[e];
                         }
-                        pk[c >> 1] = ptx::pack_bf16x2_trunc(pv[0], pv[1]);
-                        pk[(c >> 1) + 1] = ptx::pack_bf16x2_trunc(pv[2], pv[3]);
+                        pk[c >> 1] = ptx::cvt_bf16x2(pv[0], pv[1]);
+                        pk[(c >> 1) + 1] = ptx::cvt_bf16x2(pv[2], pv[3]);
                     }
                     sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
                 }
@@ -581,6 +574,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(BAR_P_FULL + s));
+                if (t == 0) advance_metadata(u);
                 if (t + 1 == w.n) {
                     // Softmax denominators for the epilogue warps (they finish O / l).  The previous
                     // unit's must have been read: that also keeps this slot's statistics barrier at
@@ -593,15 +589,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     reinterpret_cast<float *>(smem + SM::kStats)[s * 128 + row] = l;
                     __threadfence_block();
                     // LSE = ln sum exp(s) = (m + log2 l) ln 2.
-                    if (valid) a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = (m + log2f(l) - kPackShiftLog2) * 0.6931471805599453f;
-                }
-                __syncwarp();
-                if (lane == 0) {
-                    ptx::mbar_arrive(bar(BAR_P_FULL + s));
-                    if (t + 1 == w.n) ptx::mbar_arrive(bar(BAR_ML_READY + s));
+                    if (valid) a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = (m + log2f(l)) * 0.6931471805599453f;
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(bar(BAR_ML_READY + s));
                 }
             }
             if (w.n > 0) ++ul;
+            else advance_metadata(u);
         }
     } else if (warp >= 12) {
         // ------------------------------------------------------------------ epilogue
@@ -640,7 +634,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 ok = wait_bar(bar(BAR_ML_READY + s), ul & 1, abort_flag, a.status, 15);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                const float inv = kPackScale / reinterpret_cast<const float *>(smem + SM::kStats)[s * 128 + row];
+                const float inv = 1.0f / reinterpret_cast<const float *>(smem + SM::kStats)[s * 128 + row];
                 ok = wait_bar(bar(BAR_O_FINAL + s), ul & 1, abort_flag, a.status, 10);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;

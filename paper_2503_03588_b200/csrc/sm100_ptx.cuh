@@ -310,11 +310,6 @@ __device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi)
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
-// High halves of two fp32 values as a bf16 pair (lo in the low half): truncation, one permute.
-__device__ __forceinline__ uint32_t pack_bf16x2_trunc(float lo, float hi)
-{
-    return __byte_perm(__float_as_uint(lo), __float_as_uint(hi), 0x7632);
-}
 __device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b)
 {
     uint32_t r;
