@@ -87,8 +87,8 @@ enum : uint32_t {
     BAR_Q_FULL = 0, BAR_Q_EMPTY = 1, BAR_K_FULL = 2, BAR_K_EMPTY = BAR_K_FULL + kKStages,
     BAR_V_FULL = BAR_K_EMPTY + kKStages, BAR_V_EMPTY = BAR_V_FULL + kVStages,
     BAR_S_FULL = BAR_V_EMPTY + kVStages,  // [slot][buffer]
-    BAR_P_FULL = BAR_S_FULL + 4,
-    BAR_O_DONE = BAR_P_FULL + 2,  // [slot][step parity]: P V of that step has completed
+    BAR_P_FULL = BAR_S_FULL + 4,  // [slot][step parity]: P of that step is in tensor memory
+    BAR_O_DONE = BAR_P_FULL + 4,  // [slot][step parity]: P V of that step has completed
     BAR_O_FINAL = BAR_O_DONE + 4,   // [slot]: the unit's last P V has completed
     BAR_ML_READY = BAR_O_FINAL + 2,  // [slot]: the unit's row statistics are in shared memory
     BAR_O_FREE = BAR_ML_READY + 2,   // [slot]: the epilogue has read O out of tensor memory
@@ -175,7 +175,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::mbar_init(bar(BAR_O_DONE + s), 1);
         }
         for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(bar(BAR_P_FULL + s), 4);  // one arrival per softmax warp of the slot
+            ptx::mbar_init(bar(BAR_P_FULL + 2 * s), 4);  // one arrival per softmax warp of the slot
+            ptx::mbar_init(bar(BAR_P_FULL + 2 * s + 1), 4);
             ptx::mbar_init(bar(BAR_O_FINAL + s), 1);
             ptx::mbar_init(bar(BAR_ML_READY + s), 4);
             ptx::mbar_init(bar(BAR_O_FREE + s), 4);
@@ -381,7 +382,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         if (!ok) break;
                     }
                     for (int s = 0; s < 2; ++s) {
-                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + s), c & 1, abort_flag, a.status, 7));
+                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + 2 * s + (c & 1)), (c >> 1) & 1, abort_flag, a.status, 7));
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
                         if (t == 0 && ul > 0) {
@@ -464,13 +465,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             // with that block.
             const bool last_is_diag = w.n > 0 && lastcol == w.i;
             float m = -INFINITY, l = 0.f;
+            uint32_t sr[64];
             for (int t = 0; t < w.n; ++t, ++kc) {
                 const uint32_t t_s = t_s0 + (kc & 1) * 64;
                 ok = wait_bar(bar(BAR_S_FULL + 2 * s + (kc & 1)), (kc >> 1) & 1, abort_flag, a.status, 9);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                uint32_t sr[64];
                 ptx::tmem_ld32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
                 ptx::tmem_ld32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
                 ptx::tmem_wait_ld();
@@ -564,18 +565,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 l += sum;
                 // P (bf16 pairs) overlays the first 32 columns of the S buffer just read.
                 ptx::tmem_st32(t_s, pk);
-                if (kc > 0) {
-                    // Do not run two P hand-overs ahead of the issuer: its parity wait on this slot's
-                    // P barrier can tell only one completed phase from none.  Once the previous
-                    // step's P V has completed (normally long ago) the issuer has consumed that phase.
-                    ok = wait_bar(bar(BAR_O_DONE + 2 * s + ((kc - 1) & 1)), ((kc - 1) >> 1) & 1, abort_flag, a.status, 12);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                }
+                // (The hand-over barriers alternate by step parity like the S buffers: the S of step
+                // kc + 2 is issued behind the P V of step kc, so a barrier is never more than one
+                // phase ahead of the issuer, whose parity wait could not tell two from none.)
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(bar(BAR_P_FULL + s));
+                if (lane == 0) ptx::mbar_arrive(bar(BAR_P_FULL + 2 * s + (kc & 1)));
                 if (t == 0) advance_metadata(u);
                 if (t + 1 == w.n) {
                     // Softmax denominators for the epilogue warps (they finish O / l).  The previous
