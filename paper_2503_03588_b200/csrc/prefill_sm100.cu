@@ -34,9 +34,6 @@
 // A warpgroup asking for more than the pool holds would wait for ever.
 static_assert(4 * PA_REG_CTRL + 8 * PA_REG_SOFT + 4 * PA_REG_EPI <= 16 * 128, "register split exceeds the CTA's registers");
 static_assert(PA_REG_CTRL % 8 == 0 && PA_REG_SOFT % 8 == 0 && PA_REG_EPI % 8 == 0, "setmaxnreg takes multiples of 8");
-#ifndef PA_UNIFORM
-#define PA_UNIFORM 1
-#endif
 #ifndef PA_WAIT_HINT_NS
 #define PA_WAIT_HINT_NS 0
 #endif
@@ -86,8 +83,9 @@ struct SmemMap {
 enum : uint32_t {
     BAR_Q_FULL = 0, BAR_Q_EMPTY = 1, BAR_K_FULL = 2, BAR_K_EMPTY = BAR_K_FULL + kKStages,
     BAR_V_FULL = BAR_K_EMPTY + kKStages, BAR_V_EMPTY = BAR_V_FULL + kVStages,
-    BAR_S_FULL = BAR_V_EMPTY + kVStages,  // [slot][buffer]
-    BAR_P_FULL = BAR_S_FULL + 4,  // [slot][step parity]: P of that step is in tensor memory
+    BAR_S_FULL = BAR_V_EMPTY + kVStages,  // [slot]: S of the step is in tensor memory
+    BAR_S_TAKEN = BAR_S_FULL + 2,         // [slot]: the softmax warps have S in registers
+    BAR_P_FULL = BAR_S_TAKEN + 2,  // [slot][step parity]: P of that step is in tensor memory
     BAR_O_DONE = BAR_P_FULL + 4,  // [slot][step parity]: P V of that step has completed
     BAR_O_FINAL = BAR_O_DONE + 4,   // [slot]: the unit's last P V has completed
     BAR_ML_READY = BAR_O_FINAL + 2,  // [slot]: the unit's row statistics are in shared memory
@@ -170,12 +168,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::mbar_init(bar(BAR_V_FULL + s), 1);
             ptx::mbar_init(bar(BAR_V_EMPTY + s), 1);
         }
-        for (int s = 0; s < 4; ++s) {
-            ptx::mbar_init(bar(BAR_S_FULL + s), 1);
-            ptx::mbar_init(bar(BAR_O_DONE + s), 1);
-        }
+        for (int s = 0; s < 4; ++s) ptx::mbar_init(bar(BAR_O_DONE + s), 1);
         for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(bar(BAR_P_FULL + 2 * s), 4);  // one arrival per softmax warp of the slot
+            ptx::mbar_init(bar(BAR_S_FULL + s), 1);
+            ptx::mbar_init(bar(BAR_S_TAKEN + s), 4);  // one arrival per softmax warp of the slot
+            ptx::mbar_init(bar(BAR_P_FULL + 2 * s), 4);
             ptx::mbar_init(bar(BAR_P_FULL + 2 * s + 1), 4);
             ptx::mbar_init(bar(BAR_O_FINAL + s), 1);
             ptx::mbar_init(bar(BAR_ML_READY + s), 4);
@@ -265,18 +262,20 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     } else if (warp == 1) {
         // ------------------------------------------------------------------ tcgen05 issuer
         // The whole warp runs the (uniform) control flow and the barrier waits; one elected lane
-        // issues the MMAs and commits.  MMAs of one issuer execute in issue order, which is what
-        // lets the S of step t+2 overwrite the buffer whose P was read by the P V of step t.
+        // issues the MMAs and commits.  Steps are numbered through the CTA's whole run (c), so ring
+        // positions and buffer parities do not care about unit boundaries.  Per step c and slot:
+        //   S(c + 1) = Q K^T is issued as soon as the softmax warps have taken S(c) out of tensor
+        //   memory (S has one buffer per slot; P has its own two), i.e. while they still work on
+        //   step c, and it may belong to the next unit;
+        //   O += P(c) V(c) is issued when P(c) has been handed over.
         // Descriptors: the high word is constant per operand kind (stride 1024 B between 8-row
         // groups, version 1, 128-byte swizzle); the low word holds the start address >> 4 (plus
         // the leading-dimension offset for the MN-major V operand).
         {
             const bool leader = ptx::elect_one();
-#if PA_UNIFORM
+            // Every lane holds the same values; the shuffles tell the compiler so, which lets the
+            // loop bounds, ring positions and descriptors live in uniform registers.
             const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_any, 0);
-#else
-            const uint32_t tmem_base = tmem_base_any;
-#endif
             constexpr uint32_t idesc_qk = ptx::idesc_bf16_f32(128, 64, 0);
             constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(128, D, 1);
             constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
@@ -284,41 +283,32 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const uint32_t k_lo = ((smem_base + SM::kK) >> 4) | (1u << 16);
             const uint32_t v_lo = ((smem_base + SM::kV) >> 4) | ((SM::kBlkSub >> 4) << 16);
             // S = Q K^T: A = Q tile (K-major), B = K block (K-major), 16 features per MMA.
-            auto issue_qk = [&](int s, uint32_t buf, uint32_t ks) {
+            auto issue_qk = [&](int s, uint32_t ks) {
                 const uint32_t qa = q_lo + s * (SM::kQSlot >> 4);
                 const uint32_t kb = k_lo + ks * (SM::kBlkTile >> 4);
-                const uint32_t dst = tmem_base + s * 128 + buf * 64;
+                const uint32_t dst = tmem_base + s * 128;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk)
                     ptx::umma_ss_lohi(dst, qa + (((kk / 4) * SM::kQSub + (kk % 4) * 32) >> 4), desc_hi,
                                       kb + (((kk / 4) * SM::kBlkSub + (kk % 4) * 32) >> 4), desc_hi, idesc_qk,
                                       kk > 0 ? 1u : 0u);
             };
-            // O (+)= P V: A = P (tensor memory: bf16 pairs in the first 32 columns of the S buffer),
-            // B = V block (MN-major: features contiguous), 16 keys per MMA.
+            // O (+)= P V: A = P (tensor memory, bf16 pairs, buffer = step parity), B = V block
+            // (MN-major: features contiguous), 16 keys per MMA.
             auto issue_pv = [&](int s, uint32_t buf, uint32_t vs, bool acc) {
                 const uint32_t vb = v_lo + vs * (SM::kBlkTile >> 4);
                 const uint32_t dst = tmem_base + 256 + s * D;
-                const uint32_t pa_ = tmem_base + s * 128 + buf * 64;
+                const uint32_t pa_ = tmem_base + s * 128 + 64 + buf * 32;
 #pragma unroll
                 for (int kk = 0; kk < kBlk / 16; ++kk)
                     ptx::umma_ts_lohi(dst, pa_ + kk * 8, vb + ((kk * 2048) >> 4), desc_hi, idesc_pv,
                                       (acc || kk > 0) ? 1u : 0u);
             };
-            // First non-empty unit at or after u (stride: the grid), or n_units.
-#if PA_UNIFORM
-            // Every lane loads the same words; the shuffle tells the compiler so, which lets the
-            // loop bounds, ring positions and descriptors live in uniform registers.
             auto unit_blocks = [&](uint32_t u) {
                 return __shfl_sync(0xffffffffu, u < (uint32_t)a.n_units ? decode_unit(a, u).n : 0, 0);
             };
-#else
-            auto unit_blocks = [&](uint32_t u) {
-                return u < (uint32_t)a.n_units ? decode_unit(a, u).n : 0;
-            };
-#endif
-            // Block count `n` of the candidate after u is already loaded (`ahead`); the count
-            // after that is requested now, so no unit boundary waits for a load.
+            // Next non-empty unit after u.  Its block count `n` is already loaded (`ahead`); the
+            // count after that is requested now, so no unit boundary waits for a load.
             auto next_unit = [&](uint32_t u, int &n, int &ahead) {
                 do {
                     u += gridDim.x;
@@ -327,93 +317,70 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 } while (u < (uint32_t)a.n_units && n <= 0);
                 return u;
             };
-            // S of the first two steps of a unit, for one slot.  Steps are numbered through the
-            // CTA's whole run (kc0 = number of the unit's first step), so the buffer and ring
-            // arithmetic does not care about unit boundaries.
-            auto issue_head = [&](int s, uint32_t kc0, int n) {
-                for (int t0 = 0; t0 < 2 && t0 < n; ++t0) {
-                    const uint32_t c0 = kc0 + t0;
-                    issue_qk(s, c0 & 1, c0 % kKStages);
-                    ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c0 & 1)));
-                    if (s == 1) ptx::umma_commit(bar(BAR_K_EMPTY + c0 % kKStages));
-                }
-                if (s == 1 && n <= 2) ptx::umma_commit(bar(BAR_Q_EMPTY));
-            };
-            // Q of unit number ul and the K blocks of its first two steps have landed.
-            auto wait_head = [&](uint32_t ul, uint32_t kc0, int n) {
-                bool ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 4));
-                for (int t0 = 0; t0 < 2 && t0 < n && ok; ++t0) {
-                    const uint32_t c0 = kc0 + t0;
-                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + c0 % kKStages), (c0 / kKStages) & 1,
+            bool ok = true;
+            // S(c1) for both slots; `first` / `final`: c1 is the first / last step of unit number ul1.
+            auto qk_step = [&](uint32_t c1, uint32_t ul1, bool first, bool final, bool wait_taken) {
+                if (first) ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul1 & 1, abort_flag, a.status, 4));
+                if (ok)
+                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + c1 % kKStages), (c1 / kKStages) & 1,
                                                           abort_flag, a.status, 5));
+                for (int s = 0; s < 2 && ok; ++s) {
+                    if (wait_taken) {
+                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_S_TAKEN + s), (c1 - 1) & 1, abort_flag, a.status, 8));
+                        if (!ok) break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    if (leader) {
+                        issue_qk(s, c1 % kKStages);
+                        ptx::umma_commit(bar(BAR_S_FULL + s));
+                        if (s == 1) {
+                            ptx::umma_commit(bar(BAR_K_EMPTY + c1 % kKStages));
+                            if (final) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                        }
+                    }
+                    __syncwarp();
                 }
-                ptx::tc_fence_after_sync();
-                return ok;
+            };
+            // O (+)= P(c) V(c) for both slots; t = step inside its unit (number ul) of n steps.
+            auto pv_step = [&](uint32_t c, uint32_t ul, int t, int n) {
+                ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_V_FULL + c % kVStages), (c / kVStages) & 1,
+                                                      abort_flag, a.status, 6));
+                for (int s = 0; s < 2 && ok; ++s) {
+                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + 2 * s + (c & 1)), (c >> 1) & 1, abort_flag, a.status, 7));
+                    if (!ok) break;
+                    if (t == 0 && ul > 0) {
+                        // The previous unit's O must have left tensor memory.
+                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_O_FREE + s), (ul - 1) & 1, abort_flag, a.status, 14));
+                        if (!ok) break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    if (leader) {
+                        issue_pv(s, c & 1, c % kVStages, t > 0);
+                        ptx::umma_commit(bar(BAR_O_DONE + 2 * s + (c & 1)));
+                        if (t + 1 == n) ptx::umma_commit(bar(BAR_O_FINAL + s));
+                        if (s == 1) ptx::umma_commit(bar(BAR_V_EMPTY + c % kVStages));
+                    }
+                    __syncwarp();
+                }
             };
             uint32_t kc = 0, ul = 0;
-            bool ok = true;
             int n = 0, nn = 0;  // key blocks of this unit and of the next
             int ahead = unit_blocks(blockIdx.x);
             uint32_t u = next_unit(blockIdx.x - gridDim.x, n, ahead);  // (the sum wraps back to blockIdx.x)
-            if (u < (uint32_t)a.n_units) {
-                ok = wait_head(0, 0, n);
-                if (ok && leader) {
-                    issue_head(0, 0, n);
-                    issue_head(1, 0, n);
-                }
-                __syncwarp();
-            }
+            if (u < (uint32_t)a.n_units) qk_step(0, 0, true, n == 1, false);
             while (u < (uint32_t)a.n_units && ok) {
-                // The next unit's coordinates are fetched now and used at this unit's last step,
-                // where the S of its first two steps is issued right behind each slot's last P V:
-                // the softmax warps then find their next logits ready while the epilogue warps
-                // are still writing this unit's O.
                 const uint32_t un = next_unit(u, nn, ahead);
                 const bool has_next = un < (uint32_t)a.n_units;
                 for (int t = 0; t < n && ok; ++t) {
                     const uint32_t c = kc + t;
-                    const bool last = t + 1 == n;
-                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_V_FULL + c % kVStages), (c / kVStages) & 1,
-                                                          abort_flag, a.status, 6));
-                    if (!ok) break;
-                    if (t + 2 < n) {
-                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + (c + 2) % kKStages),
-                                                              ((c + 2) / kKStages) & 1, abort_flag, a.status, 8));
-                        if (!ok) break;
-                    }
-                    for (int s = 0; s < 2; ++s) {
-                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + 2 * s + (c & 1)), (c >> 1) & 1, abort_flag, a.status, 7));
-                        if (!ok) break;
-                        ptx::tc_fence_after_sync();
-                        if (t == 0 && ul > 0) {
-                            // The previous unit's O must have left tensor memory.
-                            ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_O_FREE + s), (ul - 1) & 1, abort_flag, a.status, 14));
-                            if (!ok) break;
-                            ptx::tc_fence_after_sync();
-                        }
-                        if (leader) {
-                            issue_pv(s, c & 1, c % kVStages, t > 0);
-                            ptx::umma_commit(bar(BAR_O_DONE + 2 * s + (c & 1)));
-                            if (last) ptx::umma_commit(bar(BAR_O_FINAL + s));
-                            if (s == 1) ptx::umma_commit(bar(BAR_V_EMPTY + c % kVStages));
-                            if (t + 2 < n) {
-                                issue_qk(s, c & 1, (c + 2) % kKStages);
-                                ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c & 1)));
-                                if (s == 1) {
-                                    ptx::umma_commit(bar(BAR_K_EMPTY + (c + 2) % kKStages));
-                                    if (t + 3 == n) ptx::umma_commit(bar(BAR_Q_EMPTY));
-                                }
-                            }
-                        }
-                        __syncwarp();
-                        if (last && has_next) {
-                            if (s == 0) {
-                                ok = wait_head(ul + 1, kc + n, nn);
-                                if (!ok) break;
-                            }
-                            if (leader) issue_head(s, kc + n, nn);
-                            __syncwarp();
-                        }
+                    if (t + 1 < n) {
+                        qk_step(c + 1, ul, false, t + 2 == n, true);
+                        if (ok) pv_step(c, ul, t, n);
+                    } else {
+                        // Unit boundary: this unit's last P V first (the epilogue waits for it), then
+                        // the next unit's first S, whose Q tile may still be on its way.
+                        pv_step(c, ul, t, n);
+                        if (ok && has_next) qk_step(c + 1, ul + 1, true, nn == 1, true);
                     }
                 }
                 kc += n;
@@ -467,14 +434,17 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             float m = -INFINITY, l = 0.f;
             uint32_t sr[64];
             for (int t = 0; t < w.n; ++t, ++kc) {
-                const uint32_t t_s = t_s0 + (kc & 1) * 64;
-                ok = wait_bar(bar(BAR_S_FULL + 2 * s + (kc & 1)), (kc >> 1) & 1, abort_flag, a.status, 9);
+                ok = wait_bar(bar(BAR_S_FULL + s), kc & 1, abort_flag, a.status, 9);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                ptx::tmem_ld32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
-                ptx::tmem_ld32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+                ptx::tmem_ld32(t_s0, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+                ptx::tmem_ld32(t_s0 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
                 ptx::tmem_wait_ld();
+                // S is in registers: its buffer may take the next step's logits.
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(BAR_S_TAKEN + s));
                 if (last_is_diag && t == w.n - 1) {
 #pragma unroll
                     for (int c = 0; c < 64; ++c)
@@ -563,9 +533,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
                 }
                 l += sum;
-                // P (bf16 pairs) overlays the first 32 columns of the S buffer just read.
-                ptx::tmem_st32(t_s, pk);
-                // (The hand-over barriers alternate by step parity like the S buffers: the S of step
+                if (kc >= 2) {
+                    // P has two buffers (step parity): the P V that read this one two steps ago
+                    // must have completed (normally long ago).
+                    ok = wait_bar(bar(BAR_O_DONE + 2 * s + (kc & 1)), ((kc - 2) >> 1) & 1, abort_flag, a.status, 12);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                }
+                ptx::tmem_st32(t_s0 + 64 + (kc & 1) * 32, pk);
+                // (The hand-over barriers alternate by step parity like the P buffers: the S of step
                 // kc + 2 is issued behind the P V of step kc, so a barrier is never more than one
                 // phase ahead of the issuer, whose parity wait could not tell two from none.)
                 ptx::tmem_wait_st();
