@@ -34,6 +34,13 @@
 // A warpgroup asking for more than the pool holds would wait for ever.
 static_assert(4 * PA_REG_CTRL + 8 * PA_REG_SOFT + 4 * PA_REG_EPI <= 16 * 128, "register split exceeds the CTA's registers");
 static_assert(PA_REG_CTRL % 8 == 0 && PA_REG_SOFT % 8 == 0 && PA_REG_EPI % 8 == 0, "setmaxnreg takes multiples of 8");
+#ifndef PA_PHASE_DELAY
+#define PA_PHASE_DELAY 0
+#endif
+#ifndef PA_K_STAGES
+#define PA_K_STAGES 2
+#define PA_V_STAGES 2
+#endif
 #ifndef PA_WAIT_HINT_NS
 #define PA_WAIT_HINT_NS 0
 #endif
@@ -42,8 +49,8 @@ namespace pa {
 
 constexpr int kBlk = 64;               // tokens per query / key block
 constexpr int kThreads = 512;          // 16 warps: control, two softmax warpgroups, epilogue
-constexpr int kKStages = 4;            // K block ring depth
-constexpr int kVStages = 4;            // V block ring depth
+constexpr int kKStages = PA_K_STAGES;  // K block ring depth
+constexpr int kVStages = PA_V_STAGES;  // V block ring depth
 constexpr uint32_t kTmemCols = 512;    // slot s: S/P buffers at columns 128 s + 64 b, O at 256 + s D
 // A step's row sum above this limit sends the step through the exact path (new reference).
 constexpr float kSumLimit = 1048576.0f;  // 2^20
@@ -68,7 +75,8 @@ struct SmemMap {
     static constexpr uint32_t kQ = 0;
     static constexpr uint32_t kBlkSub = 64 * 128;             // 64 keys x 64 features
     static constexpr uint32_t kBlkTile = kBlkSub * (D / 64);  // one K or V block
-    static constexpr uint32_t kK = kQ + 2 * kQSlot;
+    static constexpr uint32_t kQBuf = 2 * kQSlot;             // both slots' Q tiles of one unit
+    static constexpr uint32_t kK = kQ + 2 * kQBuf;            // two units' worth: the next unit's Q loads early
     static constexpr uint32_t kV = kK + kKStages * kBlkTile;
     static constexpr uint32_t kOStage = kV + kVStages * kBlkTile;  // one slot's O tile on its way out
     static constexpr uint32_t kOStageBytes = 128 * D * 2;
@@ -81,7 +89,8 @@ struct SmemMap {
 
 // Barrier slots inside the barrier area (8 bytes each).
 enum : uint32_t {
-    BAR_Q_FULL = 0, BAR_Q_EMPTY = 1, BAR_K_FULL = 2, BAR_K_EMPTY = BAR_K_FULL + kKStages,
+    BAR_Q_FULL = 0, BAR_Q_EMPTY = 2,  // [unit parity]
+    BAR_K_FULL = 4, BAR_K_EMPTY = BAR_K_FULL + kKStages,
     BAR_V_FULL = BAR_K_EMPTY + kKStages, BAR_V_EMPTY = BAR_V_FULL + kVStages,
     BAR_S_FULL = BAR_V_EMPTY + kVStages,  // [slot]: S of the step is in tensor memory
     BAR_S_TAKEN = BAR_S_FULL + 2,         // [slot]: the softmax warps have S in registers
@@ -158,8 +167,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        ptx::mbar_init(bar(BAR_Q_FULL), 1);
-        ptx::mbar_init(bar(BAR_Q_EMPTY), 1);
+        for (int s = 0; s < 2; ++s) {
+            ptx::mbar_init(bar(BAR_Q_FULL + s), 1);
+            ptx::mbar_init(bar(BAR_Q_EMPTY + s), 1);
+        }
         for (int s = 0; s < kKStages; ++s) {
             ptx::mbar_init(bar(BAR_K_FULL + s), 1);
             ptx::mbar_init(bar(BAR_K_EMPTY + s), 1);
@@ -215,18 +226,25 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 }
                 return u;
             };
-            Unit w;
-            int32_t j = 0;
-            uint32_t u = next_unit(blockIdx.x, w, j);
-            while (u < (uint32_t)a.n_units && ok) {
-                if (ul > 0) ok = wait_bar(bar(BAR_Q_EMPTY), (ul - 1) & 1, abort_flag, a.status, 1);
-                if (!ok) break;
-                ptx::mbar_expect_tx(bar(BAR_Q_FULL), 2 * SM::kQSlot);
+            // Q tiles of unit number ul_q go to Q buffer ul_q & 1 once the unit two before has
+            // issued its last S.
+            auto load_q = [&](const Unit &w, uint32_t ul_q) {
+                const uint32_t qb = ul_q & 1;
+                if (ul_q >= 2 && !wait_bar(bar(BAR_Q_EMPTY + qb), ((ul_q >> 1) - 1) & 1, abort_flag, a.status, 1)) return false;
+                ptx::mbar_expect_tx(bar(BAR_Q_FULL + qb), SM::kQBuf);
                 for (int s = 0; s < 2; ++s)
                     for (int dh = 0; dh < DH; ++dh)
-                        ptx::tma_load_4d(smem_base + SM::kQ + s * SM::kQSlot + dh * SM::kQSub, &tmQ,
-                                         bar(BAR_Q_FULL), dh * 64, w.i * kBlk,
+                        ptx::tma_load_4d(smem_base + SM::kQ + qb * SM::kQBuf + s * SM::kQSlot + dh * SM::kQSub, &tmQ,
+                                         bar(BAR_Q_FULL + qb), dh * 64, w.i * kBlk,
                                          w.hk * a.G + w.sub * 4 + 2 * s, w.b);
+                return true;
+            };
+            Unit w, wn;
+            int32_t j = 0, jnext = 0;
+            uint32_t u = next_unit(blockIdx.x, w, j);
+            if (u < (uint32_t)a.n_units) ok = load_q(w, 0);
+            while (u < (uint32_t)a.n_units && ok) {
+                const uint32_t un = next_unit(u + gridDim.x, wn, jnext);
                 for (int t = 0; t < w.n; ++t, ++kc) {
                     const int32_t jn = t + 1 < w.n ? __ldg(a.col_idx + w.rs + t + 1) : 0;
                     const uint32_t ks = kc % kKStages, vs = kc % kVStages;
@@ -247,9 +265,18 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         ptx::tma_load_4d(smem_base + SM::kV + vs * SM::kBlkTile + dh * SM::kBlkSub, &tmV,
                                          bar(BAR_V_FULL + vs), dh * 64, j * kBlk, w.hk, w.b);
                     j = jn;
+                    // The next unit's Q behind this unit's second block: by then the unit before
+                    // this one has issued its last S (its K stage was just reused), so the Q
+                    // buffer is free and the load has the whole unit to arrive.
+                    if (t == (w.n > 1 ? 1 : 0) && un < (uint32_t)a.n_units) {
+                        ok = load_q(wn, ul + 1);
+                        if (!ok) break;
+                    }
                 }
                 ++ul;
-                u = next_unit(u + gridDim.x, w, j);
+                u = un;
+                w = wn;
+                j = jnext;
             }
             if (!ok) {
                 // Drain: give copies already in flight a bounded chance to land before exit.
@@ -279,12 +306,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             constexpr uint32_t idesc_qk = ptx::idesc_bf16_f32(128, 64, 0);
             constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(128, D, 1);
             constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-            const uint32_t q_lo = ((smem_base + SM::kQ) >> 4) | (1u << 16);
+            const uint32_t q_lo = ((smem_base + SM::kQ) >> 4) | (1u << 16);  // + unit parity, slot
             const uint32_t k_lo = ((smem_base + SM::kK) >> 4) | (1u << 16);
             const uint32_t v_lo = ((smem_base + SM::kV) >> 4) | ((SM::kBlkSub >> 4) << 16);
             // S = Q K^T: A = Q tile (K-major), B = K block (K-major), 16 features per MMA.
-            auto issue_qk = [&](int s, uint32_t ks) {
-                const uint32_t qa = q_lo + s * (SM::kQSlot >> 4);
+            auto issue_qk = [&](int s, uint32_t qb, uint32_t ks) {
+                const uint32_t qa = q_lo + qb * (SM::kQBuf >> 4) + s * (SM::kQSlot >> 4);
                 const uint32_t kb = k_lo + ks * (SM::kBlkTile >> 4);
                 const uint32_t dst = tmem_base + s * 128;
 #pragma unroll
@@ -320,7 +347,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             bool ok = true;
             // S(c1) for both slots; `first` / `final`: c1 is the first / last step of unit number ul1.
             auto qk_step = [&](uint32_t c1, uint32_t ul1, bool first, bool final, bool wait_taken) {
-                if (first) ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul1 & 1, abort_flag, a.status, 4));
+                if (first) ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL + (ul1 & 1)), (ul1 >> 1) & 1, abort_flag, a.status, 4));
                 if (ok)
                     ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + c1 % kKStages), (c1 / kKStages) & 1,
                                                           abort_flag, a.status, 5));
@@ -331,11 +358,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     }
                     ptx::tc_fence_after_sync();
                     if (leader) {
-                        issue_qk(s, c1 % kKStages);
+                        issue_qk(s, ul1 & 1, c1 % kKStages);
                         ptx::umma_commit(bar(BAR_S_FULL + s));
                         if (s == 1) {
                             ptx::umma_commit(bar(BAR_K_EMPTY + c1 % kKStages));
-                            if (final) ptx::umma_commit(bar(BAR_Q_EMPTY));
+                            if (final) ptx::umma_commit(bar(BAR_Q_EMPTY + (ul1 & 1)));
                         }
                     }
                     __syncwarp();
@@ -377,10 +404,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         qk_step(c + 1, ul, false, t + 2 == n, true);
                         if (ok) pv_step(c, ul, t, n);
                     } else {
-                        // Unit boundary: this unit's last P V first (the epilogue waits for it), then
-                        // the next unit's first S, whose Q tile may still be on its way.
-                        pv_step(c, ul, t, n);
-                        if (ok && has_next) qk_step(c + 1, ul + 1, true, nn == 1, true);
+                        // Unit boundary: the next unit's first S goes first if its Q tile has
+                        // arrived (normally long ago), else behind this unit's last P V, for which
+                        // the epilogue waits.
+                        const bool q_here = has_next && __all_sync(0xffffffffu, ptx::mbar_test_wait(bar(BAR_Q_FULL + ((ul + 1) & 1)), ((ul + 1) >> 1) & 1));
+                        if (q_here) qk_step(c + 1, ul + 1, true, nn == 1, true);
+                        if (ok) pv_step(c, ul, t, n);
+                        if (ok && has_next && !q_here) qk_step(c + 1, ul + 1, true, nn == 1, true);
                     }
                 }
                 kc += n;
@@ -437,6 +467,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 ok = wait_bar(bar(BAR_S_FULL + s), kc & 1, abort_flag, a.status, 9);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+#if PA_PHASE_DELAY > 0
+                if (s == 1 && kc == 0) {
+                    const long long t0 = clock64();
+                    while (clock64() - t0 < PA_PHASE_DELAY) {
+                    }
+                }
+#endif
                 ptx::tc_fence_after_sync();
                 ptx::tmem_ld32(t_s0, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
                 ptx::tmem_ld32(t_s0 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
