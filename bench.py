@@ -49,6 +49,33 @@ def read_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
+# DRAM bytes moved by one prefill_kernel<128> launch on the 128K workload: dram__bytes_read.sum +
+# dram__bytes_write.sum of an ncu capture of this very workload (the command is in
+# profiles/prefill_kernel_128k_traffic.md).  The figure belongs to the kernel sources it was taken
+# on: once they change it is reported as null until the capture is repeated.
+PREFILL_TRAFFIC = dict(
+    bytes=2039873792 + 915694848,
+    sources={
+        "prefill_sm100.cu": "9de8f57e2430b2724748271b404bd246543b3ee94d8e836259538296bcb2d6c6",
+        "sm100_ptx.cuh": "cc5cb63f8da5e88ddc941ca016a41fe337c2404ca754e7ea5c384e0a1552a5ca",
+    },
+)
+
+
+def prefill_traffic():
+    import hashlib
+
+    csrc = os.path.join(ROOT, "paper_2503_03588_b200", "csrc")
+    for name, digest in PREFILL_TRAFFIC["sources"].items():
+        try:
+            with open(os.path.join(csrc, name), "rb") as f:
+                if hashlib.sha256(f.read()).hexdigest() != digest:
+                    return None
+        except OSError:
+            return None
+    return PREFILL_TRAFFIC["bytes"]
+
+
 # ------------------------------------------------------------------------------ multi-rank glue
 
 def dist_env():
@@ -351,7 +378,7 @@ def run_ours(args):
                             parallelism="replicas" if world > 1 else "single"),
                 clocks=clocks,
                 roofline=dict(bound="tensor", achieved=achieved, peak=peaks["bf16_tflops"], unit="TFLOP/s",
-                              frac=achieved / peaks["bf16_tflops"], traffic=None,
+                              frac=achieved / peaks["bf16_tflops"], traffic=prefill_traffic(),
                               peak_source=peaks["source"] + " burst bf16", kernel="prefill_kernel<128>",
                               kernel_ms=prefill_ms,
                               frac_of_sustained=achieved / peaks["bf16_tflops_sustained"]),
