@@ -9,13 +9,11 @@
 //               block index, into two rings of shared-memory tiles (128-byte swizzle)
 //   warp 1      tcgen05 issuer: S = Q K^T into tensor memory (two S buffers per slot, so the
 //               logits of step t+1 are ready while the softmax works on step t); O += P V with
-//               P read from tensor memory (it overlays the S buffer it was computed from); the
-//               next unit's first two S are issued right behind a slot's last P V
+//               P read from tensor memory (it overlays the S buffer it was computed from)
 //   warp 2      tensor-memory allocation
-//   warps 4-7   online softmax of slot 0 (thread = tile row = TMEM lane), LSE
+//   warps 4-7   online softmax of slot 0 (thread = tile row = TMEM lane)
 //   warps 8-11  online softmax of slot 1
-//   warps 12-15 epilogue: O / l out of tensor memory, staged in shared memory, bulk tensor
-//               stores to global memory; runs beside the next unit's first steps
+//   warps 12-15 epilogue: O / l and LSE out of tensor memory to global memory
 // Warps 0-3 and 12-15 give registers back (setmaxnreg) and the softmax warpgroups take them.
 // Every barrier wait is bounded; a wait that runs out records PA_ERR_TIMEOUT in the status
 // block, raises a CTA-wide abort flag and the CTA drains and exits (no trap, no endless spin).
@@ -29,20 +27,30 @@
 // Registers per thread by role: 4 control warps, 8 softmax warps, 4 epilogue warps share the
 // CTA's 16 x 128.
 #ifndef PA_REG_CTRL
-#define PA_REG_CTRL 48
-#define PA_REG_SOFT 176
-#define PA_REG_EPI 112
+#define PA_REG_CTRL 56
+#define PA_REG_SOFT 168
+#define PA_REG_EPI 120
 #endif
 // A warpgroup asking for more than the pool holds would wait for ever.
 static_assert(4 * PA_REG_CTRL + 8 * PA_REG_SOFT + 4 * PA_REG_EPI <= 16 * 128, "register split exceeds the CTA's registers");
 static_assert(PA_REG_CTRL % 8 == 0 && PA_REG_SOFT % 8 == 0 && PA_REG_EPI % 8 == 0, "setmaxnreg takes multiples of 8");
+#ifndef PA_PHASE_DELAY
+#define PA_PHASE_DELAY 0
+#endif
+#ifndef PA_K_STAGES
+#define PA_K_STAGES 3
+#define PA_V_STAGES 2
+#endif
+#ifndef PA_WAIT_HINT_NS
+#define PA_WAIT_HINT_NS 0
+#endif
 
 namespace pa {
 
 constexpr int kBlk = 64;               // tokens per query / key block
 constexpr int kThreads = 512;          // 16 warps: control, two softmax warpgroups, epilogue
-constexpr int kKStages = 4;            // K block ring depth
-constexpr int kVStages = 4;            // V block ring depth
+constexpr int kKStages = PA_K_STAGES;  // K block ring depth
+constexpr int kVStages = PA_V_STAGES;  // V block ring depth
 constexpr uint32_t kTmemCols = 512;    // slot s: S/P buffers at columns 128 s + 64 b, O at 256 + s D
 // A step's row sum above this limit sends the step through the exact path (new reference).
 constexpr float kSumLimit = 1048576.0f;  // 2^20
@@ -67,10 +75,11 @@ struct SmemMap {
     static constexpr uint32_t kQ = 0;
     static constexpr uint32_t kBlkSub = 64 * 128;             // 64 keys x 64 features
     static constexpr uint32_t kBlkTile = kBlkSub * (D / 64);  // one K or V block
-    static constexpr uint32_t kK = kQ + 2 * kQSlot;
+    static constexpr uint32_t kQBuf = 2 * kQSlot;             // both slots' Q tiles of one unit
+    static constexpr uint32_t kK = kQ + 2 * kQBuf;            // two units' worth: the next unit's Q loads early
     static constexpr uint32_t kV = kK + kKStages * kBlkTile;
-    static constexpr uint32_t kOStage = kV + kVStages * kBlkTile;  // one slot's O tile on its way out
-    static constexpr uint32_t kOStageBytes = 128 * D * 2;
+    static constexpr uint32_t kOStage = kV + kVStages * kBlkTile;  // one head's O rows on their way out
+    static constexpr uint32_t kOStageBytes = 64 * D * 2;      // one head x 64 tokens
     static constexpr uint32_t kStats = kOStage + kOStageBytes;    // [slot][row] softmax denominators
     static constexpr uint32_t kBars = kStats + 2 * 128 * 4;
     static constexpr uint32_t kTotal = kBars + 512;
@@ -80,10 +89,12 @@ struct SmemMap {
 
 // Barrier slots inside the barrier area (8 bytes each).
 enum : uint32_t {
-    BAR_Q_FULL = 0, BAR_Q_EMPTY = 1, BAR_K_FULL = 2, BAR_K_EMPTY = BAR_K_FULL + kKStages,
+    BAR_Q_FULL = 0, BAR_Q_EMPTY = 2,  // [unit parity]
+    BAR_K_FULL = 4, BAR_K_EMPTY = BAR_K_FULL + kKStages,
     BAR_V_FULL = BAR_K_EMPTY + kKStages, BAR_V_EMPTY = BAR_V_FULL + kVStages,
-    BAR_S_FULL = BAR_V_EMPTY + kVStages,  // [slot][buffer]
-    BAR_P_FULL = BAR_S_FULL + 4,  // [slot][step parity]: P of that step is in tensor memory
+    BAR_S_FULL = BAR_V_EMPTY + kVStages,  // [slot]: S of the step is in tensor memory
+    BAR_S_TAKEN = BAR_S_FULL + 2,         // [slot]: the softmax warps have S in registers
+    BAR_P_FULL = BAR_S_TAKEN + 2,  // [slot][step parity]: P of that step is in tensor memory
     BAR_O_DONE = BAR_P_FULL + 4,  // [slot][step parity]: P V of that step has completed
     BAR_O_FINAL = BAR_O_DONE + 4,   // [slot]: the unit's last P V has completed
     BAR_ML_READY = BAR_O_FINAL + 2,  // [slot]: the unit's row statistics are in shared memory
@@ -121,7 +132,11 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     const long long t0 = clock64();
     uint32_t it = 0;
     while (true) {
+#if PA_WAIT_HINT_NS > 0
+        if (ptx::mbar_try_wait_hint(bar, parity, PA_WAIT_HINT_NS)) return true;
+#else
         if (ptx::mbar_try_wait(bar, parity)) return true;
+#endif
         if ((++it & 63u) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitCycles) break;
@@ -152,8 +167,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        ptx::mbar_init(bar(BAR_Q_FULL), 1);
-        ptx::mbar_init(bar(BAR_Q_EMPTY), 1);
+        for (int s = 0; s < 2; ++s) {
+            ptx::mbar_init(bar(BAR_Q_FULL + s), 1);
+            ptx::mbar_init(bar(BAR_Q_EMPTY + s), 1);
+        }
         for (int s = 0; s < kKStages; ++s) {
             ptx::mbar_init(bar(BAR_K_FULL + s), 1);
             ptx::mbar_init(bar(BAR_K_EMPTY + s), 1);
@@ -162,12 +179,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::mbar_init(bar(BAR_V_FULL + s), 1);
             ptx::mbar_init(bar(BAR_V_EMPTY + s), 1);
         }
-        for (int s = 0; s < 4; ++s) {
-            ptx::mbar_init(bar(BAR_S_FULL + s), 1);
-            ptx::mbar_init(bar(BAR_O_DONE + s), 1);
-        }
+        for (int s = 0; s < 4; ++s) ptx::mbar_init(bar(BAR_O_DONE + s), 1);
         for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(bar(BAR_P_FULL + 2 * s), 4);  // one arrival per softmax warp of the slot
+            ptx::mbar_init(bar(BAR_S_FULL + s), 1);
+            ptx::mbar_init(bar(BAR_S_TAKEN + s), 4);  // one arrival per softmax warp of the slot
+            ptx::mbar_init(bar(BAR_P_FULL + 2 * s), 4);
             ptx::mbar_init(bar(BAR_P_FULL + 2 * s + 1), 4);
             ptx::mbar_init(bar(BAR_O_FINAL + s), 1);
             ptx::mbar_init(bar(BAR_ML_READY + s), 4);
@@ -210,18 +226,25 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 }
                 return u;
             };
-            Unit w;
-            int32_t j = 0;
-            uint32_t u = next_unit(blockIdx.x, w, j);
-            while (u < (uint32_t)a.n_units && ok) {
-                if (ul > 0) ok = wait_bar(bar(BAR_Q_EMPTY), (ul - 1) & 1, abort_flag, a.status, 1);
-                if (!ok) break;
-                ptx::mbar_expect_tx(bar(BAR_Q_FULL), 2 * SM::kQSlot);
+            // Q tiles of unit number ul_q go to Q buffer ul_q & 1 once the unit two before has
+            // issued its last S.
+            auto load_q = [&](const Unit &w, uint32_t ul_q) {
+                const uint32_t qb = ul_q & 1;
+                if (ul_q >= 2 && !wait_bar(bar(BAR_Q_EMPTY + qb), ((ul_q >> 1) - 1) & 1, abort_flag, a.status, 1)) return false;
+                ptx::mbar_expect_tx(bar(BAR_Q_FULL + qb), SM::kQBuf);
                 for (int s = 0; s < 2; ++s)
                     for (int dh = 0; dh < DH; ++dh)
-                        ptx::tma_load_4d(smem_base + SM::kQ + s * SM::kQSlot + dh * SM::kQSub, &tmQ,
-                                         bar(BAR_Q_FULL), dh * 64, w.i * kBlk,
+                        ptx::tma_load_4d(smem_base + SM::kQ + qb * SM::kQBuf + s * SM::kQSlot + dh * SM::kQSub, &tmQ,
+                                         bar(BAR_Q_FULL + qb), dh * 64, w.i * kBlk,
                                          w.hk * a.G + w.sub * 4 + 2 * s, w.b);
+                return true;
+            };
+            Unit w, wn;
+            int32_t j = 0, jnext = 0;
+            uint32_t u = next_unit(blockIdx.x, w, j);
+            if (u < (uint32_t)a.n_units) ok = load_q(w, 0);
+            while (u < (uint32_t)a.n_units && ok) {
+                const uint32_t un = next_unit(u + gridDim.x, wn, jnext);
                 for (int t = 0; t < w.n; ++t, ++kc) {
                     const int32_t jn = t + 1 < w.n ? __ldg(a.col_idx + w.rs + t + 1) : 0;
                     const uint32_t ks = kc % kKStages, vs = kc % kVStages;
@@ -242,9 +265,18 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         ptx::tma_load_4d(smem_base + SM::kV + vs * SM::kBlkTile + dh * SM::kBlkSub, &tmV,
                                          bar(BAR_V_FULL + vs), dh * 64, j * kBlk, w.hk, w.b);
                     j = jn;
+                    // The next unit's Q behind this unit's second block: by then the unit before
+                    // this one has issued its last S (its K stage was just reused), so the Q
+                    // buffer is free and the load has the whole unit to arrive.
+                    if (t == (w.n > 1 ? 1 : 0) && un < (uint32_t)a.n_units) {
+                        ok = load_q(wn, ul + 1);
+                        if (!ok) break;
+                    }
                 }
                 ++ul;
-                u = next_unit(u + gridDim.x, w, j);
+                u = un;
+                w = wn;
+                j = jnext;
             }
             if (!ok) {
                 // Drain: give copies already in flight a bounded chance to land before exit.
@@ -257,51 +289,53 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     } else if (warp == 1) {
         // ------------------------------------------------------------------ tcgen05 issuer
         // The whole warp runs the (uniform) control flow and the barrier waits; one elected lane
-        // issues the MMAs and commits.  MMAs of one issuer execute in issue order, which is what
-        // lets the S of step t+2 overwrite the buffer whose P was read by the P V of step t.
+        // issues the MMAs and commits.  Steps are numbered through the CTA's whole run (c), so ring
+        // positions and buffer parities do not care about unit boundaries.  Per step c and slot:
+        //   S(c + 1) = Q K^T is issued as soon as the softmax warps have taken S(c) out of tensor
+        //   memory (S has one buffer per slot; P has its own two), i.e. while they still work on
+        //   step c, and it may belong to the next unit;
+        //   O += P(c) V(c) is issued when P(c) has been handed over.
         // Descriptors: the high word is constant per operand kind (stride 1024 B between 8-row
         // groups, version 1, 128-byte swizzle); the low word holds the start address >> 4 (plus
         // the leading-dimension offset for the MN-major V operand).
         {
             const bool leader = ptx::elect_one();
-            // Every lane holds the same values; the shuffles (here and in unit_blocks) tell the
-            // compiler so, which lets loop bounds, ring positions and descriptors live in uniform
-            // registers: the issue loop is short enough that this shows in the kernel's time.
+            // Every lane holds the same values; the shuffles tell the compiler so, which lets the
+            // loop bounds, ring positions and descriptors live in uniform registers.
             const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_any, 0);
             constexpr uint32_t idesc_qk = ptx::idesc_bf16_f32(128, 64, 0);
             constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(128, D, 1);
             constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-            const uint32_t q_lo = ((smem_base + SM::kQ) >> 4) | (1u << 16);
+            const uint32_t q_lo = ((smem_base + SM::kQ) >> 4) | (1u << 16);  // + unit parity, slot
             const uint32_t k_lo = ((smem_base + SM::kK) >> 4) | (1u << 16);
             const uint32_t v_lo = ((smem_base + SM::kV) >> 4) | ((SM::kBlkSub >> 4) << 16);
             // S = Q K^T: A = Q tile (K-major), B = K block (K-major), 16 features per MMA.
-            auto issue_qk = [&](int s, uint32_t buf, uint32_t ks) {
-                const uint32_t qa = q_lo + s * (SM::kQSlot >> 4);
+            auto issue_qk = [&](int s, uint32_t qb, uint32_t ks) {
+                const uint32_t qa = q_lo + qb * (SM::kQBuf >> 4) + s * (SM::kQSlot >> 4);
                 const uint32_t kb = k_lo + ks * (SM::kBlkTile >> 4);
-                const uint32_t dst = tmem_base + s * 128 + buf * 64;
+                const uint32_t dst = tmem_base + s * 128;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk)
                     ptx::umma_ss_lohi(dst, qa + (((kk / 4) * SM::kQSub + (kk % 4) * 32) >> 4), desc_hi,
                                       kb + (((kk / 4) * SM::kBlkSub + (kk % 4) * 32) >> 4), desc_hi, idesc_qk,
                                       kk > 0 ? 1u : 0u);
             };
-            // O (+)= P V: A = P (tensor memory: bf16 pairs in the first 32 columns of the S buffer),
-            // B = V block (MN-major: features contiguous), 16 keys per MMA.
+            // O (+)= P V: A = P (tensor memory, bf16 pairs, buffer = step parity), B = V block
+            // (MN-major: features contiguous), 16 keys per MMA.
             auto issue_pv = [&](int s, uint32_t buf, uint32_t vs, bool acc) {
                 const uint32_t vb = v_lo + vs * (SM::kBlkTile >> 4);
                 const uint32_t dst = tmem_base + 256 + s * D;
-                const uint32_t pa_ = tmem_base + s * 128 + buf * 64;
+                const uint32_t pa_ = tmem_base + s * 128 + 64 + buf * 32;
 #pragma unroll
                 for (int kk = 0; kk < kBlk / 16; ++kk)
                     ptx::umma_ts_lohi(dst, pa_ + kk * 8, vb + ((kk * 2048) >> 4), desc_hi, idesc_pv,
                                       (acc || kk > 0) ? 1u : 0u);
             };
-            // First non-empty unit at or after u (stride: the grid), or n_units.
             auto unit_blocks = [&](uint32_t u) {
                 return __shfl_sync(0xffffffffu, u < (uint32_t)a.n_units ? decode_unit(a, u).n : 0, 0);
             };
-            // Block count `n` of the candidate after u is already loaded (`ahead`); the count
-            // after that is requested now, so no unit boundary waits for a load.
+            // Next non-empty unit after u.  Its block count `n` is already loaded (`ahead`); the
+            // count after that is requested now, so no unit boundary waits for a load.
             auto next_unit = [&](uint32_t u, int &n, int &ahead) {
                 do {
                     u += gridDim.x;
@@ -310,93 +344,73 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 } while (u < (uint32_t)a.n_units && n <= 0);
                 return u;
             };
-            // S of the first two steps of a unit, for one slot.  Steps are numbered through the
-            // CTA's whole run (kc0 = number of the unit's first step), so the buffer and ring
-            // arithmetic does not care about unit boundaries.
-            auto issue_head = [&](int s, uint32_t kc0, int n) {
-                for (int t0 = 0; t0 < 2 && t0 < n; ++t0) {
-                    const uint32_t c0 = kc0 + t0;
-                    issue_qk(s, c0 & 1, c0 % kKStages);
-                    ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c0 & 1)));
-                    if (s == 1) ptx::umma_commit(bar(BAR_K_EMPTY + c0 % kKStages));
-                }
-                if (s == 1 && n <= 2) ptx::umma_commit(bar(BAR_Q_EMPTY));
-            };
-            // Q of unit number ul and the K blocks of its first two steps have landed.
-            auto wait_head = [&](uint32_t ul, uint32_t kc0, int n) {
-                bool ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL), ul & 1, abort_flag, a.status, 4));
-                for (int t0 = 0; t0 < 2 && t0 < n && ok; ++t0) {
-                    const uint32_t c0 = kc0 + t0;
-                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + c0 % kKStages), (c0 / kKStages) & 1,
+            bool ok = true;
+            // S(c1) for both slots; `first` / `final`: c1 is the first / last step of unit number ul1.
+            auto qk_step = [&](uint32_t c1, uint32_t ul1, bool first, bool final, bool wait_taken) {
+                if (first) ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL + (ul1 & 1)), (ul1 >> 1) & 1, abort_flag, a.status, 4));
+                if (ok)
+                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + c1 % kKStages), (c1 / kKStages) & 1,
                                                           abort_flag, a.status, 5));
+                for (int s = 0; s < 2 && ok; ++s) {
+                    if (wait_taken) {
+                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_S_TAKEN + s), (c1 - 1) & 1, abort_flag, a.status, 8));
+                        if (!ok) break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    if (leader) {
+                        issue_qk(s, ul1 & 1, c1 % kKStages);
+                        ptx::umma_commit(bar(BAR_S_FULL + s));
+                        if (s == 1) {
+                            ptx::umma_commit(bar(BAR_K_EMPTY + c1 % kKStages));
+                            if (final) ptx::umma_commit(bar(BAR_Q_EMPTY + (ul1 & 1)));
+                        }
+                    }
+                    __syncwarp();
                 }
-                ptx::tc_fence_after_sync();
-                return ok;
+            };
+            // O (+)= P(c) V(c) for both slots; t = step inside its unit (number ul) of n steps.
+            auto pv_step = [&](uint32_t c, uint32_t ul, int t, int n) {
+                ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_V_FULL + c % kVStages), (c / kVStages) & 1,
+                                                      abort_flag, a.status, 6));
+                for (int s = 0; s < 2 && ok; ++s) {
+                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + 2 * s + (c & 1)), (c >> 1) & 1, abort_flag, a.status, 7));
+                    if (!ok) break;
+                    if (t == 0 && ul > 0) {
+                        // The previous unit's O must have left tensor memory.
+                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_O_FREE + s), (ul - 1) & 1, abort_flag, a.status, 14));
+                        if (!ok) break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    if (leader) {
+                        issue_pv(s, c & 1, c % kVStages, t > 0);
+                        ptx::umma_commit(bar(BAR_O_DONE + 2 * s + (c & 1)));
+                        if (t + 1 == n) ptx::umma_commit(bar(BAR_O_FINAL + s));
+                        if (s == 1) ptx::umma_commit(bar(BAR_V_EMPTY + c % kVStages));
+                    }
+                    __syncwarp();
+                }
             };
             uint32_t kc = 0, ul = 0;
-            bool ok = true;
             int n = 0, nn = 0;  // key blocks of this unit and of the next
             int ahead = unit_blocks(blockIdx.x);
             uint32_t u = next_unit(blockIdx.x - gridDim.x, n, ahead);  // (the sum wraps back to blockIdx.x)
-            if (u < (uint32_t)a.n_units) {
-                ok = wait_head(0, 0, n);
-                if (ok && leader) {
-                    issue_head(0, 0, n);
-                    issue_head(1, 0, n);
-                }
-                __syncwarp();
-            }
+            if (u < (uint32_t)a.n_units) qk_step(0, 0, true, n == 1, false);
             while (u < (uint32_t)a.n_units && ok) {
-                // The next unit's coordinates are fetched now and used at this unit's last step,
-                // where the S of its first two steps is issued right behind each slot's last P V:
-                // the softmax warps then find their next logits ready while the epilogue warps
-                // are still writing this unit's O.
                 const uint32_t un = next_unit(u, nn, ahead);
                 const bool has_next = un < (uint32_t)a.n_units;
                 for (int t = 0; t < n && ok; ++t) {
                     const uint32_t c = kc + t;
-                    const bool last = t + 1 == n;
-                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_V_FULL + c % kVStages), (c / kVStages) & 1,
-                                                          abort_flag, a.status, 6));
-                    if (!ok) break;
-                    if (t + 2 < n) {
-                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + (c + 2) % kKStages),
-                                                              ((c + 2) / kKStages) & 1, abort_flag, a.status, 8));
-                        if (!ok) break;
-                    }
-                    for (int s = 0; s < 2; ++s) {
-                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + 2 * s + (c & 1)), (c >> 1) & 1, abort_flag, a.status, 7));
-                        if (!ok) break;
-                        ptx::tc_fence_after_sync();
-                        if (t == 0 && ul > 0) {
-                            // The previous unit's O must have left tensor memory.
-                            ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_O_FREE + s), (ul - 1) & 1, abort_flag, a.status, 14));
-                            if (!ok) break;
-                            ptx::tc_fence_after_sync();
-                        }
-                        if (leader) {
-                            issue_pv(s, c & 1, c % kVStages, t > 0);
-                            ptx::umma_commit(bar(BAR_O_DONE + 2 * s + (c & 1)));
-                            if (last) ptx::umma_commit(bar(BAR_O_FINAL + s));
-                            if (s == 1) ptx::umma_commit(bar(BAR_V_EMPTY + c % kVStages));
-                            if (t + 2 < n) {
-                                issue_qk(s, c & 1, (c + 2) % kKStages);
-                                ptx::umma_commit(bar(BAR_S_FULL + 2 * s + (c & 1)));
-                                if (s == 1) {
-                                    ptx::umma_commit(bar(BAR_K_EMPTY + (c + 2) % kKStages));
-                                    if (t + 3 == n) ptx::umma_commit(bar(BAR_Q_EMPTY));
-                                }
-                            }
-                        }
-                        __syncwarp();
-                        if (last && has_next) {
-                            if (s == 0) {
-                                ok = wait_head(ul + 1, kc + n, nn);
-                                if (!ok) break;
-                            }
-                            if (leader) issue_head(s, kc + n, nn);
-                            __syncwarp();
-                        }
+                    if (t + 1 < n) {
+                        qk_step(c + 1, ul, false, t + 2 == n, true);
+                        if (ok) pv_step(c, ul, t, n);
+                    } else {
+                        // Unit boundary: the next unit's first S goes first if its Q tile has
+                        // arrived (normally long ago), else behind this unit's last P V, for which
+                        // the epilogue waits.
+                        const bool q_here = has_next && __all_sync(0xffffffffu, ptx::mbar_test_wait(bar(BAR_Q_FULL + ((ul + 1) & 1)), ((ul + 1) >> 1) & 1));
+                        if (q_here) qk_step(c + 1, ul + 1, true, nn == 1, true);
+                        if (ok) pv_step(c, ul, t, n);
+                        if (ok && has_next && !q_here) qk_step(c + 1, ul + 1, true, nn == 1, true);
                     }
                 }
                 kc += n;
@@ -450,14 +464,24 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             float m = -INFINITY, l = 0.f;
             uint32_t sr[64];
             for (int t = 0; t < w.n; ++t, ++kc) {
-                const uint32_t t_s = t_s0 + (kc & 1) * 64;
-                ok = wait_bar(bar(BAR_S_FULL + 2 * s + (kc & 1)), (kc >> 1) & 1, abort_flag, a.status, 9);
+                ok = wait_bar(bar(BAR_S_FULL + s), kc & 1, abort_flag, a.status, 9);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+#if PA_PHASE_DELAY > 0
+                if (s == 1 && kc == 0) {
+                    const long long t0 = clock64();
+                    while (clock64() - t0 < PA_PHASE_DELAY) {
+                    }
+                }
+#endif
                 ptx::tc_fence_after_sync();
-                ptx::tmem_ld32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
-                ptx::tmem_ld32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+                ptx::tmem_ld32(t_s0, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+                ptx::tmem_ld32(t_s0 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
                 ptx::tmem_wait_ld();
+                // S is in registers: its buffer may take the next step's logits.
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(BAR_S_TAKEN + s));
                 if (last_is_diag && t == w.n - 1) {
 #pragma unroll
                     for (int c = 0; c < 64; ++c)
@@ -546,9 +570,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
                 }
                 l += sum;
-                // P (bf16 pairs) overlays the first 32 columns of the S buffer just read.
-                ptx::tmem_st32(t_s, pk);
-                // (The hand-over barriers alternate by step parity like the S buffers: the S of step
+                if (kc >= 2) {
+                    // P has two buffers (step parity): the P V that read this one two steps ago
+                    // must have completed (normally long ago).
+                    ok = wait_bar(bar(BAR_O_DONE + 2 * s + (kc & 1)), ((kc - 2) >> 1) & 1, abort_flag, a.status, 12);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                }
+                ptx::tmem_st32(t_s0 + 64 + (kc & 1) * 32, pk);
+                // (The hand-over barriers alternate by step parity like the P buffers: the S of step
                 // kc + 2 is issued behind the P V of step kc, so a barrier is never more than one
                 // phase ahead of the issuer, whose parity wait could not tell two from none.)
                 ptx::tmem_wait_st();
@@ -652,40 +682,42 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     ptx::tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(bar(BAR_O_FREE + s));
-                    // The staging tile is free once the previous bulk stores have read it.
-                    if (store_thread) {
-                        ptx::bulk_wait_read_all();
-                        ptx::mbar_arrive(bar(BAR_STAGE_FREE));
-                    }
-                    ok = wait_bar(bar(BAR_STAGE_FREE), ns & 1, abort_flag, a.status, 16);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    // Box (row >> 6, half): 64 tokens x 128 bytes; 16-byte chunk j of token t sits at
-                    // chunk position j ^ (t & 7).
-                    const uint32_t rbase = stage + (uint32_t)(row >> 6) * (uint32_t)(DH * 8192) + (uint32_t)qrow * 128u;
-#pragma unroll
-                    for (int c = 0; c < D / 8; ++c) {
-                        const uint32_t dst = rbase + (uint32_t)(c >> 3) * 8192u + ((uint32_t)((c & 7) ^ (qrow & 7)) << 4);
-                        ptx::st_shared_v4(dst, pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-                    }
-                    ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(bar(BAR_STAGE_FULL));
-                    if (warp == 12) {
-                        ok = wait_bar(bar(BAR_STAGE_FULL), ns & 1, abort_flag, a.status, 17);
+                    // The two heads of the slot go through the staging tile one after the other.
+#pragma unroll 1
+                    for (int hh = 0; hh < 2 && ok; ++hh) {
+                        // The tile is free once the previous bulk stores have read it.
+                        if (store_thread) {
+                            ptx::bulk_wait_read_all();
+                            ptx::mbar_arrive(bar(BAR_STAGE_FREE));
+                        }
+                        ok = wait_bar(bar(BAR_STAGE_FREE), ns & 1, abort_flag, a.status, 16);
                         ok = __all_sync(0xffffffffu, ok);
                         if (!ok) break;
-                    }
-                    ++ns;
-                    if (store_thread) {
-                        for (int hh = 0; hh < 2; ++hh) {
-                            const int hl = w.sub * 4 + 2 * s + hh;
-                            if (hl >= a.G) continue;
-                            for (int dh = 0; dh < DH; ++dh)
-                                ptx::tma_store_4d(&tmO, stage + (uint32_t)(hh * DH + dh) * 8192u, dh * 64, w.i * kBlk,
-                                                  w.hk * a.G + hl, w.b);
+                        if ((row >> 6) == hh) {
+                            // Box (half): 64 tokens x 128 bytes; 16-byte chunk j of token t sits at
+                            // chunk position j ^ (t & 7).
+                            const uint32_t rbase = stage + (uint32_t)qrow * 128u;
+#pragma unroll
+                            for (int c = 0; c < D / 8; ++c) {
+                                const uint32_t dst = rbase + (uint32_t)(c >> 3) * 8192u + ((uint32_t)((c & 7) ^ (qrow & 7)) << 4);
+                                ptx::st_shared_v4(dst, pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                            }
+                            ptx::fence_proxy_async_smem();
                         }
-                        ptx::bulk_commit_group();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(bar(BAR_STAGE_FULL));
+                        if (warp == 12) {
+                            ok = wait_bar(bar(BAR_STAGE_FULL), ns & 1, abort_flag, a.status, 17);
+                            ok = __all_sync(0xffffffffu, ok);
+                            if (!ok) break;
+                        }
+                        ++ns;
+                        const int hl = w.sub * 4 + 2 * s + hh;
+                        if (store_thread && hl < a.G) {
+                            for (int dh = 0; dh < DH; ++dh)
+                                ptx::tma_store_4d(&tmO, stage + (uint32_t)dh * 8192u, dh * 64, w.i * kBlk, w.hk * a.G + hl, w.b);
+                            ptx::bulk_commit_group();
+                        }
                     }
                 }
             }
