@@ -206,12 +206,16 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const uint32_t tmem_base = tmem_base_any;
 
     if (warp < 4) ptx::setmaxnreg_dec<PA_REG_CTRL>();
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+    if (warp == 0 || warp == 3) {
+        // ------------------------------------------------------------------ TMA producers
+        // Two independent streams, each walking the unit list and the key-block lists by itself:
+        // warp 0 fetches the K blocks (needed at the start of a step), warp 3 the V blocks (needed
+        // at its end) and the Q tiles.  Apart, a full V ring or a Q tile in the queue cannot hold
+        // the next K block back.
         if (lane == 0) {
-            ptx::prefetch_tensormap(&tmQ);
-            ptx::prefetch_tensormap(&tmK);
-            ptx::prefetch_tensormap(&tmV);
+            const bool v_side = warp == 3;
+            ptx::prefetch_tensormap(v_side ? &tmV : &tmK);
+            if (v_side) ptx::prefetch_tensormap(&tmQ);
             uint32_t kc = 0, ul = 0;  // key blocks and units issued so far by this CTA
             bool ok = true;
             // A unit's coordinates and its first block index are fetched while the previous unit's
@@ -242,36 +246,40 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             Unit w, wn;
             int32_t j = 0, jnext = 0;
             uint32_t u = next_unit(blockIdx.x, w, j);
-            if (u < (uint32_t)a.n_units) ok = load_q(w, 0);
+            if (v_side && u < (uint32_t)a.n_units) ok = load_q(w, 0);
             while (u < (uint32_t)a.n_units && ok) {
                 const uint32_t un = next_unit(u + gridDim.x, wn, jnext);
                 for (int t = 0; t < w.n; ++t, ++kc) {
                     const int32_t jn = t + 1 < w.n ? __ldg(a.col_idx + w.rs + t + 1) : 0;
-                    const uint32_t ks = kc % kKStages, vs = kc % kVStages;
-                    if (kc >= (uint32_t)kKStages) {
-                        ok = wait_bar(bar(BAR_K_EMPTY + ks), (kc / kKStages - 1) & 1, abort_flag, a.status, 2);
-                        if (!ok) break;
+                    if (!v_side) {
+                        const uint32_t ks = kc % kKStages;
+                        if (kc >= (uint32_t)kKStages) {
+                            ok = wait_bar(bar(BAR_K_EMPTY + ks), (kc / kKStages - 1) & 1, abort_flag, a.status, 2);
+                            if (!ok) break;
+                        }
+                        ptx::mbar_expect_tx(bar(BAR_K_FULL + ks), SM::kBlkTile);
+                        for (int dh = 0; dh < DH; ++dh)
+                            ptx::tma_load_4d(smem_base + SM::kK + ks * SM::kBlkTile + dh * SM::kBlkSub, &tmK,
+                                             bar(BAR_K_FULL + ks), dh * 64, j * kBlk, w.hk, w.b);
+                    } else {
+                        const uint32_t vs = kc % kVStages;
+                        if (kc >= (uint32_t)kVStages) {
+                            ok = wait_bar(bar(BAR_V_EMPTY + vs), (kc / kVStages - 1) & 1, abort_flag, a.status, 3);
+                            if (!ok) break;
+                        }
+                        ptx::mbar_expect_tx(bar(BAR_V_FULL + vs), SM::kBlkTile);
+                        for (int dh = 0; dh < DH; ++dh)
+                            ptx::tma_load_4d(smem_base + SM::kV + vs * SM::kBlkTile + dh * SM::kBlkSub, &tmV,
+                                             bar(BAR_V_FULL + vs), dh * 64, j * kBlk, w.hk, w.b);
+                        // The next unit's Q behind this unit's second block: the unit before this
+                        // one is over by then, so the Q buffer is free and the load has the whole
+                        // unit to arrive.
+                        if (t == (w.n > 1 ? 1 : 0) && un < (uint32_t)a.n_units) {
+                            ok = load_q(wn, ul + 1);
+                            if (!ok) break;
+                        }
                     }
-                    ptx::mbar_expect_tx(bar(BAR_K_FULL + ks), SM::kBlkTile);
-                    for (int dh = 0; dh < DH; ++dh)
-                        ptx::tma_load_4d(smem_base + SM::kK + ks * SM::kBlkTile + dh * SM::kBlkSub, &tmK,
-                                         bar(BAR_K_FULL + ks), dh * 64, j * kBlk, w.hk, w.b);
-                    if (kc >= (uint32_t)kVStages) {
-                        ok = wait_bar(bar(BAR_V_EMPTY + vs), (kc / kVStages - 1) & 1, abort_flag, a.status, 3);
-                        if (!ok) break;
-                    }
-                    ptx::mbar_expect_tx(bar(BAR_V_FULL + vs), SM::kBlkTile);
-                    for (int dh = 0; dh < DH; ++dh)
-                        ptx::tma_load_4d(smem_base + SM::kV + vs * SM::kBlkTile + dh * SM::kBlkSub, &tmV,
-                                         bar(BAR_V_FULL + vs), dh * 64, j * kBlk, w.hk, w.b);
                     j = jn;
-                    // The next unit's Q behind this unit's second block: by then the unit before
-                    // this one has issued its last S (its K stage was just reused), so the Q
-                    // buffer is free and the load has the whole unit to arrive.
-                    if (t == (w.n > 1 ? 1 : 0) && un < (uint32_t)a.n_units) {
-                        ok = load_q(wn, ul + 1);
-                        if (!ok) break;
-                    }
                 }
                 ++ul;
                 u = un;
