@@ -5,15 +5,18 @@
 // holds two 128-row tiles ("slots"); a tile stacks two query heads of the KV group on the 64
 // tokens of the query block (the mask does not depend on the head, so they share the key list
 // and the K/V tiles).  The key list is walked one 64-key block per step.  Warp roles:
-//   warp 0      TMA producer: Q tiles once per unit, then the listed K and V blocks, gathered by
-//               block index, into two rings of shared-memory tiles (128-byte swizzle)
-//   warp 1      tcgen05 issuer: S = Q K^T into tensor memory (two S buffers per slot, so the
-//               logits of step t+1 are ready while the softmax works on step t); O += P V with
-//               P read from tensor memory (it overlays the S buffer it was computed from)
+//   warp 0      TMA producer: the listed K and V blocks, gathered by block index, into two rings
+//               of shared-memory tiles (128-byte swizzle); the next unit's Q tiles early in
+//               the current unit, into the second of two Q buffers
+//   warp 1      tcgen05 issuer.  S = Q K^T of step t+1 is issued as soon as the softmax warps
+//               hold S of step t in registers (one S buffer per slot), so those logits are
+//               ready when step t ends, across unit boundaries too; O += P V is issued when
+//               P has been handed over (P has its own two buffers in tensor memory)
 //   warp 2      tensor-memory allocation
-//   warps 4-7   online softmax of slot 0 (thread = tile row = TMEM lane)
+//   warps 4-7   online softmax of slot 0 (thread = tile row = TMEM lane), LSE
 //   warps 8-11  online softmax of slot 1
-//   warps 12-15 epilogue: O / l and LSE out of tensor memory to global memory
+//   warps 12-15 epilogue: O / l out of tensor memory, staged in shared memory head by head,
+//               bulk tensor stores to global memory; runs beside the next unit's first steps
 // Warps 0-3 and 12-15 give registers back (setmaxnreg) and the softmax warpgroups take them.
 // Every barrier wait is bounded; a wait that runs out records PA_ERR_TIMEOUT in the status
 // block, raises a CTA-wide abort flag and the CTA drains and exits (no trap, no endless spin).
@@ -34,24 +37,14 @@
 // A warpgroup asking for more than the pool holds would wait for ever.
 static_assert(4 * PA_REG_CTRL + 8 * PA_REG_SOFT + 4 * PA_REG_EPI <= 16 * 128, "register split exceeds the CTA's registers");
 static_assert(PA_REG_CTRL % 8 == 0 && PA_REG_SOFT % 8 == 0 && PA_REG_EPI % 8 == 0, "setmaxnreg takes multiples of 8");
-#ifndef PA_PHASE_DELAY
-#define PA_PHASE_DELAY 0
-#endif
-#ifndef PA_K_STAGES
-#define PA_K_STAGES 3
-#define PA_V_STAGES 2
-#endif
-#ifndef PA_WAIT_HINT_NS
-#define PA_WAIT_HINT_NS 0
-#endif
 
 namespace pa {
 
 constexpr int kBlk = 64;               // tokens per query / key block
 constexpr int kThreads = 512;          // 16 warps: control, two softmax warpgroups, epilogue
-constexpr int kKStages = PA_K_STAGES;  // K block ring depth
-constexpr int kVStages = PA_V_STAGES;  // V block ring depth
-constexpr uint32_t kTmemCols = 512;    // slot s: S/P buffers at columns 128 s + 64 b, O at 256 + s D
+constexpr int kKStages = 3;             // K block ring depth (a K block is needed at the start of a step)
+constexpr int kVStages = 2;             // V block ring depth (a V block is needed at its end)
+constexpr uint32_t kTmemCols = 512;    // slot s: S at columns 128 s, P buffers at 128 s + 64 + 32 b, O at 256 + s D
 // A step's row sum above this limit sends the step through the exact path (new reference).
 constexpr float kSumLimit = 1048576.0f;  // 2^20
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logits: rescale O only when the row max grows by more
@@ -132,11 +125,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     const long long t0 = clock64();
     uint32_t it = 0;
     while (true) {
-#if PA_WAIT_HINT_NS > 0
-        if (ptx::mbar_try_wait_hint(bar, parity, PA_WAIT_HINT_NS)) return true;
-#else
         if (ptx::mbar_try_wait(bar, parity)) return true;
-#endif
         if ((++it & 63u) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitCycles) break;
@@ -206,16 +195,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const uint32_t tmem_base = tmem_base_any;
 
     if (warp < 4) ptx::setmaxnreg_dec<PA_REG_CTRL>();
-    if (warp == 0 || warp == 3) {
-        // ------------------------------------------------------------------ TMA producers
-        // Two independent streams, each walking the unit list and the key-block lists by itself:
-        // warp 0 fetches the K blocks (needed at the start of a step), warp 3 the V blocks (needed
-        // at its end) and the Q tiles.  Apart, a full V ring or a Q tile in the queue cannot hold
-        // the next K block back.
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            const bool v_side = warp == 3;
-            ptx::prefetch_tensormap(v_side ? &tmV : &tmK);
-            if (v_side) ptx::prefetch_tensormap(&tmQ);
+            ptx::prefetch_tensormap(&tmQ);
+            ptx::prefetch_tensormap(&tmK);
+            ptx::prefetch_tensormap(&tmV);
             uint32_t kc = 0, ul = 0;  // key blocks and units issued so far by this CTA
             bool ok = true;
             // A unit's coordinates and its first block index are fetched while the previous unit's
@@ -246,40 +231,36 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             Unit w, wn;
             int32_t j = 0, jnext = 0;
             uint32_t u = next_unit(blockIdx.x, w, j);
-            if (v_side && u < (uint32_t)a.n_units) ok = load_q(w, 0);
+            if (u < (uint32_t)a.n_units) ok = load_q(w, 0);
             while (u < (uint32_t)a.n_units && ok) {
                 const uint32_t un = next_unit(u + gridDim.x, wn, jnext);
                 for (int t = 0; t < w.n; ++t, ++kc) {
                     const int32_t jn = t + 1 < w.n ? __ldg(a.col_idx + w.rs + t + 1) : 0;
-                    if (!v_side) {
-                        const uint32_t ks = kc % kKStages;
-                        if (kc >= (uint32_t)kKStages) {
-                            ok = wait_bar(bar(BAR_K_EMPTY + ks), (kc / kKStages - 1) & 1, abort_flag, a.status, 2);
-                            if (!ok) break;
-                        }
-                        ptx::mbar_expect_tx(bar(BAR_K_FULL + ks), SM::kBlkTile);
-                        for (int dh = 0; dh < DH; ++dh)
-                            ptx::tma_load_4d(smem_base + SM::kK + ks * SM::kBlkTile + dh * SM::kBlkSub, &tmK,
-                                             bar(BAR_K_FULL + ks), dh * 64, j * kBlk, w.hk, w.b);
-                    } else {
-                        const uint32_t vs = kc % kVStages;
-                        if (kc >= (uint32_t)kVStages) {
-                            ok = wait_bar(bar(BAR_V_EMPTY + vs), (kc / kVStages - 1) & 1, abort_flag, a.status, 3);
-                            if (!ok) break;
-                        }
-                        ptx::mbar_expect_tx(bar(BAR_V_FULL + vs), SM::kBlkTile);
-                        for (int dh = 0; dh < DH; ++dh)
-                            ptx::tma_load_4d(smem_base + SM::kV + vs * SM::kBlkTile + dh * SM::kBlkSub, &tmV,
-                                             bar(BAR_V_FULL + vs), dh * 64, j * kBlk, w.hk, w.b);
-                        // The next unit's Q behind this unit's second block: the unit before this
-                        // one is over by then, so the Q buffer is free and the load has the whole
-                        // unit to arrive.
-                        if (t == (w.n > 1 ? 1 : 0) && un < (uint32_t)a.n_units) {
-                            ok = load_q(wn, ul + 1);
-                            if (!ok) break;
-                        }
+                    const uint32_t ks = kc % kKStages, vs = kc % kVStages;
+                    if (kc >= (uint32_t)kKStages) {
+                        ok = wait_bar(bar(BAR_K_EMPTY + ks), (kc / kKStages - 1) & 1, abort_flag, a.status, 2);
+                        if (!ok) break;
                     }
+                    ptx::mbar_expect_tx(bar(BAR_K_FULL + ks), SM::kBlkTile);
+                    for (int dh = 0; dh < DH; ++dh)
+                        ptx::tma_load_4d(smem_base + SM::kK + ks * SM::kBlkTile + dh * SM::kBlkSub, &tmK,
+                                         bar(BAR_K_FULL + ks), dh * 64, j * kBlk, w.hk, w.b);
+                    if (kc >= (uint32_t)kVStages) {
+                        ok = wait_bar(bar(BAR_V_EMPTY + vs), (kc / kVStages - 1) & 1, abort_flag, a.status, 3);
+                        if (!ok) break;
+                    }
+                    ptx::mbar_expect_tx(bar(BAR_V_FULL + vs), SM::kBlkTile);
+                    for (int dh = 0; dh < DH; ++dh)
+                        ptx::tma_load_4d(smem_base + SM::kV + vs * SM::kBlkTile + dh * SM::kBlkSub, &tmV,
+                                         bar(BAR_V_FULL + vs), dh * 64, j * kBlk, w.hk, w.b);
                     j = jn;
+                    // The next unit's Q behind this unit's second block: by then the unit before
+                    // this one has issued its last S (its K stage was just reused), so the Q
+                    // buffer is free and the load has the whole unit to arrive.
+                    if (t == (w.n > 1 ? 1 : 0) && un < (uint32_t)a.n_units) {
+                        ok = load_q(wn, ul + 1);
+                        if (!ok) break;
+                    }
                 }
                 ++ul;
                 u = un;
@@ -475,13 +456,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 ok = wait_bar(bar(BAR_S_FULL + s), kc & 1, abort_flag, a.status, 9);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-#if PA_PHASE_DELAY > 0
-                if (s == 1 && kc == 0) {
-                    const long long t0 = clock64();
-                    while (clock64() - t0 < PA_PHASE_DELAY) {
-                    }
-                }
-#endif
                 ptx::tc_fence_after_sync();
                 ptx::tmem_ld32(t_s0, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
                 ptx::tmem_ld32(t_s0 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
