@@ -7,8 +7,10 @@
 // output on the warp-level tensor-core MMA.  The chunk partials (o[D], m, l) are then merged with
 // the log-sum-exp rule by a second kernel, launched with programmatic dependent launch so that
 // its start-up overlaps the first kernel's tail; it waits for the partials with griddepcontrol.wait.
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <math.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 #include "layout_rule.cuh"
@@ -257,6 +259,259 @@ __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeArgs a)
     if (d == 0) a.lse[(int64_t)b * a.Hq + h] = n > 0 ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
 }
 
+// ------------------------------------------------------------------------------------------
+// One launch per call: a thread-block cluster per (sequence, KV head).
+//
+// The row's key blocks are dealt round-robin to the CTAs of the cluster (at most kRowMaxBlk each).
+// A CTA first requests all of its K and V blocks with 16-byte asynchronous copies into shared
+// memory (everything it will ever read is in flight at once), then takes them in order as they
+// land: logits and P V as in decode_block_kernel, with the running maximum, sum and output kept
+// in registers across blocks (online softmax).  The CTAs' partial results meet in shared memory:
+// after a cluster barrier CTA r merges the heads g = r, r + R, ... reading its peers' partials
+// through distributed shared memory, and writes O and the LSE.  No workspace, no second launch.
+// ------------------------------------------------------------------------------------------
+constexpr int kRowMaxBlk = 4;      // key blocks per CTA
+constexpr int kRowMaxCluster = 8;  // portable cluster size limit
+
+template <int D>
+struct RowSmem {
+    static constexpr int kPitch = D * 2 + 16;                  // bytes per key row (padded: no bank conflicts)
+    static constexpr int kTile = kDecBlock * kPitch;           // one K or V block
+    static constexpr int kBlockBytes = 2 * kTile;              // K + V of one key block
+};
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+// Waits until at most `pending` of this thread's copy groups are still in flight.
+__device__ __forceinline__ void cp_async_wait(int pending)
+{
+    switch (pending) {
+        case 0: asm volatile("cp.async.wait_group 0;\n" ::: "memory"); break;
+        case 1: asm volatile("cp.async.wait_group 1;\n" ::: "memory"); break;
+        case 2: asm volatile("cp.async.wait_group 2;\n" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 3;\n" ::: "memory"); break;
+    }
+}
+__device__ __forceinline__ uint4 lds16(uint32_t addr)
+{
+    uint4 r;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];\n" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+    return r;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArgs a)
+{
+    namespace cg = cooperative_groups;
+    using SM = RowSmem<D>;
+    constexpr int NJ = D / 32;  // 16-byte pieces per thread and row for Q and K
+    constexpr int NP = D / 8;   // 16-byte pieces per row
+    extern __shared__ __align__(16) uint8_t row_smem[];
+    __shared__ float sS[kMaxGroup][kDecBlock + 8];  // base-2 logits of the current block
+    __shared__ float sO[kMaxGroup][D];              // this CTA's unnormalised output
+    __shared__ float sML[kMaxGroup][2];             // this CTA's running maximum and sum
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const int R = (int)gridDim.x, r = (int)blockIdx.x;  // the cluster spans grid x
+    const int hk = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int G = a.G;
+
+    const int64_t len = a.lens[b];
+    const bool valid = len >= 1 && len <= a.max_len;
+    const int64_t p = len - 1;
+    const int32_t row = valid ? (int32_t)(p / kDecBlock) : 0;
+    // Every thread walks the (short) list and keeps this CTA's entries.
+    int32_t jb[kRowMaxBlk];
+#pragma unroll
+    for (int i = 0; i < kRowMaxBlk; ++i) jb[i] = -1;
+    int n = 0;
+    if (valid)
+        n = for_each_key_block_t<int32_t>(row, a.W, a.S, [&](int pos, int32_t j) {
+#pragma unroll
+            for (int i = 0; i < kRowMaxBlk; ++i)
+                if (pos == r + i * R) jb[i] = j;
+        });
+    int mine = n > r ? (n - r + R - 1) / R : 0;
+    if (mine > kRowMaxBlk) mine = kRowMaxBlk;  // (the host sizes the cluster so that this never cuts)
+
+    // ---- all loads of this CTA, one copy group per key block
+    const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(row_smem);
+#pragma unroll
+    for (int i = 0; i < kRowMaxBlk; ++i) {
+        if (i < mine) {
+            const int n_keys = jb[i] == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
+            const __nv_bfloat16 *kb = a.k + b * a.k_sb + ((int64_t)jb[i] * kDecBlock) * a.k_ss + hk * a.k_sh;
+            const __nv_bfloat16 *vb = a.v + b * a.v_sb + ((int64_t)jb[i] * kDecBlock) * a.v_ss + hk * a.v_sh;
+            const uint32_t sk = smem0 + i * SM::kBlockBytes, sv = sk + SM::kTile;
+#pragma unroll
+            for (int q = 0; q < kDecBlock * NP / kDecThreads; ++q) {
+                const int idx = tid + q * kDecThreads;
+                const int key = idx / NP, pc = idx % NP;
+                const bool there = key < n_keys;  // rows beyond the sequence end are zero-filled
+                cp_async16(sk + key * SM::kPitch + pc * 16, there ? (const void *)(kb + key * a.k_ss + 8 * pc) : (const void *)kb,
+                           there ? 16u : 0u);
+                cp_async16(sv + key * SM::kPitch + pc * 16, there ? (const void *)(vb + key * a.v_ss + 8 * pc) : (const void *)vb,
+                           there ? 16u : 0u);
+            }
+            cp_async_commit();
+        }
+    }
+
+    uint4 qr[NJ];
+    {
+        const __nv_bfloat16 *qb = a.q + ((int64_t)b * a.Hq + (int64_t)hk * G + g) * D;
+        const uint4 zero4 = make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) qr[j] = g < G ? ldg16(qb + 8 * (4 * j + t)) : zero4;
+    }
+
+    const int base = wid * 16;             // first key of this warp's logit tile
+    const int vchunk = (g & 3) + 4 * wid;  // this thread's 8-feature piece of V rows
+    const bool pv_warp = 4 * wid < D / 8;  // warps that own output features
+    const bool hi = (g >> 2) != 0;
+    float m_run = -INFINITY, l_run = 0.f;
+    float acc[4][4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) acc[e][0] = acc[e][1] = acc[e][2] = acc[e][3] = 0.f;
+
+#pragma unroll 1
+    for (int i = 0; i < mine; ++i) {
+        const int32_t jblk = i == 0 ? jb[0] : i == 1 ? jb[1] : i == 2 ? jb[2] : jb[3];
+        const int n_keys = jblk == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
+        const uint32_t sk = smem0 + i * SM::kBlockBytes, sv_ = sk + SM::kTile;
+        cp_async_wait(mine - 1 - i);
+        __syncthreads();  // every thread's copies of this block have landed; sS is free again
+
+        // ---- S = Q K^T: rows = heads, columns = the warp's 16 keys (two 8-key tiles)
+        float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+            const int key = base + nt * 8 + g;
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) {
+                const uint4 kr = lds16(sk + key * SM::kPitch + 16 * (4 * j + t));
+                mma_bf16(sc[nt], qr[j].x, 0u, qr[j].y, 0u, kr.x, kr.y);
+                mma_bf16(sc[nt], qr[j].z, 0u, qr[j].w, 0u, kr.z, kr.w);
+            }
+        }
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+            const int key = base + nt * 8 + 2 * t;
+            float2 v2;
+            v2.x = key < n_keys ? sc[nt][0] * a.scale_log2 : -INFINITY;
+            v2.y = key + 1 < n_keys ? sc[nt][1] * a.scale_log2 : -INFINITY;
+            *reinterpret_cast<float2 *>(&sS[g][key]) = v2;
+        }
+        __syncthreads();
+
+        // ---- online softmax over the block: thread (g, t) takes keys 16 ks + {2t, 2t+1, 2t+8, 2t+9}
+        float2 sv[4][2];
+        float mrow = -INFINITY;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                sv[ks][hh] = *reinterpret_cast<const float2 *>(&sS[g][16 * ks + 8 * hh + 2 * t]);
+                mrow = fmaxf(mrow, fmaxf(sv[ks][hh].x, sv[ks][hh].y));
+            }
+        mrow = fmaxf(mrow, __shfl_xor_sync(0xffffffffu, mrow, 1));
+        mrow = fmaxf(mrow, __shfl_xor_sync(0xffffffffu, mrow, 2));  // finite: key 0 of the block exists
+        const float m_new = fmaxf(m_run, mrow);
+        const float alpha = ex2_approx(m_run - m_new);  // 0 on the first block
+        uint32_t pa[4][2];
+        float lrow = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const float p0 = ex2_approx(sv[ks][hh].x - m_new), p1 = ex2_approx(sv[ks][hh].y - m_new);
+                lrow += p0 + p1;
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+                pa[ks][hh] = *reinterpret_cast<const uint32_t *>(&h2);
+            }
+        lrow += __shfl_xor_sync(0xffffffffu, lrow, 1);
+        lrow += __shfl_xor_sync(0xffffffffu, lrow, 2);
+        l_run = l_run * alpha + lrow;
+        m_run = m_new;
+
+        // ---- O = alpha O + P V for this warp's 32 features (see decode_block_kernel)
+        if (pv_warp) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                acc[e][0] *= alpha;
+                acc[e][1] *= alpha;
+            }
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                uint4 vr[4];
+#pragma unroll
+                for (int kx = 0; kx < 4; ++kx) {
+                    const int key = 16 * ks + 2 * t + (kx & 1) + (kx >> 1) * 8;
+                    vr[kx] = lds16(sv_ + key * SM::kPitch + 16 * vchunk);
+                }
+                uint32_t w0[2], w1[2], w2[2], w3[2];
+                w0[0] = hi ? vr[0].z : vr[0].x; w0[1] = hi ? vr[0].w : vr[0].y;
+                w1[0] = hi ? vr[1].z : vr[1].x; w1[1] = hi ? vr[1].w : vr[1].y;
+                w2[0] = hi ? vr[2].z : vr[2].x; w2[1] = hi ? vr[2].w : vr[2].y;
+                w3[0] = hi ? vr[3].z : vr[3].x; w3[1] = hi ? vr[3].w : vr[3].y;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
+                    const uint32_t b0 = __byte_perm(w0[e >> 1], w1[e >> 1], sel);
+                    const uint32_t b1 = __byte_perm(w2[e >> 1], w3[e >> 1], sel);
+                    mma_bf16(acc[e], pa[ks][0], 0u, pa[ks][1], 0u, b0, b1);
+                }
+            }
+        }
+    }
+
+    // ---- this CTA's partial result to shared memory
+    if (pv_warp && g < G) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                const int nn = 2 * t + x;
+                sO[g][8 * ((nn & 3) + 4 * wid) + e + 4 * (nn >> 2)] = acc[e][x];
+            }
+    }
+    if (wid == 0 && t == 0 && g < G) {
+        sML[g][0] = m_run;
+        sML[g][1] = l_run;
+    }
+    cluster.sync();
+
+    // ---- merge across the cluster: CTA r takes heads r, r + R, ...; thread d one feature
+    if (tid < D) {
+        for (int h = r; h < G; h += R) {
+            float m = -INFINITY;
+            for (int rr = 0; rr < R; ++rr) m = fmaxf(m, cluster.map_shared_rank(&sML[0][0], rr)[2 * h]);
+            float l = 0.f, o = 0.f;
+            for (int rr = 0; rr < R; ++rr) {
+                const float *ml = cluster.map_shared_rank(&sML[0][0], rr);
+                const float *po = cluster.map_shared_rank(&sO[0][0], rr);
+                const float wgt = ml[2 * h] == -INFINITY ? 0.f : exp2f(ml[2 * h] - m);
+                l += ml[2 * h + 1] * wgt;
+                o += po[h * D + tid] * wgt;
+            }
+            const float out = n > 0 ? o / l : 0.f;
+            const int64_t oi = ((int64_t)b * a.Hq + (int64_t)hk * G + h) * D + tid;
+            if (a.o_is_f32)
+                reinterpret_cast<float *>(a.o)[oi] = out;
+            else
+                reinterpret_cast<__nv_bfloat16 *>(a.o)[oi] = __float2bfloat16_rn(out);
+            if (tid == 0)
+                a.lse[(int64_t)b * a.Hq + (int64_t)hk * G + h] = n > 0 ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+        }
+    }
+    cluster.sync();  // peers may still be reading this CTA's shared memory
+}
+
 __global__ void decode_block_list_kernel(int64_t len, int32_t W, int32_t S, int32_t *out,
                                          int32_t *count, int32_t capacity)
 {
@@ -277,6 +532,20 @@ static int max_row_blocks(int64_t n_rows, int32_t W, int32_t S)
         if (pw >= w) ++powers;
     const int64_t bound = w + S + powers;
     return (int)(bound < n_rows ? bound : n_rows);
+}
+
+// PA_DECODE_PATH=splitk forces the two-launch split-K path (tests use it to cover that path on
+// workloads the cluster path would take); PA_DECODE_CLUSTER=n sets the cluster size (1..8).
+static int decode_path()
+{
+    const char *e = getenv("PA_DECODE_PATH");
+    return e && e[0] == 's' ? 1 : 0;
+}
+static int decode_cluster()
+{
+    const char *e = getenv("PA_DECODE_CLUSTER");
+    const int v = e ? atoi(e) : 0;
+    return v >= 1 && v <= kRowMaxCluster ? v : 4;
 }
 
 static pa_status check_decode(const pa_decode_params *p)
@@ -356,6 +625,44 @@ extern "C" pa_status pa_decode(const pa_decode_params *p, const void *q, const v
     a.scale_log2 = scale * 1.4426950408889634f;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // Rows short enough for one cluster per (sequence, KV head) take the single-launch path.
+    if (decode_path() != 1 && a.chunks <= kRowMaxBlk * kRowMaxCluster) {
+        int R = decode_cluster();
+        if (R * kRowMaxBlk < a.chunks) R = (a.chunks + kRowMaxBlk - 1) / kRowMaxBlk;
+        if (R > a.chunks) R = a.chunks;
+        const int per_cta = (a.chunks + R - 1) / R;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)R, (unsigned)a.Hkv, (unsigned)a.batch);
+        cfg.blockDim = dim3(kDecThreads, 1, 1);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)R;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (p->head_dim == 128) {
+            cfg.dynamicSmemBytes = (size_t)per_cta * RowSmem<128>::kBlockBytes;
+            static bool sized128 = false;  // (idempotent: a race between threads only repeats the call)
+            if (!sized128) {
+                PA_CUDA_OK(cudaFuncSetAttribute(decode_row_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                kRowMaxBlk * RowSmem<128>::kBlockBytes));
+                sized128 = true;
+            }
+            PA_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_row_kernel<128>, a));
+        } else {
+            cfg.dynamicSmemBytes = (size_t)per_cta * RowSmem<64>::kBlockBytes;
+            static bool sized64 = false;
+            if (!sized64) {
+                PA_CUDA_OK(cudaFuncSetAttribute(decode_row_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                kRowMaxBlk * RowSmem<64>::kBlockBytes));
+                sized64 = true;
+            }
+            PA_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_row_kernel<64>, a));
+        }
+        return PA_OK;
+    }
     const dim3 grid1((unsigned)a.chunks, (unsigned)a.Hkv, (unsigned)a.batch);
     if (p->head_dim == 128)
         decode_block_kernel<128><<<grid1, kDecThreads, 0, st>>>(a);

@@ -85,3 +85,18 @@ def test_decode_full_size_workload(pa, oracle):
     q, kc, vc, lens = si.decode_inputs(w)
     st = _run(pa, oracle, q, kc, vc, lens, w.window_blocks, w.sink_blocks)
     print("decode full-size error stats", st)
+
+
+@pytest.mark.parametrize("env", [{"PA_DECODE_PATH": "splitk"}, {"PA_DECODE_CLUSTER": "1"}, {"PA_DECODE_CLUSTER": "2"},
+                                 {"PA_DECODE_CLUSTER": "7"}, {"PA_DECODE_CLUSTER": "8"}])
+def test_decode_paths(pa, oracle, monkeypatch, env):
+    """The two-launch split-K path and the single-launch cluster path at several cluster sizes
+    (the library reads these switches on every call) give the same row of Eq. (1)."""
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    batch, max_len, Hq, Hkv, D = 4, 9000, 28, 4, 128
+    q = si.bf16_randn((batch, Hq, D), 31)
+    kc, vc = si.bf16_randn((batch, max_len, Hkv, D), 32, 2.0), si.bf16_randn((batch, max_len, Hkv, D), 33)
+    lens = np.array([9000, 8193, 130, 7])
+    _run(pa, oracle, q, kc, vc, lens, 5, 1)
+    _run(pa, oracle, q, kc, vc, lens, 3, 2, o_dtype=torch.float32)
