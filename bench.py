@@ -255,7 +255,7 @@ def run_ours(args):
             ev_p1[i].record(stream)
         pa.pa_decode(qd, kc, vc, lens_d, wd.window_blocks, wd.sink_blocks, o=Od, lse=LSEd, workspace=wsd)
 
-    launches_per_step = 3 + 1 + 2  # layout (count, scan, fill) + prefill + decode (partial, combine)
+    launches_per_step = 3 + 1 + 1  # layout (count, scan, fill) + prefill + decode (one cluster kernel)
 
     for _ in range(max(args.warmup, 3)):
         step()

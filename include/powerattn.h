@@ -146,9 +146,16 @@ size_t pa_decode_workspace_bytes(const pa_decode_params *p);
  * strides.  cache_lens: device int32 [batch], each in [1, max_len] (a length outside that
  * range makes the sequence's outputs zero and its LSE -inf; nothing faults).
  * o: device [batch, n_q_heads, head_dim] contiguous, o_dtype.  lse: device fp32
- * [batch, n_q_heads].  Enqueues two kernels: partial attention per (sequence, KV head, chunk),
- * then the log-sum-exp combine  m = max m_c, l = sum l_c e^(m_c - m), o = sum o_c e^(m_c - m) / l.
- * Calls that share a workspace must not overlap on the GPU. */
+ * [batch, n_q_heads].  When no row can list more than 32 key blocks (any default-window row up
+ * to millions of tokens) one kernel is enqueued: a thread-block cluster per (sequence, KV head)
+ * shares the row's blocks, each CTA runs an online softmax over its blocks, and the partial
+ * results are merged inside the cluster with the log-sum-exp rule
+ * m = max m_c, l = sum l_c e^(m_c - m), o = sum o_c e^(m_c - m) / l; the workspace is then not
+ * touched.  Otherwise two kernels are enqueued: partial attention per (sequence, KV head,
+ * block) into the workspace, then the same merge.  The workspace must be given in both cases.
+ * Calls that share a workspace must not overlap on the GPU.  Environment switches read on every
+ * call (for tests and measurements): PA_DECODE_PATH=splitk forces the two-kernel path,
+ * PA_DECODE_CLUSTER=n (1..8) sets the cluster size. */
 pa_status pa_decode(const pa_decode_params *p, const void *q, const void *k_cache,
                     const void *v_cache, const int32_t *cache_lens, void *o, float *lse,
                     void *workspace, size_t workspace_bytes, void *stream);

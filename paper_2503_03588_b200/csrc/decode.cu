@@ -1,6 +1,10 @@
 // pa_decode: one query token per sequence against its KV cache under the PowerAttention row of
 // its position (Section 4.1: same pattern in prefilling and decoding; Eq. (1) for the row).
 //
+// Two paths.  Rows of at most 32 listed blocks (every PowerAttention row with the default window
+// up to millions of tokens) take decode_row_kernel: one launch, a thread-block cluster per
+// (sequence, KV head), described at that kernel.  Longer rows take the split-K pair below.
+//
 // Split-K: one CTA per (sequence, KV head, chunk) where a chunk is one 64-key block of the
 // row's block list.  Each CTA reads its K and V block with coalesced 16-byte loads and computes
 // the logits of all query heads of the group, a chunk-local softmax and the unnormalised partial
@@ -545,8 +549,9 @@ static int decode_cluster()
 {
     const char *e = getenv("PA_DECODE_CLUSTER");
     const int v = e ? atoi(e) : 0;
-    return v >= 1 && v <= kRowMaxCluster ? v : 4;
+    return v >= 1 && v <= kRowMaxCluster ? v : kRowMaxCluster;
 }
+
 
 static pa_status check_decode(const pa_decode_params *p)
 {
