@@ -267,7 +267,7 @@ __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeArgs a)
 // One launch per call: a thread-block cluster per (sequence, KV head).
 //
 // The row's key blocks are dealt round-robin to the CTAs of the cluster (at most kRowMaxBlk each).
-// A CTA first requests all of its K and V blocks with 16-byte asynchronous copies into shared
+// A CTA first requests all of its K and V blocks with one bulk copy per key row into shared
 // memory (everything it will ever read is in flight at once), then takes them in order as they
 // land: logits and P V as in decode_block_kernel, with the running maximum, sum and output kept
 // in registers across blocks (online softmax).  The CTAs' partial results meet in shared memory:
@@ -284,21 +284,6 @@ struct RowSmem {
     static constexpr int kBlockBytes = 2 * kTile;              // K + V of one key block
 };
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32_t src_bytes)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-// Waits until at most `pending` of this thread's copy groups are still in flight.
-__device__ __forceinline__ void cp_async_wait(int pending)
-{
-    switch (pending) {
-        case 0: asm volatile("cp.async.wait_group 0;\n" ::: "memory"); break;
-        case 1: asm volatile("cp.async.wait_group 1;\n" ::: "memory"); break;
-        case 2: asm volatile("cp.async.wait_group 2;\n" ::: "memory"); break;
-        default: asm volatile("cp.async.wait_group 3;\n" ::: "memory"); break;
-    }
-}
 __device__ __forceinline__ uint4 lds16(uint32_t addr)
 {
     uint4 r;
@@ -312,11 +297,11 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
     namespace cg = cooperative_groups;
     using SM = RowSmem<D>;
     constexpr int NJ = D / 32;  // 16-byte pieces per thread and row for Q and K
-    constexpr int NP = D / 8;   // 16-byte pieces per row
     extern __shared__ __align__(16) uint8_t row_smem[];
     __shared__ float sS[kMaxGroup][kDecBlock + 8];  // base-2 logits of the current block
     __shared__ float sO[kMaxGroup][D];              // this CTA's unnormalised output
     __shared__ float sML[kMaxGroup][2];             // this CTA's running maximum and sum
+    __shared__ __align__(8) uint64_t s_bar[kRowMaxBlk];  // one per key block: its copies have landed
 
     cg::cluster_group cluster = cg::this_cluster();
     const int R = (int)gridDim.x, r = (int)blockIdx.x;  // the cluster spans grid x
@@ -329,40 +314,72 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
     const bool valid = len >= 1 && len <= a.max_len;
     const int64_t p = len - 1;
     const int32_t row = valid ? (int32_t)(p / kDecBlock) : 0;
-    // Every thread walks the (short) list and keeps this CTA's entries.
-    int32_t jb[kRowMaxBlk];
-#pragma unroll
-    for (int i = 0; i < kRowMaxBlk; ++i) jb[i] = -1;
-    int n = 0;
-    if (valid)
-        n = for_each_key_block_t<int32_t>(row, a.W, a.S, [&](int pos, int32_t j) {
-#pragma unroll
-            for (int i = 0; i < kRowMaxBlk; ++i)
-                if (pos == r + i * R) jb[i] = j;
-        });
+    // The row's block set, one candidate per lane (the order does not matter for Eq. (1), so the
+    // set is not sorted: window distances 0 .. w-1, then the power-of-two distances >= w that do
+    // not land on a sink block, then the sink blocks outside the window).  The host takes this
+    // path only when window + powers + sinks fit the 32 lanes.
+    int32_t cand = -1;
+    if (valid) {
+        const int32_t w_eff = a.W > 1 ? a.W : 1;
+        const int k0 = w_eff <= 1 ? 0 : 32 - __clz(w_eff - 1);  // first k with 2^k >= w_eff
+        const int kmax = row >= 1 ? 31 - __clz(row) : -1;       // last k with 2^k <= row
+        const int n_pow = kmax >= k0 ? kmax - k0 + 1 : 0;
+        if (lane < w_eff) {
+            cand = row - lane;  // negative: before the sequence start
+        } else if (lane < w_eff + n_pow) {
+            const int32_t j = row - (1 << (k0 + lane - w_eff));
+            if (j >= a.S) cand = j;
+        } else if (lane < w_eff + n_pow + a.S) {
+            const int32_t j = lane - w_eff - n_pow;
+            if (row - j >= w_eff) cand = j;  // also implies j <= row
+        }
+    }
+    const uint32_t have = __ballot_sync(0xffffffffu, cand >= 0);
+    const int n = __popc(have);
     int mine = n > r ? (n - r + R - 1) / R : 0;
     if (mine > kRowMaxBlk) mine = kRowMaxBlk;  // (the host sizes the cluster so that this never cuts)
+    int32_t jb[kRowMaxBlk];
+#pragma unroll
+    for (int i = 0; i < kRowMaxBlk; ++i) {
+        const int src = i < mine ? (int)__fns(have, 0, r + i * R + 1) : 0;
+        jb[i] = __shfl_sync(0xffffffffu, cand, src & 31);
+    }
 
-    // ---- all loads of this CTA, one copy group per key block
+    // ---- all loads of this CTA at once: one bulk copy per key row of K and of V (thread = row),
+    // counted on one mbarrier per key block; rows past the sequence end are zero-filled instead.
     const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(row_smem);
+    const uint32_t bars0 = (uint32_t)__cvta_generic_to_shared(&s_bar[0]);
+    if (tid == 0) {
+#pragma unroll
+        for (int i = 0; i < kRowMaxBlk; ++i)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bars0 + 8 * i));
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    }
+    __syncthreads();
 #pragma unroll
     for (int i = 0; i < kRowMaxBlk; ++i) {
         if (i < mine) {
             const int n_keys = jb[i] == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
-            const __nv_bfloat16 *kb = a.k + b * a.k_sb + ((int64_t)jb[i] * kDecBlock) * a.k_ss + hk * a.k_sh;
-            const __nv_bfloat16 *vb = a.v + b * a.v_sb + ((int64_t)jb[i] * kDecBlock) * a.v_ss + hk * a.v_sh;
-            const uint32_t sk = smem0 + i * SM::kBlockBytes, sv = sk + SM::kTile;
+            const int key = tid & (kDecBlock - 1);
+            const bool is_v = tid >= kDecBlock;
+            const __nv_bfloat16 *src = is_v ? a.v + b * a.v_sb + ((int64_t)jb[i] * kDecBlock + key) * a.v_ss + hk * a.v_sh
+                                            : a.k + b * a.k_sb + ((int64_t)jb[i] * kDecBlock + key) * a.k_ss + hk * a.k_sh;
+            const uint32_t dst = smem0 + i * SM::kBlockBytes + (is_v ? SM::kTile : 0) + key * SM::kPitch;
+            if (key < n_keys) {
+                asm volatile(
+                    "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
+                    "l"(src), "r"((uint32_t)(D * 2)), "r"(bars0 + 8 * i)
+                    : "memory");
+            } else {
 #pragma unroll
-            for (int q = 0; q < kDecBlock * NP / kDecThreads; ++q) {
-                const int idx = tid + q * kDecThreads;
-                const int key = idx / NP, pc = idx % NP;
-                const bool there = key < n_keys;  // rows beyond the sequence end are zero-filled
-                cp_async16(sk + key * SM::kPitch + pc * 16, there ? (const void *)(kb + key * a.k_ss + 8 * pc) : (const void *)kb,
-                           there ? 16u : 0u);
-                cp_async16(sv + key * SM::kPitch + pc * 16, there ? (const void *)(vb + key * a.v_ss + 8 * pc) : (const void *)vb,
-                           there ? 16u : 0u);
+                for (int c = 0; c < D * 2 / 16; ++c)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};\n" ::"r"(dst + 16 * c), "r"(0u) : "memory");
             }
-            cp_async_commit();
+            if (tid == 0)
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bars0 + 8 * i),
+                             "r"((uint32_t)(n_keys * 2 * D * 2))
+                             : "memory");
         }
     }
 
@@ -388,8 +405,19 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
         const int32_t jblk = i == 0 ? jb[0] : i == 1 ? jb[1] : i == 2 ? jb[2] : jb[3];
         const int n_keys = jblk == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
         const uint32_t sk = smem0 + i * SM::kBlockBytes, sv_ = sk + SM::kTile;
-        cp_async_wait(mine - 1 - i);
-        __syncthreads();  // every thread's copies of this block have landed; sS is free again
+        // The block's copies have landed (bounded poll; they always do).
+        {
+            uint32_t done = 0;
+            for (uint32_t it = 0; !done && it < (1u << 26); ++it)
+                asm volatile(
+                    "{\n\t.reg .pred p;\n\t"
+                    "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
+                    "selp.u32 %0, 1, 0, p;\n\t}\n"
+                    : "=r"(done)
+                    : "r"(bars0 + 8 * i)
+                    : "memory");
+        }
+        __syncthreads();  // zero-filled rows are visible; sS is free again
 
         // ---- S = Q K^T: rows = heads, columns = the warp's 16 keys (two 8-key tiles)
         float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -490,18 +518,36 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
     }
     cluster.sync();
 
-    // ---- merge across the cluster: CTA r takes heads r, r + R, ...; thread d one feature
+    // ---- merge across the cluster: CTA r takes heads r, r + R, ...; thread d one feature.  All
+    // remote reads of a head are issued before the first one is used (they are independent, and
+    // each costs a trip through the cluster's shared-memory network).
     if (tid < D) {
+        const float *peer_ml[kRowMaxCluster];
+        const float *peer_o[kRowMaxCluster];
+#pragma unroll
+        for (int rr = 0; rr < kRowMaxCluster; ++rr) {
+            const int src = rr < R ? rr : r;  // (slots beyond the cluster are given weight 0 below)
+            peer_ml[rr] = cluster.map_shared_rank(&sML[0][0], src);
+            peer_o[rr] = cluster.map_shared_rank(&sO[0][0], src);
+        }
         for (int h = r; h < G; h += R) {
+            float mr[kRowMaxCluster], lr[kRowMaxCluster], orr[kRowMaxCluster];
+#pragma unroll
+            for (int rr = 0; rr < kRowMaxCluster; ++rr) {
+                mr[rr] = peer_ml[rr][2 * h];
+                lr[rr] = peer_ml[rr][2 * h + 1];
+                orr[rr] = peer_o[rr][h * D + tid];
+            }
             float m = -INFINITY;
-            for (int rr = 0; rr < R; ++rr) m = fmaxf(m, cluster.map_shared_rank(&sML[0][0], rr)[2 * h]);
+#pragma unroll
+            for (int rr = 0; rr < kRowMaxCluster; ++rr)
+                if (rr < R) m = fmaxf(m, mr[rr]);
             float l = 0.f, o = 0.f;
-            for (int rr = 0; rr < R; ++rr) {
-                const float *ml = cluster.map_shared_rank(&sML[0][0], rr);
-                const float *po = cluster.map_shared_rank(&sO[0][0], rr);
-                const float wgt = ml[2 * h] == -INFINITY ? 0.f : exp2f(ml[2 * h] - m);
-                l += ml[2 * h + 1] * wgt;
-                o += po[h * D + tid] * wgt;
+#pragma unroll
+            for (int rr = 0; rr < kRowMaxCluster; ++rr) {
+                const float wgt = (rr < R && mr[rr] != -INFINITY) ? exp2f(mr[rr] - m) : 0.f;
+                l += lr[rr] * wgt;
+                o += orr[rr] * wgt;
             }
             const float out = n > 0 ? o / l : 0.f;
             const int64_t oi = ((int64_t)b * a.Hq + (int64_t)hk * G + h) * D + tid;
