@@ -267,7 +267,7 @@ __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeArgs a)
 // One launch per call: a thread-block cluster per (sequence, KV head).
 //
 // The row's key blocks are dealt round-robin to the CTAs of the cluster (at most kRowMaxBlk each).
-// A CTA first requests all of its K and V blocks with one bulk copy per key row into shared
+// A CTA first requests all of its K and V blocks with 16-byte asynchronous copies into shared
 // memory (everything it will ever read is in flight at once), then takes them in order as they
 // land: logits and P V as in decode_block_kernel, with the running maximum, sum and output kept
 // in registers across blocks (online softmax).  The CTAs' partial results meet in shared memory:
@@ -284,6 +284,21 @@ struct RowSmem {
     static constexpr int kBlockBytes = 2 * kTile;              // K + V of one key block
 };
 
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+// Waits until at most `pending` of this thread's copy groups are still in flight.
+__device__ __forceinline__ void cp_async_wait(int pending)
+{
+    switch (pending) {
+        case 0: asm volatile("cp.async.wait_group 0;\n" ::: "memory"); break;
+        case 1: asm volatile("cp.async.wait_group 1;\n" ::: "memory"); break;
+        case 2: asm volatile("cp.async.wait_group 2;\n" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 3;\n" ::: "memory"); break;
+    }
+}
 __device__ __forceinline__ uint4 lds16(uint32_t addr)
 {
     uint4 r;
@@ -301,7 +316,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
     __shared__ float sS[kMaxGroup][kDecBlock + 8];  // base-2 logits of the current block
     __shared__ float sO[kMaxGroup][D];              // this CTA's unnormalised output
     __shared__ float sML[kMaxGroup][2];             // this CTA's running maximum and sum
-    __shared__ __align__(8) uint64_t s_bar[kRowMaxBlk];  // one per key block: its copies have landed
 
     cg::cluster_group cluster = cg::this_cluster();
     const int R = (int)gridDim.x, r = (int)blockIdx.x;  // the cluster spans grid x
@@ -345,41 +359,28 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
         jb[i] = __shfl_sync(0xffffffffu, cand, src & 31);
     }
 
-    // ---- all loads of this CTA at once: one bulk copy per key row of K and of V (thread = row),
-    // counted on one mbarrier per key block; rows past the sequence end are zero-filled instead.
+    // ---- all loads of this CTA at once, one copy group per key block; a thread copies one
+    // 16-byte piece of every eighth key row (rows past the sequence end are zero-filled)
     const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(row_smem);
-    const uint32_t bars0 = (uint32_t)__cvta_generic_to_shared(&s_bar[0]);
-    if (tid == 0) {
+    {
+        constexpr int NP = D / 8;                       // 16-byte pieces per row
+        constexpr int kRowsPerPass = kDecThreads / NP;  // key rows covered by one pass of the CTA
+        const int key0 = tid / NP, pc = tid % NP;
 #pragma unroll
-        for (int i = 0; i < kRowMaxBlk; ++i)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bars0 + 8 * i));
-        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-    }
-    __syncthreads();
+        for (int i = 0; i < kRowMaxBlk; ++i) {
+            if (i < mine) {
+                const int n_keys = jb[i] == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
+                const __nv_bfloat16 *kb = a.k + b * a.k_sb + ((int64_t)jb[i] * kDecBlock + key0) * a.k_ss + hk * a.k_sh + 8 * pc;
+                const __nv_bfloat16 *vb = a.v + b * a.v_sb + ((int64_t)jb[i] * kDecBlock + key0) * a.v_ss + hk * a.v_sh + 8 * pc;
+                const uint32_t sk = smem0 + i * SM::kBlockBytes + key0 * SM::kPitch + pc * 16, sv = sk + SM::kTile;
 #pragma unroll
-    for (int i = 0; i < kRowMaxBlk; ++i) {
-        if (i < mine) {
-            const int n_keys = jb[i] == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
-            const int key = tid & (kDecBlock - 1);
-            const bool is_v = tid >= kDecBlock;
-            const __nv_bfloat16 *src = is_v ? a.v + b * a.v_sb + ((int64_t)jb[i] * kDecBlock + key) * a.v_ss + hk * a.v_sh
-                                            : a.k + b * a.k_sb + ((int64_t)jb[i] * kDecBlock + key) * a.k_ss + hk * a.k_sh;
-            const uint32_t dst = smem0 + i * SM::kBlockBytes + (is_v ? SM::kTile : 0) + key * SM::kPitch;
-            if (key < n_keys) {
-                asm volatile(
-                    "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
-                    "l"(src), "r"((uint32_t)(D * 2)), "r"(bars0 + 8 * i)
-                    : "memory");
-            } else {
-#pragma unroll
-                for (int c = 0; c < D * 2 / 16; ++c)
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};\n" ::"r"(dst + 16 * c), "r"(0u) : "memory");
+                for (int q = 0; q < kDecBlock / kRowsPerPass; ++q) {
+                    const uint32_t bytes = key0 + q * kRowsPerPass < n_keys ? 16u : 0u;
+                    cp_async16(sk + q * kRowsPerPass * SM::kPitch, kb + (int64_t)q * kRowsPerPass * a.k_ss, bytes);
+                    cp_async16(sv + q * kRowsPerPass * SM::kPitch, vb + (int64_t)q * kRowsPerPass * a.v_ss, bytes);
+                }
+                cp_async_commit();
             }
-            if (tid == 0)
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bars0 + 8 * i),
-                             "r"((uint32_t)(n_keys * 2 * D * 2))
-                             : "memory");
         }
     }
 
@@ -405,19 +406,8 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
         const int32_t jblk = i == 0 ? jb[0] : i == 1 ? jb[1] : i == 2 ? jb[2] : jb[3];
         const int n_keys = jblk == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
         const uint32_t sk = smem0 + i * SM::kBlockBytes, sv_ = sk + SM::kTile;
-        // The block's copies have landed (bounded poll; they always do).
-        {
-            uint32_t done = 0;
-            for (uint32_t it = 0; !done && it < (1u << 26); ++it)
-                asm volatile(
-                    "{\n\t.reg .pred p;\n\t"
-                    "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
-                    "selp.u32 %0, 1, 0, p;\n\t}\n"
-                    : "=r"(done)
-                    : "r"(bars0 + 8 * i)
-                    : "memory");
-        }
-        __syncthreads();  // zero-filled rows are visible; sS is free again
+        cp_async_wait(mine - 1 - i);
+        __syncthreads();  // every thread's copies of this block have landed; sS is free again
 
         // ---- S = Q K^T: rows = heads, columns = the warp's 16 keys (two 8-key tiles)
         float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
