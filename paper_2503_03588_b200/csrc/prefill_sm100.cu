@@ -475,10 +475,21 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 // step's row sum, which is needed anyway: it bounds every p of the row from above,
                 // so a sum within the limit means no p came near the fp32 / bf16 range, and an
                 // overflow shows up as inf.
+                if (t == 0) {
+                    // A unit's first step: the reference is the exact row maximum of this block
+                    // (l and O are still empty, so nothing has to be rescaled), then the common pass.
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                    for (int c = 0; c < 64; c += 4) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) mx4[e] = fmaxf(mx4[e], __uint_as_float(sr[c + e]));
+                    }
+                    m = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
+                }
                 const uint64_t negm_2 = ptx::pack_f32x2(-m, -m);
                 uint64_t sum2[2] = {0ull, 0ull};
                 uint32_t pk[32];
-                if (t > 0) {  // the first step of a unit has no reference yet: straight to the exact path
+                {
 #pragma unroll
                 for (int c = 0; c < 64; c += 4) {
 #pragma unroll
@@ -502,7 +513,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     sum = (s0 + s1) + (s2 + s3);
                 }
                 // !(x <= limit) also catches inf and NaN.
-                const bool suspect = t == 0 || !(sum <= kSumLimit);
+                const bool suspect = !(sum <= kSumLimit);
                 if (__any_sync(0xffffffffu, suspect)) {
                     // Rare path: exact row maximum, new reference for the rows that need it, what
                     // was accumulated so far brought to the new reference, P recomputed from the
@@ -516,7 +527,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     const float mx2 = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
                     const bool grow = t == 0 || mx2 > m + kRescaleThreshold;
                     const float m_new = grow ? mx2 : m;
-                    const float alpha = grow ? ptx::ex2(m - m_new) : 1.0f;  // 0 on the first step
+                    const float alpha = grow ? ptx::ex2(m - m_new) : 1.0f;  // (l and O are still empty on a first step)
                     l *= alpha;
                     m = m_new;
                     if (t > 0) {
