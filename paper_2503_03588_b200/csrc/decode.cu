@@ -270,10 +270,9 @@ __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeArgs a)
 // A CTA first requests all of its K and V blocks with 16-byte asynchronous copies into shared
 // memory (everything it will ever read is in flight at once), then takes them in order as they
 // land: logits and P V as in decode_block_kernel, with the running maximum, sum and output kept
-// in registers across blocks (online softmax).  The partial results meet in shared memory: every
-// CTA pushes its partial for head h into CTA (h mod R) through distributed shared memory and
-// arrives on that CTA's mbarrier; CTA r merges heads r, r + R, ... once all R pushes have landed
-// and writes O and the LSE.  No workspace, no second launch.
+// in registers across blocks (online softmax).  The CTAs' partial results meet in shared memory:
+// after a cluster barrier CTA r merges the heads g = r, r + R, ... reading its peers' partials
+// through distributed shared memory, and writes O and the LSE.  No workspace, no second launch.
 // ------------------------------------------------------------------------------------------
 constexpr int kRowMaxBlk = 4;      // key blocks per CTA
 constexpr int kRowMaxCluster = 8;  // portable cluster size limit
@@ -315,10 +314,8 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
     constexpr int NJ = D / 32;  // 16-byte pieces per thread and row for Q and K
     extern __shared__ __align__(16) uint8_t row_smem[];
     __shared__ float sS[kMaxGroup][kDecBlock + 8];  // base-2 logits of the current block
-    // Partial results pushed here by the CTAs of the cluster for the heads this CTA merges:
-    // slot (head / R) * R + source rank holds o[D], m, l.  ceil(G / R) * R <= G + R - 1 slots.
-    __shared__ float sIn[kMaxGroup + kRowMaxCluster - 1][D + 2];
-    __shared__ __align__(8) uint64_t s_in_bar;      // R arrivals: every CTA's push has landed
+    __shared__ float sO[kMaxGroup][D];              // this CTA's unnormalised output
+    __shared__ float sML[kMaxGroup][2];             // this CTA's running maximum and sum
 
     cg::cluster_group cluster = cg::this_cluster();
     const int R = (int)gridDim.x, r = (int)blockIdx.x;  // the cluster spans grid x
@@ -365,14 +362,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
     // ---- all loads of this CTA at once, one copy group per key block; a thread copies one
     // 16-byte piece of every eighth key row (rows past the sequence end are zero-filled)
     const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(row_smem);
-    const uint32_t bar_in = (uint32_t)__cvta_generic_to_shared(&s_in_bar);
-    if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar_in), "r"((uint32_t)R));
-        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
-    }
-    __syncthreads();
-    // Tell the cluster that this CTA's mbarrier exists; the matching wait comes just before the push.
-    asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
     {
         constexpr int NP = D / 8;                       // 16-byte pieces per row
         constexpr int kRowsPerPass = kDecThreads / NP;  // key rows covered by one pass of the CTA
@@ -503,78 +492,64 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
         }
     }
 
-    // ---- merge across the cluster.  Head h is merged by CTA h mod R.  Every CTA pushes its
-    // partial result for a head (o, m, l) straight into the merging CTA's shared memory and then
-    // arrives on that CTA's mbarrier; the merging CTA waits for the R arrivals and combines from
-    // its own shared memory.  CTAs that merge nothing leave at once: nobody reads their memory.
-    asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");  // the peers' mbarriers are initialised
-    if (g < G) {
-        const uint32_t target = (uint32_t)(g % R);
-        float *in = cluster.map_shared_rank(&sIn[(g / R) * R + r][0], target);
-        if (pv_warp) {
+    // ---- this CTA's partial result to shared memory
+    if (pv_warp && g < G) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
+        for (int e = 0; e < 4; ++e)
 #pragma unroll
-                for (int x = 0; x < 2; ++x) {
-                    const int nn = 2 * t + x;
-                    in[8 * ((nn & 3) + 4 * wid) + e + 4 * (nn >> 2)] = acc[e][x];
-                }
-        }
-        if (wid == 0 && t == 0) {
-            in[D] = m_run;
-            in[D + 1] = l_run;
-        }
-    }
-    __syncthreads();
-    if (tid < R && tid < G) {
-        // One arrival per merging CTA, releasing this CTA's pushes at cluster scope.
-        uint32_t remote;
-        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(bar_in), "r"((uint32_t)tid));
-        asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];\n" ::"r"(remote) : "memory");
-    }
-    if (r < G) {
-        // (bounded poll: the arrivals always come)
-        uint32_t done = 0;
-        for (uint32_t it = 0; !done && it < (1u << 26); ++it)
-            asm volatile(
-                "{\n\t.reg .pred p;\n\t"
-                "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], 0;\n\t"
-                "selp.u32 %0, 1, 0, p;\n\t}\n"
-                : "=r"(done)
-                : "r"(bar_in)
-                : "memory");
-        if (tid < D) {
-            for (int h = r, hi = 0; h < G; h += R, ++hi) {
-                float mr[kRowMaxCluster], lr[kRowMaxCluster], orr[kRowMaxCluster];
-#pragma unroll
-                for (int rr = 0; rr < kRowMaxCluster; ++rr) {
-                    const float *src = sIn[hi * R + (rr < R ? rr : 0)];
-                    mr[rr] = src[D];
-                    lr[rr] = src[D + 1];
-                    orr[rr] = src[tid];
-                }
-                float m = -INFINITY;
-#pragma unroll
-                for (int rr = 0; rr < kRowMaxCluster; ++rr)
-                    if (rr < R) m = fmaxf(m, mr[rr]);
-                float l = 0.f, o = 0.f;
-#pragma unroll
-                for (int rr = 0; rr < kRowMaxCluster; ++rr) {
-                    const float wgt = (rr < R && mr[rr] != -INFINITY) ? exp2f(mr[rr] - m) : 0.f;
-                    l += lr[rr] * wgt;
-                    o += orr[rr] * wgt;
-                }
-                const float out = n > 0 ? o / l : 0.f;
-                const int64_t oi = ((int64_t)b * a.Hq + (int64_t)hk * G + h) * D + tid;
-                if (a.o_is_f32)
-                    reinterpret_cast<float *>(a.o)[oi] = out;
-                else
-                    reinterpret_cast<__nv_bfloat16 *>(a.o)[oi] = __float2bfloat16_rn(out);
-                if (tid == 0)
-                    a.lse[(int64_t)b * a.Hq + (int64_t)hk * G + h] = n > 0 ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+            for (int x = 0; x < 2; ++x) {
+                const int nn = 2 * t + x;
+                sO[g][8 * ((nn & 3) + 4 * wid) + e + 4 * (nn >> 2)] = acc[e][x];
             }
+    }
+    if (wid == 0 && t == 0 && g < G) {
+        sML[g][0] = m_run;
+        sML[g][1] = l_run;
+    }
+    cluster.sync();
+
+    // ---- merge across the cluster: CTA r takes heads r, r + R, ...; thread d one feature.  All
+    // remote reads of a head are issued before the first one is used (they are independent, and
+    // each costs a trip through the cluster's shared-memory network).
+    if (tid < D) {
+        const float *peer_ml[kRowMaxCluster];
+        const float *peer_o[kRowMaxCluster];
+#pragma unroll
+        for (int rr = 0; rr < kRowMaxCluster; ++rr) {
+            const int src = rr < R ? rr : r;  // (slots beyond the cluster are given weight 0 below)
+            peer_ml[rr] = cluster.map_shared_rank(&sML[0][0], src);
+            peer_o[rr] = cluster.map_shared_rank(&sO[0][0], src);
+        }
+        for (int h = r; h < G; h += R) {
+            float mr[kRowMaxCluster], lr[kRowMaxCluster], orr[kRowMaxCluster];
+#pragma unroll
+            for (int rr = 0; rr < kRowMaxCluster; ++rr) {
+                mr[rr] = peer_ml[rr][2 * h];
+                lr[rr] = peer_ml[rr][2 * h + 1];
+                orr[rr] = peer_o[rr][h * D + tid];
+            }
+            float m = -INFINITY;
+#pragma unroll
+            for (int rr = 0; rr < kRowMaxCluster; ++rr)
+                if (rr < R) m = fmaxf(m, mr[rr]);
+            float l = 0.f, o = 0.f;
+#pragma unroll
+            for (int rr = 0; rr < kRowMaxCluster; ++rr) {
+                const float wgt = (rr < R && mr[rr] != -INFINITY) ? exp2f(mr[rr] - m) : 0.f;
+                l += lr[rr] * wgt;
+                o += orr[rr] * wgt;
+            }
+            const float out = n > 0 ? o / l : 0.f;
+            const int64_t oi = ((int64_t)b * a.Hq + (int64_t)hk * G + h) * D + tid;
+            if (a.o_is_f32)
+                reinterpret_cast<float *>(a.o)[oi] = out;
+            else
+                reinterpret_cast<__nv_bfloat16 *>(a.o)[oi] = __float2bfloat16_rn(out);
+            if (tid == 0)
+                a.lse[(int64_t)b * a.Hq + (int64_t)hk * G + h] = n > 0 ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
         }
     }
+    cluster.sync();  // peers may still be reading this CTA's shared memory
 }
 
 __global__ void decode_block_list_kernel(int64_t len, int32_t W, int32_t S, int32_t *out,
