@@ -322,6 +322,46 @@ def run_ours(args):
     dec_us = 1e3 * d0.elapsed_time(d1) / (n_sets * reps)
     dec_gbs = dec_bytes / (dec_us * 1e-6) / 1e9
 
+    # ---- decode scale-up (labelled, beside the batch-8 figure): the same per-sequence pattern at
+    # larger batches, where one call moves enough bytes to outlast its launch.  Caches are drawn on
+    # the device (values do not matter for bandwidth); lengths are seeded like the batch-8 sets.
+    scale_up = []
+    if not args.no_decode_scale_up:
+        for big in (64, 256):
+            cache_bytes = 2 * big * wd.max_len * wd.n_kv_heads * wd.head_dim * 2
+            if torch.cuda.mem_get_info(dev)[0] < cache_bytes + (8 << 30):
+                continue
+            gen = torch.Generator(device=dev)
+            gen.manual_seed(wd.seed + big)
+            kcb = torch.randn((big, wd.max_len, wd.n_kv_heads, wd.head_dim), device=dev, dtype=torch.bfloat16, generator=gen)
+            vcb = torch.randn((big, wd.max_len, wd.n_kv_heads, wd.head_dim), device=dev, dtype=torch.bfloat16, generator=gen)
+            qb = torch.randn((big, wd.n_q_heads, wd.head_dim), device=dev, dtype=torch.bfloat16, generator=gen)
+            rngb = np.random.Generator(np.random.PCG64(wd.lens_seed + big))
+            sets_b = [rngb.integers(wd.min_len, wd.max_len + 1, size=big, dtype=np.int64) for _ in range(4)]
+            sets_bd = [torch.as_tensor(x, dtype=torch.int32, device=dev) for x in sets_b]
+            bytes_b = float(np.mean([touched_bytes(ls) for ls in sets_b]))
+            ob, lb, wsb = pa.pa_decode(qb, kcb, vcb, sets_bd[0], wd.window_blocks, wd.sink_blocks)
+            with torch.cuda.stream(side):
+                torch.cuda.synchronize()
+                gb = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gb, stream=side):
+                    for _ in range(4):
+                        for ld in sets_bd:
+                            pa.pa_decode(qb, kcb, vcb, ld, wd.window_blocks, wd.sink_blocks, o=ob, lse=lb, workspace=wsb)
+                gb.replay()
+                torch.cuda.synchronize()
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record(side)
+                gb.replay()
+                g1.record(side)
+                torch.cuda.synchronize()
+            us_b = 1e3 * g0.elapsed_time(g1) / 16
+            scale_up.append(dict(batch=big, us_per_call=us_b, kv_bytes_per_call=bytes_b,
+                                 value=bytes_b / (us_b * 1e-6) / 1e9, unit="GB/s",
+                                 frac=bytes_b / (us_b * 1e-6) / 1e9 / peaks["hbm_gbs"]))
+            del kcb, vcb, qb, ob, lb, wsb, gb
+            torch.cuda.empty_cache()
+
     # ---- end to end through the public API with host buffers: pinned H2D of Q, K, V, the call,
     # D2H of O and LSE, all inside the timed region.  Consecutive steps overlap as a serving loop
     # would run them: the copies in of step i+1 and the copies out of step i-1 travel while step i
@@ -407,7 +447,7 @@ def run_ours(args):
                 decode=dict(metric="decode_kv_gbs", value=dec_gbs, unit="GB/s", us_per_call=dec_us,
                             kv_bytes_per_call=dec_bytes, peak=peaks["hbm_gbs"], frac=dec_gbs / peaks["hbm_gbs"],
                             bound="hbm", timing=f"CUDA graph of {n_sets * reps} calls rotating over {n_sets} seeded length sets",
-                            workload=wd.name),
+                            workload=wd.name, scale_up=scale_up),
                 e2e=dict(value=flops / (e2e_ms * 1e-3) / 1e12, unit=UNIT, ms_per_step=e2e_ms,
                          h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps,
                          overlap="copies in, compute and copies out of consecutive steps overlap (3 streams)"),
@@ -523,6 +563,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode-scale-up", action="store_true", help="skip the batch-64/256 decode lines")
     ap.add_argument("--case", default=None, choices=["prefill32k", "decode"],
                     help="run only a small single-kernel case (for profiler captures)")
     ap.add_argument("--sweep", action="store_true", help="sequence-length sweep with comparison layouts")
