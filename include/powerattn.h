@@ -146,8 +146,9 @@ size_t pa_decode_workspace_bytes(const pa_decode_params *p);
  * strides.  cache_lens: device int32 [batch], each in [1, max_len] (a length outside that
  * range makes the sequence's outputs zero and its LSE -inf; nothing faults).
  * o: device [batch, n_q_heads, head_dim] contiguous, o_dtype.  lse: device fp32
- * [batch, n_q_heads].  When no row can list more than 32 key blocks (any default-window row up
- * to millions of tokens) one kernel is enqueued: a thread-block cluster per (sequence, KV head)
+ * [batch, n_q_heads].  When a row's window, power-of-two and sink candidates number at most 32
+ * (window_blocks + sink_blocks + log2 of the row count: any default-window row up to millions of
+ * tokens) one kernel is enqueued: a thread-block cluster per (sequence, KV head)
  * shares the row's blocks, each CTA runs an online softmax over its blocks, and the partial
  * results are merged inside the cluster with the log-sum-exp rule
  * m = max m_c, l = sum l_c e^(m_c - m), o = sum o_c e^(m_c - m) / l; the workspace is then not

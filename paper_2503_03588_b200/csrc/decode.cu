@@ -1,8 +1,8 @@
 // pa_decode: one query token per sequence against its KV cache under the PowerAttention row of
 // its position (Section 4.1: same pattern in prefilling and decoding; Eq. (1) for the row).
 //
-// Two paths.  Rows of at most 32 listed blocks (every PowerAttention row with the default window
-// up to millions of tokens) take decode_row_kernel: one launch, a thread-block cluster per
+// Two paths.  Rows with at most 32 window, power-of-two and sink candidates (every PowerAttention
+// row with the default window up to millions of tokens) take decode_row_kernel: one launch, a thread-block cluster per
 // (sequence, KV head), described at that kernel.  Longer rows take the split-K pair below.
 //
 // Split-K: one CTA per (sequence, KV head, chunk) where a chunk is one 64-key block of the
@@ -562,6 +562,18 @@ __global__ void decode_block_list_kernel(int64_t len, int32_t W, int32_t S, int3
     *count = n;
 }
 
+// Window distances + power-of-two distances beyond the window + sink blocks that a row below
+// n_rows can have, before any of them coincide or fall off the sequence start: the number of
+// candidate slots the cluster kernel enumerates (one per lane, so it needs this to be <= 32).
+static int64_t row_candidate_slots(int64_t n_rows, int32_t W, int32_t S)
+{
+    const int64_t w = W > 1 ? W : 1;
+    int powers = 0;
+    for (int64_t pw = 1; pw <= n_rows - 1; pw *= 2)
+        if (pw >= w) ++powers;
+    return w + S + powers;
+}
+
 // Upper bound on the number of listed blocks of any row below n_rows.
 static int max_row_blocks(int64_t n_rows, int32_t W, int32_t S)
 {
@@ -667,7 +679,8 @@ extern "C" pa_status pa_decode(const pa_decode_params *p, const void *q, const v
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // Rows short enough for one cluster per (sequence, KV head) take the single-launch path.
-    if (decode_path() != 1 && a.chunks <= kRowMaxBlk * kRowMaxCluster) {
+    if (decode_path() != 1 && row_candidate_slots(rows, p->window_blocks, p->sink_blocks) <= 32 &&
+        a.chunks <= kRowMaxBlk * kRowMaxCluster) {
         int R = decode_cluster();
         if (R * kRowMaxBlk < a.chunks) R = (a.chunks + kRowMaxBlk - 1) / kRowMaxBlk;
         if (R > a.chunks) R = a.chunks;

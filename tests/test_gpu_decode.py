@@ -100,3 +100,15 @@ def test_decode_paths(pa, oracle, monkeypatch, env):
     lens = np.array([9000, 8193, 130, 7])
     _run(pa, oracle, q, kc, vc, lens, 5, 1)
     _run(pa, oracle, q, kc, vc, lens, 3, 2, o_dtype=torch.float32)
+
+
+def test_decode_short_cache_with_wide_window_and_sinks(pa, oracle):
+    """A cache of 32 blocks whose window + sink candidates exceed 32: the bound on listed blocks is
+    clamped by the row count, the candidate count is not (the library must pick its path by the
+    latter)."""
+    batch, max_len, Hq, Hkv, D = 3, 2048, 14, 2, 128
+    q = si.bf16_randn((batch, Hq, D), 41)
+    kc, vc = si.bf16_randn((batch, max_len, Hkv, D), 42), si.bf16_randn((batch, max_len, Hkv, D), 43)
+    lens = np.array([2048, 1999, 700])
+    _run(pa, oracle, q, kc, vc, lens, 30, 4)
+    _run(pa, oracle, q, kc, vc, lens, 26, 4)   # 26 + 4 + 0 powers = 30 candidates: the cluster path
