@@ -111,7 +111,12 @@ size_t pa_prefill_workspace_bytes(const pa_prefill_params *p);
  * workspace: device, >= pa_prefill_workspace_bytes(p); cleared by the call itself.
  * Enqueues one memset and one kernel.  Errors: PA_ERR_INVALID_ARG, PA_ERR_SHAPE,
  * PA_ERR_ALIGNMENT, PA_ERR_LAYOUT (nnz < n_qblocks), PA_ERR_WORKSPACE, PA_ERR_UNSUPPORTED,
- * PA_ERR_CUDA.  Outputs are undefined after a failure. */
+ * PA_ERR_CUDA.  Outputs are undefined after a failure.  The CSR is trusted: extents that point
+ * outside col_idx would be read out of bounds.  With PA_VALIDATE=1 in the environment the call
+ * first checks it on the device (row_ptr from 0 to nnz, extents inside col_idx, every index in
+ * [0, row] and ascending within its row), synchronises the stream, and returns PA_ERR_LAYOUT with
+ * the first offending row in pa_last_error_message() instead of enqueuing the kernel; do not
+ * use that switch while capturing the stream. */
 pa_status pa_prefill(const pa_prefill_params *p, const void *q, const void *k, const void *v,
                      const int32_t *row_ptr, const int32_t *col_idx, int64_t nnz, void *o,
                      float *lse, void *workspace, size_t workspace_bytes, void *stream);

@@ -23,6 +23,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <math.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -802,6 +803,30 @@ static pa_status check_prefill(const pa_prefill_params *p)
 
 constexpr size_t kPrefillWorkspace = 256;
 
+// Optional check of a caller's CSR (PA_VALIDATE=1): one thread per row.  The first violation
+// found is recorded as (kind, row) in check[0..1]: 1 row_ptr does not start at 0 / end at nnz,
+// 2 row extent negative or beyond nnz, 3 block index outside [0, row], 4 indices not ascending.
+__global__ void validate_csr_kernel(const int32_t *row_ptr, const int32_t *col_idx, int32_t nqb, int64_t nnz,
+                                    int32_t *check)
+{
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nqb) return;
+    int kind = 0;
+    const int32_t lo = row_ptr[i], hi = row_ptr[i + 1];
+    if ((i == 0 && lo != 0) || (i == nqb - 1 && (int64_t)hi != nnz)) kind = 1;
+    else if (lo < 0 || hi < lo || (int64_t)hi > nnz) kind = 2;
+    else {
+        int32_t prev = -1;
+        for (int32_t e = lo; e < hi && kind == 0; ++e) {
+            const int32_t j = col_idx[e];
+            if (j < 0 || j > i) kind = 3;
+            else if (j <= prev) kind = 4;
+            prev = j;
+        }
+    }
+    if (kind != 0 && atomicCAS(check, 0, kind) == 0) check[1] = i;
+}
+
 }  // namespace pa
 
 extern "C" size_t pa_prefill_workspace_bytes(const pa_prefill_params *p)
@@ -868,6 +893,24 @@ extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const
     const unsigned grid = (unsigned)(a.n_units < sms ? a.n_units : sms);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     PA_CUDA_OK(cudaMemsetAsync(workspace, 0, kPrefillWorkspace, st));
+    {
+        // PA_VALIDATE=1: check the CSR on the device before the attention kernel is enqueued.  This
+        // synchronises the stream (so not during stream capture) and is meant for bring-up: a CSR
+        // whose extents point outside col_idx would otherwise be read out of bounds.
+        const char *e = getenv("PA_VALIDATE");
+        if (e && e[0] == '1') {
+            int32_t *check = static_cast<int32_t *>(workspace) + 32;
+            validate_csr_kernel<<<(unsigned)((nqb + 127) / 128), 128, 0, st>>>(row_ptr, col_idx, (int32_t)nqb, nnz, check);
+            PA_CUDA_OK(cudaGetLastError());
+            int32_t found[2] = {0, 0};
+            PA_CUDA_OK(cudaMemcpyAsync(found, check, sizeof(found), cudaMemcpyDeviceToHost, st));
+            PA_CUDA_OK(cudaStreamSynchronize(st));
+            static const char *const what[] = {"", "row_ptr must start at 0 and end at nnz", "row extent negative or beyond nnz",
+                                               "block index outside [0, row]", "block indices of a row must ascend"};
+            if (found[0] >= 1 && found[0] <= 4)
+                return fail(PA_ERR_LAYOUT, "CSR check: %s (row %d)", what[found[0]], (int)found[1]);
+        }
+    }
     if (D == 128) {
         PA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)SmemMap<128>::kAlloc));

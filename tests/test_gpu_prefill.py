@@ -135,3 +135,30 @@ def test_full_size_workloads_on_sampled_rows(pa, oracle, w):
     st = compare(o[:, ridx], lse[:, :, ridx], o_ref, lse_ref, w.name)
     print(w.name, st)
     assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+
+
+def test_csr_check_switch_rejects_malformed_layouts(pa, monkeypatch):
+    """PA_VALIDATE=1 makes pa_prefill check the caller's CSR on the device before any attention
+    work: each kind of violation comes back as PA_ERR_LAYOUT, and a good layout still runs."""
+    monkeypatch.setenv("PA_VALIDATE", "1")
+    N, Hq, Hkv, D = 1024, 4, 2, 64
+    Q = si.bf16_randn((1, N, Hq, D), 51).cuda()
+    K = si.bf16_randn((1, N, Hkv, D), 52).cuda()
+    V = si.bf16_randn((1, N, Hkv, D), 53).cuda()
+    rp, ci = pa.pa_build_layout(N, 64, 2, 1)
+    pa.pa_prefill(Q, K, V, rp, ci)  # passes the check
+    torch.cuda.synchronize()
+
+    def expect_layout_error(rp_bad, ci_bad):
+        with pytest.raises(pa.PaError) as err:
+            pa.pa_prefill(Q, K, V, rp_bad, ci_bad)
+        assert "PA_ERR_LAYOUT" in str(err.value) or "CSR check" in str(err.value)
+
+    bad = ci.clone(); bad[int(rp[5])] = 9          # a block after the row (non-causal)
+    expect_layout_error(rp, bad)
+    bad = ci.clone(); bad[int(rp[7]) + 1] = bad[int(rp[7])]  # not ascending
+    expect_layout_error(rp, bad)
+    bad = rp.clone(); bad[3] = bad[4] + 1           # negative extent
+    expect_layout_error(bad, ci)
+    bad = rp.clone(); bad[0] = 1                    # does not start at 0
+    expect_layout_error(bad, ci)
