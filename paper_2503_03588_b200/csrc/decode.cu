@@ -34,6 +34,7 @@ struct DecodeArgs {
     int64_t k_sb, k_ss, k_sh, v_sb, v_ss, v_sh;
     int64_t max_len;
     int32_t batch, Hq, Hkv, G, W, S, chunks, o_is_f32;
+    int32_t stages;  // (cluster kernel) shared-memory stages of this launch
     float scale_log2;  // softmax_scale * log2(e)
 };
 
@@ -266,15 +267,15 @@ __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeArgs a)
 // ------------------------------------------------------------------------------------------
 // One launch per call: a thread-block cluster per (sequence, KV head).
 //
-// The row's key blocks are dealt round-robin to the CTAs of the cluster (at most kRowMaxBlk each).
-// A CTA first requests all of its K and V blocks with 16-byte asynchronous copies into shared
-// memory (everything it will ever read is in flight at once), then takes them in order as they
+// The row's key blocks are dealt round-robin to the CTAs of the cluster.  A CTA requests its K and
+// V blocks with 16-byte asynchronous copies into a ring of shared-memory stages (with few blocks
+// per CTA everything it will ever read is in flight at once), then takes them in order as they
 // land: logits and P V as in decode_block_kernel, with the running maximum, sum and output kept
 // in registers across blocks (online softmax).  The CTAs' partial results meet in shared memory:
 // after a cluster barrier CTA r merges the heads g = r, r + R, ... reading its peers' partials
 // through distributed shared memory, and writes O and the LSE.  No workspace, no second launch.
 // ------------------------------------------------------------------------------------------
-constexpr int kRowMaxBlk = 4;      // key blocks per CTA
+constexpr int kRowMaxStages = 4;   // shared-memory stages (key blocks in flight) per CTA
 constexpr int kRowMaxCluster = 8;  // portable cluster size limit
 
 template <int D>
@@ -350,39 +351,37 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
     }
     const uint32_t have = __ballot_sync(0xffffffffu, cand >= 0);
     const int n = __popc(have);
-    int mine = n > r ? (n - r + R - 1) / R : 0;
-    if (mine > kRowMaxBlk) mine = kRowMaxBlk;  // (the host sizes the cluster so that this never cuts)
-    int32_t jb[kRowMaxBlk];
-#pragma unroll
-    for (int i = 0; i < kRowMaxBlk; ++i) {
-        const int src = i < mine ? (int)__fns(have, 0, r + i * R + 1) : 0;
-        jb[i] = __shfl_sync(0xffffffffu, cand, src & 31);
-    }
+    const int mine = n > r ? (n - r + R - 1) / R : 0;
+    // Key block number i of this CTA: the (r + i R)-th candidate that exists.
+    auto block_of = [&](int i) {
+        const int src = (int)__fns(have, 0, r + i * R + 1);
+        return __shfl_sync(0xffffffffu, cand, src & 31);
+    };
 
-    // ---- all loads of this CTA at once, one copy group per key block; a thread copies one
-    // 16-byte piece of every eighth key row (rows past the sequence end are zero-filled)
+    // ---- loads: one copy group per key block into a ring of `stages` shared-memory stages, as many
+    // blocks in flight as there are stages (all of the CTA's blocks when they fit); a thread
+    // copies one 16-byte piece of every eighth key row (rows past the sequence end are zero-filled)
     const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(row_smem);
-    {
+    const int stages = a.stages;
+    auto issue_block = [&](int i) {
         constexpr int NP = D / 8;                       // 16-byte pieces per row
         constexpr int kRowsPerPass = kDecThreads / NP;  // key rows covered by one pass of the CTA
         const int key0 = tid / NP, pc = tid % NP;
+        const int32_t j = block_of(i);
+        const int n_keys = j == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
+        const __nv_bfloat16 *kb = a.k + b * a.k_sb + ((int64_t)j * kDecBlock + key0) * a.k_ss + hk * a.k_sh + 8 * pc;
+        const __nv_bfloat16 *vb = a.v + b * a.v_sb + ((int64_t)j * kDecBlock + key0) * a.v_ss + hk * a.v_sh + 8 * pc;
+        const uint32_t sk = smem0 + (i % stages) * SM::kBlockBytes + key0 * SM::kPitch + pc * 16, sv = sk + SM::kTile;
 #pragma unroll
-        for (int i = 0; i < kRowMaxBlk; ++i) {
-            if (i < mine) {
-                const int n_keys = jb[i] == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
-                const __nv_bfloat16 *kb = a.k + b * a.k_sb + ((int64_t)jb[i] * kDecBlock + key0) * a.k_ss + hk * a.k_sh + 8 * pc;
-                const __nv_bfloat16 *vb = a.v + b * a.v_sb + ((int64_t)jb[i] * kDecBlock + key0) * a.v_ss + hk * a.v_sh + 8 * pc;
-                const uint32_t sk = smem0 + i * SM::kBlockBytes + key0 * SM::kPitch + pc * 16, sv = sk + SM::kTile;
-#pragma unroll
-                for (int q = 0; q < kDecBlock / kRowsPerPass; ++q) {
-                    const uint32_t bytes = key0 + q * kRowsPerPass < n_keys ? 16u : 0u;
-                    cp_async16(sk + q * kRowsPerPass * SM::kPitch, kb + (int64_t)q * kRowsPerPass * a.k_ss, bytes);
-                    cp_async16(sv + q * kRowsPerPass * SM::kPitch, vb + (int64_t)q * kRowsPerPass * a.v_ss, bytes);
-                }
-                cp_async_commit();
-            }
+        for (int q = 0; q < kDecBlock / kRowsPerPass; ++q) {
+            const uint32_t bytes = key0 + q * kRowsPerPass < n_keys ? 16u : 0u;
+            cp_async16(sk + q * kRowsPerPass * SM::kPitch, kb + (int64_t)q * kRowsPerPass * a.k_ss, bytes);
+            cp_async16(sv + q * kRowsPerPass * SM::kPitch, vb + (int64_t)q * kRowsPerPass * a.v_ss, bytes);
         }
-    }
+        cp_async_commit();
+    };
+    int issued = 0;
+    for (; issued < mine && issued < stages; ++issued) issue_block(issued);
 
     uint4 qr[NJ];
     {
@@ -403,11 +402,15 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
 
 #pragma unroll 1
     for (int i = 0; i < mine; ++i) {
-        const int32_t jblk = i == 0 ? jb[0] : i == 1 ? jb[1] : i == 2 ? jb[2] : jb[3];
+        const int32_t jblk = block_of(i);
         const int n_keys = jblk == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
-        const uint32_t sk = smem0 + i * SM::kBlockBytes, sv_ = sk + SM::kTile;
-        cp_async_wait(mine - 1 - i);
-        __syncthreads();  // every thread's copies of this block have landed; sS is free again
+        const uint32_t sk = smem0 + (i % stages) * SM::kBlockBytes, sv_ = sk + SM::kTile;
+        cp_async_wait(issued - 1 - i);
+        __syncthreads();  // every thread's copies of this block have landed; sS and the stage of block i - 1 are free
+        if (i >= 1 && issued < mine) {
+            issue_block(issued);  // into the stage block i - 1 has just left
+            ++issued;
+        }
 
         // ---- S = Q K^T: rows = heads, columns = the warp's 16 keys (two 8-key tiles)
         float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -587,17 +590,25 @@ static int max_row_blocks(int64_t n_rows, int32_t W, int32_t S)
 }
 
 // PA_DECODE_PATH=splitk forces the two-launch split-K path (tests use it to cover that path on
-// workloads the cluster path would take); PA_DECODE_CLUSTER=n sets the cluster size (1..8).
+// workloads the cluster path would take); PA_DECODE_CLUSTER=n sets the cluster size (1..8)
+// instead of the choice by batch size.
 static int decode_path()
 {
     const char *e = getenv("PA_DECODE_PATH");
     return e && e[0] == 's' ? 1 : 0;
 }
-static int decode_cluster()
+static int decode_cluster()  // 0: chosen from the batch size
 {
     const char *e = getenv("PA_DECODE_CLUSTER");
     const int v = e ? atoi(e) : 0;
-    return v >= 1 && v <= kRowMaxCluster ? v : kRowMaxCluster;
+    return v >= 1 && v <= kRowMaxCluster ? v : 0;
+}
+// PA_DECODE_STAGES=n (1..4): shared-memory stages per CTA of the cluster kernel.
+static int decode_stages()
+{
+    const char *e = getenv("PA_DECODE_STAGES");
+    const int v = e ? atoi(e) : 0;
+    return v >= 1 && v <= kRowMaxStages ? v : kRowMaxStages;
 }
 
 
@@ -674,17 +685,29 @@ extern "C" pa_status pa_decode(const pa_decode_params *p, const void *q, const v
     const int64_t rows = (p->max_len + kDecBlock - 1) / kDecBlock;
     a.chunks = max_row_blocks(rows, p->window_blocks, p->sink_blocks);
     a.o_is_f32 = p->o_dtype == PA_F32;
+    a.stages = 0;
     const float scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // Rows short enough for one cluster per (sequence, KV head) take the single-launch path.
-    if (decode_path() != 1 && row_candidate_slots(rows, p->window_blocks, p->sink_blocks) <= 32 &&
-        a.chunks <= kRowMaxBlk * kRowMaxCluster) {
+    if (decode_path() != 1 && row_candidate_slots(rows, p->window_blocks, p->sink_blocks) <= 32) {
+        // Cluster size: enough CTAs to fill the GPU about three times over at small batches (the call
+        // is latency-bound there and short CTAs help), one CTA per row at large ones (no merge).
+        int dev = 0, sms = 0;
+        PA_CUDA_OK(cudaGetDevice(&dev));
+        PA_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        const int64_t rows_in_call = (int64_t)a.batch * a.Hkv;
         int R = decode_cluster();
-        if (R * kRowMaxBlk < a.chunks) R = (a.chunks + kRowMaxBlk - 1) / kRowMaxBlk;
+        if (R == 0) {
+            R = (int)((3 * (int64_t)sms + rows_in_call - 1) / rows_in_call);
+            if (R > kRowMaxCluster) R = kRowMaxCluster;
+            if (R < 1) R = 1;
+        }
         if (R > a.chunks) R = a.chunks;
         const int per_cta = (a.chunks + R - 1) / R;
+        a.stages = per_cta < decode_stages() ? per_cta : decode_stages();
+        const int smem_stages = a.stages;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)R, (unsigned)a.Hkv, (unsigned)a.batch);
         cfg.blockDim = dim3(kDecThreads, 1, 1);
@@ -697,20 +720,20 @@ extern "C" pa_status pa_decode(const pa_decode_params *p, const void *q, const v
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         if (p->head_dim == 128) {
-            cfg.dynamicSmemBytes = (size_t)per_cta * RowSmem<128>::kBlockBytes;
+            cfg.dynamicSmemBytes = (size_t)smem_stages * RowSmem<128>::kBlockBytes;
             static bool sized128 = false;  // (idempotent: a race between threads only repeats the call)
             if (!sized128) {
                 PA_CUDA_OK(cudaFuncSetAttribute(decode_row_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                kRowMaxBlk * RowSmem<128>::kBlockBytes));
+                                                kRowMaxStages * RowSmem<128>::kBlockBytes));
                 sized128 = true;
             }
             PA_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_row_kernel<128>, a));
         } else {
-            cfg.dynamicSmemBytes = (size_t)per_cta * RowSmem<64>::kBlockBytes;
+            cfg.dynamicSmemBytes = (size_t)smem_stages * RowSmem<64>::kBlockBytes;
             static bool sized64 = false;
             if (!sized64) {
                 PA_CUDA_OK(cudaFuncSetAttribute(decode_row_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                kRowMaxBlk * RowSmem<64>::kBlockBytes));
+                                                kRowMaxStages * RowSmem<64>::kBlockBytes));
                 sized64 = true;
             }
             PA_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_row_kernel<64>, a));
