@@ -307,7 +307,7 @@ __device__ __forceinline__ uint4 lds16(uint32_t addr)
     return r;
 }
 
-template <int D>
+template <int D, bool kRing>
 __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArgs a)
 {
     namespace cg = cooperative_groups;
@@ -352,17 +352,30 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
     const uint32_t have = __ballot_sync(0xffffffffu, cand >= 0);
     const int n = __popc(have);
     const int mine = n > r ? (n - r + R - 1) / R : 0;
-    // Key block number i of this CTA: the (r + i R)-th candidate that exists.
-    auto block_of = [&](int i) {
-        const int src = (int)__fns(have, 0, r + i * R + 1);
-        return __shfl_sync(0xffffffffu, cand, src & 31);
+    // Key block number i of this CTA: the (r + i R)-th candidate that exists.  Without the ring a
+    // CTA has at most kRowMaxStages blocks and keeps their indices in registers.
+    int32_t jb[kRowMaxStages];
+    if constexpr (!kRing) {
+#pragma unroll
+        for (int i = 0; i < kRowMaxStages; ++i) {
+            const int src = i < mine ? (int)__fns(have, 0, r + i * R + 1) : 0;
+            jb[i] = __shfl_sync(0xffffffffu, cand, src & 31);
+        }
+    }
+    auto block_of = [&](int i) -> int32_t {
+        if constexpr (!kRing) {
+            return i == 0 ? jb[0] : i == 1 ? jb[1] : i == 2 ? jb[2] : jb[3];
+        } else {
+            const int src = (int)__fns(have, 0, r + i * R + 1);
+            return __shfl_sync(0xffffffffu, cand, src & 31);
+        }
     };
 
-    // ---- loads: one copy group per key block into a ring of `stages` shared-memory stages, as many
-    // blocks in flight as there are stages (all of the CTA's blocks when they fit); a thread
-    // copies one 16-byte piece of every eighth key row (rows past the sequence end are zero-filled)
+    // ---- loads: one copy group per key block; a thread copies one 16-byte piece of every eighth
+    // key row (rows past the sequence end are zero-filled).  Without the ring every block has its
+    // own stage and all are requested here; with it, `stages` blocks are in flight at a time.
     const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(row_smem);
-    const int stages = a.stages;
+    const int stages = kRing ? a.stages : kRowMaxStages;
     auto issue_block = [&](int i) {
         constexpr int NP = D / 8;                       // 16-byte pieces per row
         constexpr int kRowsPerPass = kDecThreads / NP;  // key rows covered by one pass of the CTA
@@ -381,7 +394,14 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
         cp_async_commit();
     };
     int issued = 0;
-    for (; issued < mine && issued < stages; ++issued) issue_block(issued);
+    if constexpr (!kRing) {
+#pragma unroll
+        for (int i = 0; i < kRowMaxStages; ++i)
+            if (i < mine) issue_block(i);
+        issued = mine;
+    } else {
+        for (; issued < mine && issued < stages; ++issued) issue_block(issued);
+    }
 
     uint4 qr[NJ];
     {
@@ -407,9 +427,11 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
         const uint32_t sk = smem0 + (i % stages) * SM::kBlockBytes, sv_ = sk + SM::kTile;
         cp_async_wait(issued - 1 - i);
         __syncthreads();  // every thread's copies of this block have landed; sS and the stage of block i - 1 are free
-        if (i >= 1 && issued < mine) {
-            issue_block(issued);  // into the stage block i - 1 has just left
-            ++issued;
+        if constexpr (kRing) {
+            if (i >= 1 && issued < mine) {
+                issue_block(issued);  // into the stage block i - 1 has just left
+                ++issued;
+            }
         }
 
         // ---- S = Q K^T: rows = heads, columns = the warp's 16 keys (two 8-key tiles)
@@ -604,11 +626,11 @@ static int decode_cluster()  // 0: chosen from the batch size
     return v >= 1 && v <= kRowMaxCluster ? v : 0;
 }
 // PA_DECODE_STAGES=n (1..4): shared-memory stages per CTA of the cluster kernel.
-static int decode_stages()
+static int decode_stages()  // 0: chosen from the cluster size
 {
     const char *e = getenv("PA_DECODE_STAGES");
     const int v = e ? atoi(e) : 0;
-    return v >= 1 && v <= kRowMaxStages ? v : kRowMaxStages;
+    return v >= 1 && v <= kRowMaxStages ? v : 0;
 }
 
 
@@ -704,9 +726,15 @@ extern "C" pa_status pa_decode(const pa_decode_params *p, const void *q, const v
             if (R > kRowMaxCluster) R = kRowMaxCluster;
             if (R < 1) R = 1;
         }
+        const bool widest = R == kRowMaxCluster;  // a small call: as many CTAs per row as a cluster allows
         if (R > a.chunks) R = a.chunks;
         const int per_cta = (a.chunks + R - 1) / R;
-        a.stages = per_cta < decode_stages() ? per_cta : decode_stages();
+        // Few blocks per CTA: every block gets its own stage and all copies start at once (best for
+        // the latency of a small call).  Many: one stage per CTA by default, so that six CTAs share
+        // an SM and keep its memory pipe full (best for throughput; measured).
+        const bool ring = decode_stages() != 0 || per_cta > kRowMaxStages || !widest;
+        a.stages = ring ? (decode_stages() != 0 ? decode_stages() : 1) : per_cta;
+        if (a.stages > per_cta) a.stages = per_cta;
         const int smem_stages = a.stages;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)R, (unsigned)a.Hkv, (unsigned)a.batch);
@@ -719,24 +747,26 @@ extern "C" pa_status pa_decode(const pa_decode_params *p, const void *q, const v
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
+        // (setting the limit is idempotent: a race between threads only repeats the call)
+        static bool sized = false;
+        if (!sized) {
+            PA_CUDA_OK(cudaFuncSetAttribute(decode_row_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            kRowMaxStages * RowSmem<128>::kBlockBytes));
+            PA_CUDA_OK(cudaFuncSetAttribute(decode_row_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            kRowMaxStages * RowSmem<128>::kBlockBytes));
+            PA_CUDA_OK(cudaFuncSetAttribute(decode_row_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            kRowMaxStages * RowSmem<64>::kBlockBytes));
+            PA_CUDA_OK(cudaFuncSetAttribute(decode_row_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            kRowMaxStages * RowSmem<64>::kBlockBytes));
+            sized = true;
+        }
+        cfg.dynamicSmemBytes = (size_t)smem_stages * (p->head_dim == 128 ? RowSmem<128>::kBlockBytes : RowSmem<64>::kBlockBytes);
         if (p->head_dim == 128) {
-            cfg.dynamicSmemBytes = (size_t)smem_stages * RowSmem<128>::kBlockBytes;
-            static bool sized128 = false;  // (idempotent: a race between threads only repeats the call)
-            if (!sized128) {
-                PA_CUDA_OK(cudaFuncSetAttribute(decode_row_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                kRowMaxStages * RowSmem<128>::kBlockBytes));
-                sized128 = true;
-            }
-            PA_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_row_kernel<128>, a));
+            if (ring) PA_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_row_kernel<128, true>, a));
+            else PA_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_row_kernel<128, false>, a));
         } else {
-            cfg.dynamicSmemBytes = (size_t)smem_stages * RowSmem<64>::kBlockBytes;
-            static bool sized64 = false;
-            if (!sized64) {
-                PA_CUDA_OK(cudaFuncSetAttribute(decode_row_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                kRowMaxStages * RowSmem<64>::kBlockBytes));
-                sized64 = true;
-            }
-            PA_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_row_kernel<64>, a));
+            if (ring) PA_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_row_kernel<64, true>, a));
+            else PA_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_row_kernel<64, false>, a));
         }
         return PA_OK;
     }
