@@ -161,7 +161,9 @@ size_t pa_decode_workspace_bytes(const pa_decode_params *p);
  * block) into the workspace, then the same merge.  The workspace must be given in both cases.
  * Calls that share a workspace must not overlap on the GPU.  Environment switches read on every
  * call (for tests and measurements): PA_DECODE_PATH=splitk forces the two-kernel path,
- * PA_DECODE_CLUSTER=n (1..8) sets the cluster size. */
+ * PA_DECODE_CLUSTER=n (1..8) sets the cluster size (default: 8 for small calls, fewer CTAs per
+ * row as batch x n_kv_heads grows, down to one), PA_DECODE_STAGES=n (1..4) the number of key
+ * blocks a CTA keeps in flight when it has more blocks than that. */
 pa_status pa_decode(const pa_decode_params *p, const void *q, const void *k_cache,
                     const void *v_cache, const int32_t *cache_lens, void *o, float *lse,
                     void *workspace, size_t workspace_bytes, void *stream);

@@ -268,10 +268,13 @@ __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeArgs a)
 // One launch per call: a thread-block cluster per (sequence, KV head).
 //
 // The row's key blocks are dealt round-robin to the CTAs of the cluster.  A CTA requests its K and
-// V blocks with 16-byte asynchronous copies into a ring of shared-memory stages (with few blocks
-// per CTA everything it will ever read is in flight at once), then takes them in order as they
-// land: logits and P V as in decode_block_kernel, with the running maximum, sum and output kept
-// in registers across blocks (online softmax).  The CTAs' partial results meet in shared memory:
+// V blocks with 16-byte asynchronous copies into shared memory and takes them in order as they
+// land.  Two forms (kRing): a small call uses the widest cluster, so a CTA has at most four
+// blocks, each with its own stage, all requested at once (lowest latency); a large call uses
+// few CTAs per row, each walking its blocks through a ring of stages (one by default: six CTAs
+// then share an SM, which is what fills the memory pipe).  Per block: logits and P V as in
+// decode_block_kernel, with the running maximum, sum and output kept in registers across blocks
+// (online softmax).  The CTAs' partial results meet in shared memory:
 // after a cluster barrier CTA r merges the heads g = r, r + R, ... reading its peers' partials
 // through distributed shared memory, and writes O and the LSE.  No workspace, no second launch.
 // ------------------------------------------------------------------------------------------
@@ -425,14 +428,17 @@ __global__ void __launch_bounds__(kDecThreads) decode_row_kernel(const DecodeArg
         const int32_t jblk = block_of(i);
         const int n_keys = jblk == row ? (int)(p % kDecBlock) + 1 : kDecBlock;
         const uint32_t sk = smem0 + (i % stages) * SM::kBlockBytes, sv_ = sk + SM::kTile;
-        cp_async_wait(issued - 1 - i);
-        __syncthreads();  // every thread's copies of this block have landed; sS and the stage of block i - 1 are free
         if constexpr (kRing) {
-            if (i >= 1 && issued < mine) {
-                issue_block(issued);  // into the stage block i - 1 has just left
-                ++issued;
+            if (i >= 1) {
+                __syncthreads();  // every warp has finished block i - 1: its stage is free
+                if (issued < mine) {
+                    issue_block(issued);  // block i - 1 + stages (block i itself when there is one stage)
+                    ++issued;
+                }
             }
         }
+        cp_async_wait(issued - 1 - i);
+        __syncthreads();  // every thread's copies of this block have landed; sS is free again
 
         // ---- S = Q K^T: rows = heads, columns = the warp's 16 keys (two 8-key tiles)
         float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};

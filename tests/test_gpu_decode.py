@@ -88,10 +88,13 @@ def test_decode_full_size_workload(pa, oracle):
 
 
 @pytest.mark.parametrize("env", [{"PA_DECODE_PATH": "splitk"}, {"PA_DECODE_CLUSTER": "1"}, {"PA_DECODE_CLUSTER": "2"},
-                                 {"PA_DECODE_CLUSTER": "7"}, {"PA_DECODE_CLUSTER": "8"}])
+                                 {"PA_DECODE_CLUSTER": "7"}, {"PA_DECODE_CLUSTER": "8"},
+                                 {"PA_DECODE_CLUSTER": "2", "PA_DECODE_STAGES": "2"},
+                                 {"PA_DECODE_CLUSTER": "1", "PA_DECODE_STAGES": "3"},
+                                 {"PA_DECODE_CLUSTER": "8", "PA_DECODE_STAGES": "1"}])
 def test_decode_paths(pa, oracle, monkeypatch, env):
-    """The two-launch split-K path and the single-launch cluster path at several cluster sizes
-    (the library reads these switches on every call) give the same row of Eq. (1)."""
+    """The two-launch split-K path and the single-launch cluster path at several cluster sizes and
+    ring depths (the library reads these switches on every call) give the same row of Eq. (1)."""
     for k, v in env.items():
         monkeypatch.setenv(k, v)
     batch, max_len, Hq, Hkv, D = 4, 9000, 28, 4, 128
