@@ -162,3 +162,22 @@ def test_csr_check_switch_rejects_malformed_layouts(pa, monkeypatch):
     expect_layout_error(bad, ci)
     bad = rp.clone(); bad[0] = 1                    # does not start at 0
     expect_layout_error(bad, ci)
+
+
+@pytest.mark.parametrize("o_dtype", [torch.bfloat16, torch.float32])
+def test_strided_output_is_written_only_inside_its_view(pa, oracle, o_dtype):
+    """O as a view into a larger buffer (extra heads, extra tokens, extra batch stride), with a
+    ragged last query block and a 7-head group (one padded head in the kernel's tiles): the view
+    holds the result, every element of the buffer outside it keeps its sentinel."""
+    N, Hq, Hkv, D = 1000, 7, 1, 128
+    Q, K, V = si.bf16_randn((2, N, Hq, D), 61), si.bf16_randn((2, N, Hkv, D), 62), si.bf16_randn((2, N, Hkv, D), 63)
+    big = torch.full((2, N + 100, Hq + 3, D), 7.0, dtype=o_dtype, device="cuda")
+    o_view = big[:, :N, 1:1 + Hq]
+    rp, ci = pa.pa_build_layout(N, 64, 5, 1)
+    o, lse, ws = pa.pa_prefill(Q.cuda(), K.cuda(), V.cuda(), rp, ci, o=o_view, o_dtype=o_dtype)
+    pa.pa_prefill_status(ws)
+    o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, 5, 1)
+    compare(o_view, lse, o_ref, lse_ref, "strided output")
+    outside = torch.ones_like(big, dtype=torch.bool)
+    outside[:, :N, 1:1 + Hq] = False
+    assert bool((big[outside] == 7.0).all()), "elements outside the output view were overwritten"
