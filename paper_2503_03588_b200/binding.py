@@ -53,7 +53,7 @@ class pa_decode_params(ctypes.Structure):
 
 def _load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
-        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2503_03588_b200.build` "
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python paper_2503_03588_b200/build.py` "
                           "(there is no fallback path)")
     lib = ctypes.CDLL(LIB_PATH)
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
