@@ -142,6 +142,39 @@ def block_layout(N: int, B: int, W: int, S: int = 1,
     return row_ptr, col_idx.astype(np.int32)
 
 
+def tile_layout_from_tokens(N: int, B: int, W: int, S: int, T: int,
+                            use_power: bool = True) -> Tuple[np.ndarray, np.ndarray]:
+    """Brute force at a tile size T that differs from the mask's block size B (the paper's
+    efficiency runs use B = 256, Section 4.1): key tile tj is listed for query tile ti iff some
+    token pair (q, kv) in those T-token tiles satisfies the token-level predicate of
+    Algorithm 1 evaluated with block size B.  O(N^2); for small N only."""
+    m = dense_mask(N, B, W, S, use_power)
+    nt = -(-N // T)
+    pad = np.zeros((nt * T, nt * T), dtype=bool)
+    pad[:N, :N] = m
+    return _csr_from_block_matrix(pad.reshape(nt, T, nt, T).any(axis=(1, 3)))
+
+
+def tile_layout(N: int, B: int, W: int, S: int, T: int,
+                use_power: bool = True) -> Tuple[np.ndarray, np.ndarray]:
+    """The same list without the token matrix, usable at large N, for T dividing B: the window,
+    power and sink terms of Algorithm 1 see only the B-token blocks that hold the two tiles, and
+    its causal term (kv_idx <= q_idx) leaves tile tj <= ti non-empty and tile tj > ti empty."""
+    assert B % T == 0
+    r = B // T
+    nt = -(-N // T)
+    row_ptr = np.zeros(nt + 1, dtype=np.int32)
+    cols = []
+    for ti in range(nt):
+        i = ti // r
+        js = [tj for j in _candidate_blocks(i, W, S, use_power) if block_predicate(i, j, W, S, use_power)
+              for tj in range(j * r, min((j + 1) * r, ti + 1))]
+        cols.append(np.asarray(js, dtype=np.int32))
+        row_ptr[ti + 1] = row_ptr[ti] + len(js)
+    col_idx = np.concatenate(cols) if cols else np.zeros(0, dtype=np.int32)
+    return row_ptr, col_idx.astype(np.int32)
+
+
 def _candidate_blocks(i: int, W: int, S: int, use_power: bool):
     """All j <= i when that is cheap; else only the j that can possibly pass (a superset of
     sink, window and power-of-two distances), still filtered by block_predicate."""

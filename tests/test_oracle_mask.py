@@ -209,3 +209,37 @@ def test_active_block_counts_scale_as_n_log_n(oracle):
     rp, _ = oracle.block_layout(131072, 256, 5, 1)
     nqb = 512
     assert 20 < (nqb * (nqb + 1) // 2) / int(rp[-1]) < 27   # paper reports 21.6x in time
+
+
+# ------------------------------------------------------------------ tile layouts (tile != block)
+
+@pytest.mark.parametrize("B,T", [(8, 2), (16, 4), (256, 64)])
+def test_tile_layout_matches_token_brute_force(oracle, B, T):
+    """Tile-level enumeration == brute force over every token pair when the mask's block is a
+    multiple of the tile (the paper's 256-token blocks on 64-token tiles, Section 4.1)."""
+    for N in (1, T + 1, B - 1, B, B + T + 1, 3 * B + 1, 7 * B - T - 1, min(1280, 12 * B)):
+        for W in (0, 1, 3, 5):
+            for S in (0, 1, 2):
+                a = oracle.tile_layout_from_tokens(N, B, W, S, T)
+                b = oracle.tile_layout(N, B, W, S, T)
+                assert (a[0] == b[0]).all() and (a[1] == b[1]).all(), (N, B, T, W, S)
+
+
+def test_tile_layout_special_cases(oracle):
+    """T == B is the block layout; row length in closed form; the tiles' token count equals the
+    token mask's row sums (64 * tiles - (63 - q mod 64) per row, the diagonal tile being partial)."""
+    for (N, B, W, S) in [(1000, 8, 5, 1), (515, 4, 0, 0)]:
+        a, b = oracle.tile_layout(N, B, W, S, B), oracle.block_layout(N, B, W, S)
+        assert (a[0] == b[0]).all() and (a[1] == b[1]).all()
+    N, B, T, W, S = 1536, 256, 64, 2, 1
+    r = B // T
+    rp, ci = oracle.tile_layout(N, B, W, S, T)
+    brp, _ = oracle.block_layout(N, B, W, S)
+    m = oracle.dense_mask(N, B, W, S)
+    for ti in range(N // T):
+        i = ti // r
+        assert rp[ti + 1] - rp[ti] == r * (brp[i + 1] - brp[i] - 1) + (ti - i * r + 1)
+        row = ci[rp[ti]:rp[ti + 1]]
+        assert (np.diff(row) > 0).all() and row[-1] == ti
+        for q in (ti * T, ti * T + 17, ti * T + T - 1):
+            assert m[q].sum() == T * len(row) - (T - 1 - q % T)
