@@ -556,6 +556,8 @@ def run_sweep(args):
         layouts = {"powerattention": (rp_pa, ci_pa)}
         rw, cw = row_matched_window_csr(rp_host)
         layouts["sliding_window_row_matched"] = (torch.as_tensor(rw).to(dev), torch.as_tensor(cw).to(dev))
+        # The paper's own block size (256 tokens, Section 4.1), listed by the kernel's 64-token tiles.
+        layouts["powerattention_block256"] = pa.pa_build_tile_layout(N, 256, w.window_blocks, w.sink_blocks, w.block)
         if N <= args.sweep_dense_max_len:
             rc, cc = causal_csr(nqb)
             layouts["dense_causal"] = (torch.as_tensor(rc).to(dev), torch.as_tensor(cc).to(dev))

@@ -72,6 +72,31 @@ pa_status pa_build_layout(int64_t seq_len, int32_t block, int32_t window_blocks,
                           int32_t sink_blocks, int32_t *row_ptr, int32_t *col_idx,
                           int64_t col_capacity, void *stream);
 
+/* Tile layouts: the same mask listed at the granularity of the attention kernel.
+ *
+ * The paper's efficiency runs use 256-token blocks (Section 4.1, "Implementation"), the kernels
+ * here walk 64-token tiles.  For `block` a multiple of `tile`, query tile ti (tokens
+ * [ti tile, ti tile + tile)) lists key tile tj exactly when some token pair of the two tiles
+ * passes Algorithm 1 evaluated with `block`: with i = ti tile / block and j = tj tile / block,
+ * that is tj <= ti and block j is listed for block i.  Every listed block before the diagonal
+ * one contributes all its tiles, the diagonal block its tiles up to ti.  The CSR has
+ * n_qtiles = ceil(seq_len / tile) ascending rows and can be given to pa_prefill with
+ * block = tile: the only pair that the kernel masks by token is tj == ti, which is the only
+ * partial one here as well.  With tile == block this is pa_layout_size / pa_build_layout. */
+
+/* Host-only closed-form sizes.  n_qtiles, nnz: host pointers, written on success.
+ * Errors: as pa_layout_size, and PA_ERR_INVALID_ARG (tile < 1), PA_ERR_SHAPE (block is not a
+ * multiple of tile). */
+pa_status pa_tile_layout_size(int64_t seq_len, int32_t block, int32_t window_blocks,
+                              int32_t sink_blocks, int32_t tile, int32_t *n_qtiles, int64_t *nnz);
+
+/* Writes the tile CSR on the device.  row_ptr: device int32[n_qtiles + 1]; col_idx: device
+ * int32[col_capacity], col_capacity >= nnz from pa_tile_layout_size (else PA_ERR_LAYOUT, nothing
+ * launched).  Three small kernels are enqueued on `stream`; no scratch memory is used. */
+pa_status pa_build_tile_layout(int64_t seq_len, int32_t block, int32_t window_blocks,
+                               int32_t sink_blocks, int32_t tile, int32_t *row_ptr,
+                               int32_t *col_idx, int64_t col_capacity, void *stream);
+
 /* ------------------------------------------------------------------------------------------
  * Prefill: Eq. (1) (Section 3.1) over the listed key blocks of each query block.
  *

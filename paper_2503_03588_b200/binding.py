@@ -21,7 +21,7 @@ STATUS_NAMES = ["PA_OK", "PA_ERR_INVALID_ARG", "PA_ERR_SHAPE", "PA_ERR_ALIGNMENT
                 "PA_ERR_WORKSPACE", "PA_ERR_UNSUPPORTED", "PA_ERR_CUDA", "PA_ERR_TIMEOUT"]
 
 EXPORTS = ["pa_status_string", "pa_last_error_message", "pa_version", "pa_layout_size",
-           "pa_build_layout", "pa_prefill_workspace_bytes", "pa_prefill", "pa_prefill_status",
+           "pa_build_layout", "pa_tile_layout_size", "pa_build_tile_layout", "pa_prefill_workspace_bytes", "pa_prefill", "pa_prefill_status",
            "pa_decode_workspace_bytes", "pa_decode", "pa_decode_block_list", "pa_decode_static"]
 
 
@@ -66,6 +66,10 @@ def _load() -> ctypes.CDLL:
     lib.pa_layout_size.argtypes = [i64, i32, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i64)]
     lib.pa_build_layout.restype = ctypes.c_int
     lib.pa_build_layout.argtypes = [i64, i32, i32, i32, vp, vp, i64, vp]
+    lib.pa_tile_layout_size.restype = ctypes.c_int
+    lib.pa_tile_layout_size.argtypes = [i64, i32, i32, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i64)]
+    lib.pa_build_tile_layout.restype = ctypes.c_int
+    lib.pa_build_tile_layout.argtypes = [i64, i32, i32, i32, i32, vp, vp, i64, vp]
     lib.pa_prefill_workspace_bytes.restype = ctypes.c_size_t
     lib.pa_prefill_workspace_bytes.argtypes = [ctypes.POINTER(pa_prefill_params)]
     lib.pa_prefill.restype = ctypes.c_int
@@ -132,6 +136,30 @@ def pa_build_layout(seq_len: int, block: int, window_blocks: int, sink_blocks: i
     assert row_ptr.dtype == torch.int32 and col_idx.dtype == torch.int32 and row_ptr.numel() >= nqb + 1
     _check(lib.pa_build_layout(seq_len, block, window_blocks, sink_blocks, _ptr(row_ptr), _ptr(col_idx),
                                col_idx.numel(), _stream()))
+    return row_ptr, col_idx
+
+
+def pa_tile_layout_size(seq_len: int, block: int, window_blocks: int, sink_blocks: int,
+                        tile: int = 64) -> Tuple[int, int]:
+    nqt, nnz = ctypes.c_int32(0), ctypes.c_int64(0)
+    _check(lib.pa_tile_layout_size(seq_len, block, window_blocks, sink_blocks, tile, ctypes.byref(nqt),
+                                   ctypes.byref(nnz)))
+    return int(nqt.value), int(nnz.value)
+
+
+def pa_build_tile_layout(seq_len: int, block: int, window_blocks: int, sink_blocks: int, tile: int = 64,
+                         row_ptr: Optional[torch.Tensor] = None, col_idx: Optional[torch.Tensor] = None,
+                         device="cuda"):
+    """Returns (row_ptr, col_idx) int32 device tensors of the mask with `block`-token blocks listed by
+    `tile`-token tiles (allocated here when not passed in)."""
+    nqt, nnz = pa_tile_layout_size(seq_len, block, window_blocks, sink_blocks, tile)
+    if row_ptr is None:
+        row_ptr = torch.empty(nqt + 1, dtype=torch.int32, device=device)
+    if col_idx is None:
+        col_idx = torch.empty(nnz, dtype=torch.int32, device=device)
+    assert row_ptr.dtype == torch.int32 and col_idx.dtype == torch.int32 and row_ptr.numel() >= nqt + 1
+    _check(lib.pa_build_tile_layout(seq_len, block, window_blocks, sink_blocks, tile, _ptr(row_ptr),
+                                    _ptr(col_idx), col_idx.numel(), _stream()))
     return row_ptr, col_idx
 
 

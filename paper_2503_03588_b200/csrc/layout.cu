@@ -59,6 +59,44 @@ __global__ void layout_fill_kernel(int32_t nqb, int32_t W, int32_t S, const int3
     for_each_key_block(i, W, S, StoreCols{col_idx + row_ptr[i]});
 }
 
+// Tile layouts: the mask's block holds r tiles of the attention kernel.  Algorithm 1's window,
+// power and sink terms see the blocks only, so every listed block j < i contributes its r tiles;
+// its causal term cuts the diagonal block i down to the tiles i r .. ti.
+__host__ __device__ inline int64_t tile_row_length(int64_t ti, int32_t r, int32_t W, int32_t S)
+{
+    const int64_t i = ti / r;
+    return (int64_t)r * (row_length(i, W, S) - 1) + (ti - i * r + 1);
+}
+
+__global__ void tile_layout_count_kernel(int32_t nqt, int32_t r, int32_t W, int32_t S, int32_t *row_ptr)
+{
+    const int64_t ti = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (ti == 0) row_ptr[0] = 0;
+    if (ti < nqt) row_ptr[ti + 1] = (int32_t)tile_row_length(ti, r, W, S);
+}
+
+struct StoreTileCols {
+    int32_t *out;
+    int64_t i, ti;
+    int32_t r;
+    __device__ void operator()(int pos, int64_t j) const
+    {
+        // (The diagonal block is the last one listed, so every block before it is whole.)
+        const int64_t last = j == i ? ti : j * r + r - 1;
+        int32_t *dst = out + (int64_t)pos * r;
+        for (int64_t tj = j * r; tj <= last; ++tj) *dst++ = (int32_t)tj;
+    }
+};
+
+__global__ void tile_layout_fill_kernel(int32_t nqt, int32_t r, int32_t W, int32_t S, const int32_t *row_ptr,
+                                        int32_t *col_idx)
+{
+    const int64_t ti = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (ti >= nqt) return;
+    const int64_t i = ti / r;
+    for_each_key_block(i, W, S, StoreTileCols{col_idx + row_ptr[ti], i, ti, r});
+}
+
 static pa_status check_layout_args(int64_t seq_len, int32_t block, int32_t W, int32_t S)
 {
     if (seq_len < 1) return fail(PA_ERR_INVALID_ARG, "seq_len must be >= 1 (got %lld)", (long long)seq_len);
@@ -104,6 +142,53 @@ extern "C" pa_status pa_build_layout(int64_t seq_len, int32_t block, int32_t win
     layout_count_kernel<<<blocks, threads, 0, st>>>(nqb, window_blocks, sink_blocks, row_ptr);
     layout_scan_kernel<<<1, 1024, 0, st>>>(nqb, row_ptr);
     layout_fill_kernel<<<blocks, threads, 0, st>>>(nqb, window_blocks, sink_blocks, row_ptr, col_idx);
+    PA_CUDA_OK(cudaGetLastError());
+    return PA_OK;
+}
+
+extern "C" pa_status pa_tile_layout_size(int64_t seq_len, int32_t block, int32_t window_blocks,
+                                         int32_t sink_blocks, int32_t tile, int32_t *n_qtiles, int64_t *nnz)
+{
+    using namespace pa;
+    clear_error();
+    if (pa_status s = check_layout_args(seq_len, block, window_blocks, sink_blocks)) return s;
+    if (tile < 1) return fail(PA_ERR_INVALID_ARG, "tile must be >= 1 (got %d)", tile);
+    if (block % tile != 0) return fail(PA_ERR_SHAPE, "block %d is not a multiple of tile %d", block, tile);
+    if (!n_qtiles || !nnz) return fail(PA_ERR_INVALID_ARG, "n_qtiles and nnz must be non-null");
+    const int32_t r = block / tile;
+    const int64_t nqt = (seq_len + tile - 1) / tile;
+    if (nqt >= INT32_MAX) return fail(PA_ERR_SHAPE, "n_qtiles %lld does not fit in int32", (long long)nqt);
+    // Tiles of one block share the block's row length; their diagonal parts are 1, 2, ..., r.
+    int64_t total = 0;
+    for (int64_t i = 0; i * r < nqt; ++i) {
+        const int64_t tiles = nqt - i * r < r ? nqt - i * r : r;  // the last block may be cut short
+        total += tiles * r * (int64_t)(row_length(i, window_blocks, sink_blocks) - 1) + tiles * (tiles + 1) / 2;
+    }
+    if (total > INT32_MAX) return fail(PA_ERR_SHAPE, "nnz %lld does not fit in int32", (long long)total);
+    *n_qtiles = (int32_t)nqt;
+    *nnz = total;
+    return PA_OK;
+}
+
+extern "C" pa_status pa_build_tile_layout(int64_t seq_len, int32_t block, int32_t window_blocks,
+                                          int32_t sink_blocks, int32_t tile, int32_t *row_ptr,
+                                          int32_t *col_idx, int64_t col_capacity, void *stream)
+{
+    using namespace pa;
+    clear_error();
+    int32_t nqt = 0;
+    int64_t nnz = 0;
+    if (pa_status s = pa_tile_layout_size(seq_len, block, window_blocks, sink_blocks, tile, &nqt, &nnz)) return s;
+    if (!row_ptr || !col_idx) return fail(PA_ERR_INVALID_ARG, "row_ptr and col_idx must be non-null");
+    if (col_capacity < nnz)
+        return fail(PA_ERR_LAYOUT, "col_capacity %lld < nnz %lld", (long long)col_capacity, (long long)nnz);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int threads = 256;
+    const unsigned blocks = (unsigned)((nqt + threads - 1) / threads);
+    const int32_t r = block / tile;
+    tile_layout_count_kernel<<<blocks, threads, 0, st>>>(nqt, r, window_blocks, sink_blocks, row_ptr);
+    layout_scan_kernel<<<1, 1024, 0, st>>>(nqt, row_ptr);
+    tile_layout_fill_kernel<<<blocks, threads, 0, st>>>(nqt, r, window_blocks, sink_blocks, row_ptr, col_idx);
     PA_CUDA_OK(cudaGetLastError());
     return PA_OK;
 }

@@ -50,6 +50,20 @@ def test_layout_size_matches_oracle(pa, oracle):
         assert (nqb, nnz) == (len(rp) - 1, int(rp[-1]))
 
 
+def test_tile_layout_size_matches_oracle(pa, oracle):
+    """Masks with blocks that are a multiple of the 64-token tile (the paper's 256-token blocks)."""
+    for (B, T) in [(256, 64), (128, 64), (64, 64), (8, 2), (256, 256)]:
+        for N in (1, T, T + 1, B - 1, B, 5 * B + T + 3, 40 * B):
+            for (W, S) in [(5, 1), (0, 0), (1, 2), (9, 3)]:
+                nqt, nnz = pa.pa_tile_layout_size(N, B, W, S, T)
+                rp, ci = oracle.tile_layout(N, B, W, S, T)
+                assert nqt == len(rp) - 1 and nnz == int(rp[-1]) == len(ci), (N, B, T, W, S)
+    assert pa.pa_tile_layout_size(32768, 64, 5, 1, 64) == pa.pa_layout_size(32768, 64, 5, 1)
+    for bad in [(1000, 256, 5, 1, 96), (1000, 64, 5, 1, 128), (1000, 256, 5, 1, 0)]:
+        with pytest.raises(pa.PaError):
+            pa.pa_tile_layout_size(*bad)
+
+
 def test_active_block_counts_of_the_workloads(pa):
     expect = {2048: 215, 4096: 502, 8192: 1141, 16384: 2548, 32768: 5619, 65536: 12274,
               131072: 26609, 262144: 57328}

@@ -45,6 +45,27 @@ def test_layout_workload_configs(pa, oracle, N, W, S):
     _check(pa, oracle, N, 64, W, S)
 
 
+def test_tile_layout_bit_exact(pa, oracle):
+    """The mask with `block`-token blocks listed by `tile`-token tiles: against the tile-level
+    enumeration, against token-level brute force on small sizes, and at the paper's block size
+    (256) for the 32K and 128K workloads."""
+    def check(N, B, W, S, T, ref):
+        rp, ci = pa.pa_build_tile_layout(N, B, W, S, T)
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(rp.cpu().numpy(), ref[0])
+        np.testing.assert_array_equal(ci.cpu().numpy(), ref[1])
+
+    for N in (1, 64, 65, 255, 256, 257, 1000, 5000, 70000):
+        for (W, S) in [(5, 1), (0, 0), (1, 2), (9, 3)]:
+            check(N, 256, W, S, 64, oracle.tile_layout(N, 256, W, S, 64))
+    for (N, B, W, S, T) in [(900, 256, 2, 1, 64), (700, 16, 3, 1, 4), (513, 8, 0, 2, 2), (640, 128, 1, 0, 64)]:
+        check(N, B, W, S, T, oracle.tile_layout_from_tokens(N, B, W, S, T))
+    check(5000, 64, 5, 1, 64, oracle.block_layout(5000, 64, 5, 1))      # tile == block
+    for N in (32768, 131072):
+        check(N, 256, 5, 1, 64, oracle.tile_layout(N, 256, 5, 1, 64))
+    check(256 * 1500 + 77, 256, 5, 1, 64, oracle.tile_layout(256 * 1500 + 77, 256, 5, 1, 64))  # > 1 scan tile
+
+
 def test_layout_larger_than_one_scan_tile(pa, oracle):
     _check(pa, oracle, 64 * 5000 + 5, 64, 5, 1)   # 5001 rows: several 1024-row scan tiles + tail
 

@@ -87,6 +87,37 @@ def test_other_causal_layouts_through_the_same_kernel(pa, oracle):
         compare(o, lse, o_ref, lse_ref, f"use_power={use_power} W={W}")
 
 
+@pytest.mark.parametrize("N,Hq,Hkv,D,B,W,S", [
+    (1500, 7, 1, 128, 256, 5, 1),     # window covers the whole sequence at this size: dense causal
+    (3000, 14, 2, 128, 256, 2, 1),    # ragged tail, power-of-two distances 1, 2, 4, 8 in blocks
+    (2100, 4, 2, 64, 128, 1, 0),      # 128-token blocks, no sink
+    (2048, 8, 2, 128, 256, 0, 0),     # pure power-of-two pattern
+])
+def test_mask_blocks_larger_than_the_tile(pa, oracle, N, Hq, Hkv, D, B, W, S):
+    """The paper's block size (256 tokens, Section 4.1) and other multiples of the kernel's
+    64-token tile: the tile CSR of pa_build_tile_layout through pa_prefill against the oracle,
+    which applies the token-level predicate with that block size."""
+    Q = si.bf16_randn((1, N, Hq, D), 400 + N)
+    K = si.bf16_randn((1, N, Hkv, D), 500 + N)
+    V = si.bf16_randn((1, N, Hkv, D), 600 + N)
+    layout = pa.pa_build_tile_layout(N, B, W, S, 64)
+    o, lse = _gpu_prefill(pa, Q, K, V, W, S, layout=layout)
+    o_ref, lse_ref, _ = oracle.prefill(Q, K, V, B, W, S)
+    compare(o, lse, o_ref, lse_ref, f"B={B} N={N} W={W} S={S}")
+
+
+def test_paper_block_size_at_32k_on_sampled_rows(pa, oracle):
+    """32K tokens in 256-token blocks (the paper's efficiency setting) with the 7B-like heads."""
+    w = si.PREFILL_32K
+    Q, K, V = si.prefill_inputs(w)
+    layout = pa.pa_build_tile_layout(w.seq_len, 256, w.window_blocks, w.sink_blocks, 64)
+    o, lse = _gpu_prefill(pa, Q, K, V, w.window_blocks, w.sink_blocks, layout=layout)
+    rows = _sampled_rows(w.seq_len, np.random.default_rng(w.seed + 7), n_random=48)
+    o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 256, w.window_blocks, w.sink_blocks, rows=rows)
+    ridx = torch.as_tensor(rows).cuda()
+    compare(o[:, ridx], lse[:, :, ridx], o_ref, lse_ref, "32K, 256-token blocks")
+
+
 def test_constant_keys_count_the_attended_tokens(pa, oracle):
     """K rows all equal => LSE_q - s_q = ln |A_q|, |A_q| = 64 * #blocks(row) - (63 - q mod 64);
     holds at any size, so it is checked at 32K with the 7B-like heads."""
