@@ -44,7 +44,7 @@ namespace pa {
 constexpr int kBlk = 64;               // tokens per query / key block
 constexpr int kThreads = 512;          // 16 warps: control, two softmax warpgroups, epilogue
 constexpr int kKStages = 3;             // K block ring depth (a K block is needed at the start of a step)
-constexpr int kVStages = 2;             // V block ring depth (a V block is needed at its end)
+constexpr int kVStages = 3;             // V block ring depth (a V block is needed at its end; loads take longer than two steps)
 constexpr uint32_t kTmemCols = 512;    // slot s: S at columns 128 s, P buffers at 128 s + 64 + 32 b, O at 256 + s D
 // A step's row sum above this limit sends the step through the exact path (new reference).
 constexpr float kSumLimit = 1048576.0f;  // 2^20
@@ -72,9 +72,11 @@ struct SmemMap {
     static constexpr uint32_t kQBuf = 2 * kQSlot;             // both slots' Q tiles of one unit
     static constexpr uint32_t kK = kQ + 2 * kQBuf;            // two units' worth: the next unit's Q loads early
     static constexpr uint32_t kV = kK + kKStages * kBlkTile;
-    static constexpr uint32_t kOStage = kV + kVStages * kBlkTile;  // one head's O rows on their way out
-    static constexpr uint32_t kOStageBytes = 64 * D * 2;      // one head x 64 tokens
-    static constexpr uint32_t kStats = kOStage + kOStageBytes;    // [slot][row] softmax denominators
+    // A finished unit's output is staged in that unit's own Q buffer (its four heads x 64 tokens
+    // take exactly the room of the two 128-row Q tiles), so it needs no area of its own.
+    static constexpr uint32_t kOHead = 64 * D * 2;            // one head x 64 tokens of staged O
+    static_assert(4 * kOHead == kQBuf, "the staged output of a unit fills its Q buffer");
+    static constexpr uint32_t kStats = kV + kVStages * kBlkTile;  // [slot][row] softmax denominators
     static constexpr uint32_t kBars = kStats + 2 * 128 * 4;
     static constexpr uint32_t kTotal = kBars + 512;
     static constexpr uint32_t kAlloc = kTotal + 1024;         // slack for 1024-byte alignment
@@ -93,9 +95,10 @@ enum : uint32_t {
     BAR_O_FINAL = BAR_O_DONE + 4,   // [slot]: the unit's last P V has completed
     BAR_ML_READY = BAR_O_FINAL + 2,  // [slot]: the unit's row statistics are in shared memory
     BAR_O_FREE = BAR_ML_READY + 2,   // [slot]: the epilogue has read O out of tensor memory
-    BAR_STAGE_FREE = BAR_O_FREE + 2,  // the output staging tile has been read by its bulk stores
-    BAR_STAGE_FULL = BAR_STAGE_FREE + 1,  // ... has been written by the four epilogue warps
-    BAR_COUNT = BAR_STAGE_FULL + 1
+    BAR_STAGE_FREE = BAR_O_FREE + 2,  // [unit parity]: the bulk stores have read the unit's staged output
+    BAR_STAGE_FULL = BAR_STAGE_FREE + 2,  // a slot's two heads have been staged by the four epilogue warps
+    BAR_TURN = BAR_STAGE_FULL + 1,  // [slot]: the other slot has finished a pass of exponentials
+    BAR_COUNT = BAR_TURN + 2
 };
 
 struct Unit {
@@ -159,15 +162,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(bar(BAR_Q_FULL + s), 1);
-            ptx::mbar_init(bar(BAR_Q_EMPTY + s), 1);
+            ptx::mbar_init(bar(BAR_Q_EMPTY + s), 2);  // (the "empty" barriers: one commit per issuing warp)
         }
         for (int s = 0; s < kKStages; ++s) {
             ptx::mbar_init(bar(BAR_K_FULL + s), 1);
-            ptx::mbar_init(bar(BAR_K_EMPTY + s), 1);
+            ptx::mbar_init(bar(BAR_K_EMPTY + s), 2);
         }
         for (int s = 0; s < kVStages; ++s) {
             ptx::mbar_init(bar(BAR_V_FULL + s), 1);
-            ptx::mbar_init(bar(BAR_V_EMPTY + s), 1);
+            ptx::mbar_init(bar(BAR_V_EMPTY + s), 2);
         }
         for (int s = 0; s < 4; ++s) ptx::mbar_init(bar(BAR_O_DONE + s), 1);
         for (int s = 0; s < 2; ++s) {
@@ -180,7 +183,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::mbar_init(bar(BAR_O_FREE + s), 4);
         }
         ptx::mbar_init(bar(BAR_STAGE_FREE), 1);
+        ptx::mbar_init(bar(BAR_STAGE_FREE + 1), 1);
         ptx::mbar_init(bar(BAR_STAGE_FULL), 4);
+        ptx::mbar_init(bar(BAR_TURN), 4);
+        ptx::mbar_init(bar(BAR_TURN + 1), 4);
         *abort_flag = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
@@ -217,10 +223,16 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 return u;
             };
             // Q tiles of unit number ul_q go to Q buffer ul_q & 1 once the unit two before has
-            // issued its last S.
+            // issued its last S and its output, staged in that buffer, has left.  (Both barriers
+            // complete once per two units; this thread's own wait two units ago keeps them
+            // within one phase of the parity asked for.)
+            auto q_buffer_free = [&](uint32_t ul_q) {
+                return ul_q < 2 || ptx::mbar_test_wait(bar(BAR_STAGE_FREE + (ul_q & 1)), ((ul_q >> 1) - 1) & 1);
+            };
             auto load_q = [&](const Unit &w, uint32_t ul_q) {
                 const uint32_t qb = ul_q & 1;
                 if (ul_q >= 2 && !wait_bar(bar(BAR_Q_EMPTY + qb), ((ul_q >> 1) - 1) & 1, abort_flag, a.status, 1)) return false;
+                if (ul_q >= 2 && !wait_bar(bar(BAR_STAGE_FREE + qb), ((ul_q >> 1) - 1) & 1, abort_flag, a.status, 16)) return false;
                 ptx::mbar_expect_tx(bar(BAR_Q_FULL + qb), SM::kQBuf);
                 for (int s = 0; s < 2; ++s)
                     for (int dh = 0; dh < DH; ++dh)
@@ -235,6 +247,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             if (u < (uint32_t)a.n_units) ok = load_q(w, 0);
             while (u < (uint32_t)a.n_units && ok) {
                 const uint32_t un = next_unit(u + gridDim.x, wn, jnext);
+                bool q_pending = un < (uint32_t)a.n_units;  // the next unit's Q tiles are still to be requested
                 for (int t = 0; t < w.n; ++t, ++kc) {
                     const int32_t jn = t + 1 < w.n ? __ldg(a.col_idx + w.rs + t + 1) : 0;
                     const uint32_t ks = kc % kKStages, vs = kc % kVStages;
@@ -255,11 +268,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         ptx::tma_load_4d(smem_base + SM::kV + vs * SM::kBlkTile + dh * SM::kBlkSub, &tmV,
                                          bar(BAR_V_FULL + vs), dh * 64, j * kBlk, w.hk, w.b);
                     j = jn;
-                    // The next unit's Q behind this unit's second block: by then the unit before
-                    // this one has issued its last S (its K stage was just reused), so the Q
-                    // buffer is free and the load has the whole unit to arrive.
-                    if (t == (w.n > 1 ? 1 : 0) && un < (uint32_t)a.n_units) {
+                    // The next unit's Q goes where the unit before this one kept its Q and then
+                    // staged its output, which leaves during this unit's first steps: the request
+                    // is made behind the first block (from the second on) that finds the buffer
+                    // free, so the key blocks are not held up, and behind the last one at the latest.
+                    if (q_pending && (t + 1 == w.n || (t >= 1 && q_buffer_free(ul + 1)))) {
                         ok = load_q(wn, ul + 1);
+                        q_pending = false;
                         if (!ok) break;
                     }
                 }
@@ -276,11 +291,16 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ tcgen05 issuer
+    } else if (warp == 1 || warp == 3) {
+        // ------------------------------------------------------------------ tcgen05 issuers
+        // One issuing warp per slot (warp 1: slot 0, warp 3: slot 1): a step's waits and MMA
+        // issue cost the issuing warp about a thousand cycles per slot, and one warp serving both
+        // slots in turn was the longest chain of the step.  The two warps share nothing but the
+        // operand tiles: a commit covers the MMAs of the committing thread only, so the barriers
+        // that free a K, V or Q tile count one arrival from each.
         // The whole warp runs the (uniform) control flow and the barrier waits; one elected lane
         // issues the MMAs and commits.  Steps are numbered through the CTA's whole run (c), so ring
-        // positions and buffer parities do not care about unit boundaries.  Per step c and slot:
+        // positions and buffer parities do not care about unit boundaries.  Per step c:
         //   S(c + 1) = Q K^T is issued as soon as the softmax warps have taken S(c) out of tensor
         //   memory (S has one buffer per slot; P has its own two), i.e. while they still work on
         //   step c, and it may belong to the next unit;
@@ -290,6 +310,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         // the leading-dimension offset for the MN-major V operand).
         {
             const bool leader = ptx::elect_one();
+            const int s = __shfl_sync(0xffffffffu, warp >> 1, 0);  // this warp's slot
             // Every lane holds the same values; the shuffles tell the compiler so, which lets the
             // loop bounds, ring positions and descriptors live in uniform registers.
             const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_any, 0);
@@ -300,7 +321,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const uint32_t k_lo = ((smem_base + SM::kK) >> 4) | (1u << 16);
             const uint32_t v_lo = ((smem_base + SM::kV) >> 4) | ((SM::kBlkSub >> 4) << 16);
             // S = Q K^T: A = Q tile (K-major), B = K block (K-major), 16 features per MMA.
-            auto issue_qk = [&](int s, uint32_t qb, uint32_t ks) {
+            auto issue_qk = [&](uint32_t qb, uint32_t ks) {
                 const uint32_t qa = q_lo + qb * (SM::kQBuf >> 4) + s * (SM::kQSlot >> 4);
                 const uint32_t kb = k_lo + ks * (SM::kBlkTile >> 4);
                 const uint32_t dst = tmem_base + s * 128;
@@ -312,7 +333,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             };
             // O (+)= P V: A = P (tensor memory, bf16 pairs, buffer = step parity), B = V block
             // (MN-major: features contiguous), 16 keys per MMA.
-            auto issue_pv = [&](int s, uint32_t buf, uint32_t vs, bool acc) {
+            auto issue_pv = [&](uint32_t buf, uint32_t vs, bool acc) {
                 const uint32_t vb = v_lo + vs * (SM::kBlkTile >> 4);
                 const uint32_t dst = tmem_base + 256 + s * D;
                 const uint32_t pa_ = tmem_base + s * 128 + 64 + buf * 32;
@@ -335,50 +356,42 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 return u;
             };
             bool ok = true;
-            // S(c1) for both slots; `first` / `final`: c1 is the first / last step of unit number ul1.
+            // S(c1) of this slot; `first` / `final`: c1 is the first / last step of unit number ul1.
             auto qk_step = [&](uint32_t c1, uint32_t ul1, bool first, bool final, bool wait_taken) {
                 if (first) ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_Q_FULL + (ul1 & 1)), (ul1 >> 1) & 1, abort_flag, a.status, 4));
                 if (ok)
                     ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_K_FULL + c1 % kKStages), (c1 / kKStages) & 1,
                                                           abort_flag, a.status, 5));
-                for (int s = 0; s < 2 && ok; ++s) {
-                    if (wait_taken) {
-                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_S_TAKEN + s), (c1 - 1) & 1, abort_flag, a.status, 8));
-                        if (!ok) break;
-                    }
-                    ptx::tc_fence_after_sync();
-                    if (leader) {
-                        issue_qk(s, ul1 & 1, c1 % kKStages);
-                        ptx::umma_commit(bar(BAR_S_FULL + s));
-                        if (s == 1) {
-                            ptx::umma_commit(bar(BAR_K_EMPTY + c1 % kKStages));
-                            if (final) ptx::umma_commit(bar(BAR_Q_EMPTY + (ul1 & 1)));
-                        }
-                    }
-                    __syncwarp();
+                if (ok && wait_taken)
+                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_S_TAKEN + s), (c1 - 1) & 1, abort_flag, a.status, 8));
+                if (!ok) return;
+                ptx::tc_fence_after_sync();
+                if (leader) {
+                    issue_qk(ul1 & 1, c1 % kKStages);
+                    ptx::umma_commit(bar(BAR_S_FULL + s));
+                    ptx::umma_commit(bar(BAR_K_EMPTY + c1 % kKStages));
+                    if (final) ptx::umma_commit(bar(BAR_Q_EMPTY + (ul1 & 1)));
                 }
+                __syncwarp();
             };
-            // O (+)= P(c) V(c) for both slots; t = step inside its unit (number ul) of n steps.
+            // O (+)= P(c) V(c) of this slot; t = step inside its unit (number ul) of n steps.
             auto pv_step = [&](uint32_t c, uint32_t ul, int t, int n) {
                 ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_V_FULL + c % kVStages), (c / kVStages) & 1,
                                                       abort_flag, a.status, 6));
-                for (int s = 0; s < 2 && ok; ++s) {
+                if (ok)
                     ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_P_FULL + 2 * s + (c & 1)), (c >> 1) & 1, abort_flag, a.status, 7));
-                    if (!ok) break;
-                    if (t == 0 && ul > 0) {
-                        // The previous unit's O must have left tensor memory.
-                        ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_O_FREE + s), (ul - 1) & 1, abort_flag, a.status, 14));
-                        if (!ok) break;
-                    }
-                    ptx::tc_fence_after_sync();
-                    if (leader) {
-                        issue_pv(s, c & 1, c % kVStages, t > 0);
-                        ptx::umma_commit(bar(BAR_O_DONE + 2 * s + (c & 1)));
-                        if (t + 1 == n) ptx::umma_commit(bar(BAR_O_FINAL + s));
-                        if (s == 1) ptx::umma_commit(bar(BAR_V_EMPTY + c % kVStages));
-                    }
-                    __syncwarp();
+                // The previous unit's O must have left tensor memory.
+                if (ok && t == 0 && ul > 0)
+                    ok = __all_sync(0xffffffffu, wait_bar(bar(BAR_O_FREE + s), (ul - 1) & 1, abort_flag, a.status, 14));
+                if (!ok) return;
+                ptx::tc_fence_after_sync();
+                if (leader) {
+                    issue_pv(c & 1, c % kVStages, t > 0);
+                    ptx::umma_commit(bar(BAR_O_DONE + 2 * s + (c & 1)));
+                    if (t + 1 == n) ptx::umma_commit(bar(BAR_O_FINAL + s));
+                    ptx::umma_commit(bar(BAR_V_EMPTY + c % kVStages));
                 }
+                __syncwarp();
             };
             uint32_t kc = 0, ul = 0;
             int n = 0, nn = 0;  // key blocks of this unit and of the next
@@ -490,6 +503,18 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const uint64_t negm_2 = ptx::pack_f32x2(-m, -m);
                 uint64_t sum2[2] = {0ull, 0ull};
                 uint32_t pk[32];
+                // The two slots take turns at the exponentials: slot 0's pass of step kc, then slot
+                // 1's, then slot 0's of step kc + 1, ...  A pass that has the exponential unit to
+                // itself takes half as long, and the rest of a slot's step (loads from and stores to
+                // tensor memory, barrier traffic) then runs beside the other slot's pass instead
+                // of beside its own idle time.  (Turn barrier s completes once per pass of the
+                // other slot, which cannot start its next pass before this slot's, so the parity
+                // asked for is never more than one phase behind.)
+                if (s == 1 || kc > 0) {
+                    ok = wait_bar(bar(BAR_TURN + s), (kc - 1 + s) & 1, abort_flag, a.status, 18);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                }
                 {
 #pragma unroll
                 for (int c = 0; c < 64; c += 4) {
@@ -506,6 +531,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     }
                 }
                 }
+                if (lane == 0) ptx::mbar_arrive(bar(BAR_TURN + (s ^ 1)));
                 float sum;
                 {
                     float s0, s1, s2, s3;
@@ -612,12 +638,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const int row = quad * 32 + lane;
         const int qrow = row & 63;
         const bool store_thread = threadIdx.x == 12 * 32;
-        const uint32_t stage = smem_base + SM::kOStage;
-        uint32_t ul = 0, ns = 0;  // units and staged tiles so far
+        uint32_t ul = 0, ns = 0;  // units and staged slots so far
         bool ok = true;
         for (uint32_t u = blockIdx.x; u < (uint32_t)a.n_units && ok; u += gridDim.x) {
             const Unit w = decode_unit(a, u);
             const int64_t tok = (int64_t)w.i * kBlk + qrow;
+            // The unit's Q buffer is no longer read once its last P V has completed (every S of
+            // the unit was issued before it); its output is staged there.
+            const uint32_t stage = smem_base + SM::kQ + (ul & 1) * SM::kQBuf;
 #pragma unroll 1
             for (int s = 0; s < 2; ++s) {
                 const int head_local = w.sub * 4 + 2 * s + (row >> 6);
@@ -663,59 +691,61 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         }
                     }
                 } else {
-                    uint32_t pk[D / 2];
+                    // Head 2 s + (row >> 6) of the unit: two boxes of 64 tokens x 128 bytes (one per
+                    // 64-feature half); 16-byte chunk j of token t sits at chunk position j ^ (t & 7).
+                    const uint32_t rbase = stage + (uint32_t)(2 * s + (row >> 6)) * SM::kOHead + (uint32_t)qrow * 128u;
 #pragma unroll
                     for (int ch = 0; ch < D / 32; ++ch) {
                         uint32_t orr[32];
                         ptx::tmem_ld32(t_o + ch * 32, orr);
                         ptx::tmem_wait_ld();
+                        if (ch == D / 32 - 1) {
+                            // O is in registers: tensor memory may take the next unit's first P V.
+                            ptx::tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive(bar(BAR_O_FREE + s));
+                        }
 #pragma unroll
-                        for (int c = 0; c < 16; ++c)
-                            pk[ch * 16 + c] = ptx::cvt_bf16x2(__uint_as_float(orr[2 * c]) * inv, __uint_as_float(orr[2 * c + 1]) * inv);
+                        for (int k = 0; k < 4; ++k) {
+                            const int c = 4 * ch + k;  // 16-byte chunk of the row
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                pk[e] = ptx::cvt_bf16x2(__uint_as_float(orr[8 * k + 2 * e]) * inv,
+                                                        __uint_as_float(orr[8 * k + 2 * e + 1]) * inv);
+                            const uint32_t dst = rbase + (uint32_t)(c >> 3) * 8192u + ((uint32_t)((c & 7) ^ (qrow & 7)) << 4);
+                            ptx::st_shared_v4(dst, pk[0], pk[1], pk[2], pk[3]);
+                        }
                     }
-                    ptx::tc_fence_before_sync();
+                    ptx::fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(bar(BAR_O_FREE + s));
-                    // The two heads of the slot go through the staging tile one after the other.
-#pragma unroll 1
-                    for (int hh = 0; hh < 2 && ok; ++hh) {
-                        // The tile is free once the previous bulk stores have read it.
-                        if (store_thread) {
-                            ptx::bulk_wait_read_all();
-                            ptx::mbar_arrive(bar(BAR_STAGE_FREE));
-                        }
-                        ok = wait_bar(bar(BAR_STAGE_FREE), ns & 1, abort_flag, a.status, 16);
-                        ok = __all_sync(0xffffffffu, ok);
-                        if (!ok) break;
-                        if ((row >> 6) == hh) {
-                            // Box (half): 64 tokens x 128 bytes; 16-byte chunk j of token t sits at
-                            // chunk position j ^ (t & 7).
-                            const uint32_t rbase = stage + (uint32_t)qrow * 128u;
-#pragma unroll
-                            for (int c = 0; c < D / 8; ++c) {
-                                const uint32_t dst = rbase + (uint32_t)(c >> 3) * 8192u + ((uint32_t)((c & 7) ^ (qrow & 7)) << 4);
-                                ptx::st_shared_v4(dst, pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-                            }
-                            ptx::fence_proxy_async_smem();
-                        }
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(bar(BAR_STAGE_FULL));
-                        if (warp == 12) {
-                            ok = wait_bar(bar(BAR_STAGE_FULL), ns & 1, abort_flag, a.status, 17);
-                            ok = __all_sync(0xffffffffu, ok);
-                            if (!ok) break;
-                        }
-                        ++ns;
-                        const int hl = w.sub * 4 + 2 * s + hh;
-                        if (store_thread && hl < a.G) {
+                    if (lane == 0) ptx::mbar_arrive(bar(BAR_STAGE_FULL));
+                    // All four warps wait (not only the storing one), so none can arrive for the
+                    // next slot before this phase has completed.
+                    ok = wait_bar(bar(BAR_STAGE_FULL), ns & 1, abort_flag, a.status, 17);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    ++ns;
+                    if (store_thread) {
+                        for (int hh = 0; hh < 2; ++hh) {
+                            const int hl = w.sub * 4 + 2 * s + hh;
+                            if (hl >= a.G) continue;  // the padding head of an odd group
                             for (int dh = 0; dh < DH; ++dh)
-                                ptx::tma_store_4d(&tmO, stage + (uint32_t)dh * 8192u, dh * 64, w.i * kBlk, w.hk * a.G + hl, w.b);
-                            ptx::bulk_commit_group();
+                                ptx::tma_store_4d(&tmO, stage + (uint32_t)(2 * s + hh) * SM::kOHead + (uint32_t)dh * 8192u,
+                                                  dh * 64, w.i * kBlk, w.hk * a.G + hl, w.b);
                         }
+                        ptx::bulk_commit_group();
                     }
                 }
             }
-            if (w.n > 0) ++ul;
+            if (w.n > 0 && ok) {
+                // The Q buffer may be loaded again once the bulk stores have read it.
+                if (store_thread) {
+                    ptx::bulk_wait_read_all();
+                    ptx::mbar_arrive(bar(BAR_STAGE_FREE + (ul & 1)));
+                }
+                ++ul;
+            }
         }
         if (store_thread) ptx::bulk_wait_all();
     }
