@@ -590,13 +590,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
                 }
                 l += sum;
-                if (kc >= 2) {
-                    // P has two buffers (step parity): the P V that read this one two steps ago
-                    // must have completed (normally long ago).
-                    ok = wait_bar(bar(BAR_O_DONE + 2 * s + (kc & 1)), ((kc - 2) >> 1) & 1, abort_flag, a.status, 12);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                }
+                // P has two buffers (step parity).  The P V that read this one two steps ago has
+                // completed: this slot's issuing thread issued it before the S of this step, whose
+                // completion (which covers everything that thread issued earlier) was waited for above.
                 ptx::tmem_st32(t_s0 + 64 + (kc & 1) * 32, pk);
                 // (The hand-over barriers alternate by step parity like the P buffers: the S of step
                 // kc + 2 is issued behind the P V of step kc, so a barrier is never more than one
