@@ -116,7 +116,13 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-i", str(self.gpu), "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                 "-i", str(self.gpu), "-lms", "20"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            # The timed region is a few tens of milliseconds: return only once the sampler is
+            # producing lines, so that it is known to run while the steps are timed.
+            t0 = time.time()
+            while time.time() - t0 < 3.0 and os.path.getsize(self.path) == 0:
+                time.sleep(0.01)
+            self.first_bytes = os.path.getsize(self.path)
         except Exception:
             self.proc = None
 
@@ -132,7 +138,10 @@ class ClockSampler:
         sm, smax, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         try:
-            for line in open(self.path):
+            with open(self.path) as fh:
+                idle = fh.read(getattr(self, "first_bytes", 0)).splitlines()  # taken before start() returned
+                lines = fh.readlines() or idle[-1:]
+            for line in lines:
                 f = [x.strip() for x in line.split(",")]
                 if len(f) < 9:
                     continue
