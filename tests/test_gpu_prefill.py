@@ -118,6 +118,23 @@ def test_paper_block_size_at_32k_on_sampled_rows(pa, oracle):
     compare(o[:, ridx], lse[:, :, ridx], o_ref, lse_ref, "32K, 256-token blocks")
 
 
+@pytest.mark.parametrize("W", [1, 2, 3])
+def test_short_rows_with_several_units_per_cta(pa, oracle, W):
+    """Rows of one, two or three blocks on a sequence long enough that every CTA of the
+    persistent grid walks several work units: the unit-to-unit hand-overs (Q buffers reloaded
+    behind the staged output, first and last step falling together) with nothing in between."""
+    N, Hq, Hkv, D = 64 * 200 + 17, 8, 2, 128        # 201 query blocks x 2 KV heads = 402 units
+    Q = si.bf16_randn((1, N, Hq, D), 700 + W)
+    K = si.bf16_randn((1, N, Hkv, D), 710 + W)
+    V = si.bf16_randn((1, N, Hkv, D), 720 + W)
+    rp, ci = oracle.block_layout(N, 64, W, 0, use_power=False)
+    assert int(np.diff(rp).max()) == W
+    layout = (torch.as_tensor(rp).cuda(), torch.as_tensor(ci).cuda())
+    o, lse = _gpu_prefill(pa, Q, K, V, W, 0, layout=layout)
+    o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, W, 0, use_power=False)
+    compare(o, lse, o_ref, lse_ref, f"short rows W={W}")
+
+
 def test_constant_keys_count_the_attended_tokens(pa, oracle):
     """K rows all equal => LSE_q - s_q = ln |A_q|, |A_q| = 64 * #blocks(row) - (63 - q mod 64);
     holds at any size, so it is checked at 32K with the 7B-like heads."""
