@@ -32,8 +32,8 @@
 // CTA's 16 x 128.
 #ifndef PA_REG_CTRL
 #define PA_REG_CTRL 56
-#define PA_REG_SOFT 168
-#define PA_REG_EPI 120
+#define PA_REG_SOFT 176
+#define PA_REG_EPI 104
 #endif
 // A warpgroup asking for more than the pool holds would wait for ever.
 static_assert(4 * PA_REG_CTRL + 8 * PA_REG_SOFT + 4 * PA_REG_EPI <= 16 * 128, "register split exceeds the CTA's registers");
@@ -59,6 +59,7 @@ struct PrefillArgs {
     int64_t o_sb, o_ss, o_sh;
     int64_t N, n_units;
     int32_t nqb, batch, Hq, Hkv, G, nsub, o_is_f32;
+    uint32_t inv_nsub, inv_Hkv, inv_nqb;  // floor(2^32 / d) of the three divisors of a unit index
     float scale_log2;
 };
 
@@ -105,16 +106,33 @@ struct Unit {
     int32_t b, hk, i, sub, rs, n;
 };
 
+// u / d and u % d with inv = floor(2^32 / d) (2^32 - 1 for d = 1): the high product falls short of
+// the quotient by at most one for every 32-bit u, which one compare puts right.  Every role decodes
+// a unit index per unit, the softmax warps on their critical path; division by a run-time divisor
+// costs some ten times as many instructions.
+__device__ __forceinline__ uint32_t divmod(uint32_t u, uint32_t d, uint32_t inv, uint32_t &rem)
+{
+    uint32_t q = __umulhi(u, inv);
+    uint32_t r = u - q * d;
+    if (r >= d) {
+        ++q;
+        r -= d;
+    }
+    rem = r;
+    return q;
+}
+
 // Unit index -> coordinates (the unit count fits in 30 bits; checked on the host).
 __device__ __forceinline__ Unit decode_unit(const PrefillArgs &a, uint32_t u)
 {
     Unit r;
-    r.sub = (int32_t)(u % (uint32_t)a.nsub);
-    u /= (uint32_t)a.nsub;
-    r.hk = (int32_t)(u % (uint32_t)a.Hkv);
-    u /= (uint32_t)a.Hkv;
-    r.i = a.nqb - 1 - (int32_t)(u % (uint32_t)a.nqb);  // long rows first
-    r.b = (int32_t)(u / (uint32_t)a.nqb);
+    uint32_t rem;
+    u = divmod(u, (uint32_t)a.nsub, a.inv_nsub, rem);
+    r.sub = (int32_t)rem;
+    u = divmod(u, (uint32_t)a.Hkv, a.inv_Hkv, rem);
+    r.hk = (int32_t)rem;
+    r.b = (int32_t)divmod(u, (uint32_t)a.nqb, a.inv_nqb, rem);
+    r.i = a.nqb - 1 - (int32_t)rem;  // long rows first
     r.rs = __ldg(a.row_ptr + r.i);
     r.n = __ldg(a.row_ptr + r.i + 1) - r.rs;
     return r;
@@ -479,9 +497,21 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(bar(BAR_S_TAKEN + s));
                 if (last_is_diag && t == w.n - 1) {
+                    // Keys after the query's own token are masked (-inf).  A warp's 32 rows are
+                    // tokens 0..31 or 32..63 of the block, so half of the columns need no compare:
+                    // for the first half of the rows columns 32..63 are masked for every row, for
+                    // the second half columns 0..32 for none.
+                    if ((quad & 1) == 0) {
 #pragma unroll
-                    for (int c = 0; c < 64; ++c)
-                        if (c > qrow) sr[c] = 0xff800000u;  // -inf
+                        for (int c = 0; c < 32; ++c)
+                            if (c > lane) sr[c] = 0xff800000u;
+#pragma unroll
+                        for (int c = 32; c < 64; ++c) sr[c] = 0xff800000u;
+                    } else {
+#pragma unroll
+                        for (int c = 33; c < 64; ++c)
+                            if (c - 32 > lane) sr[c] = 0xff800000u;
+                    }
                 }
                 // Fast path: p = exp2(s * scale - m) against the reference maximum m carried from
                 // earlier steps (lazy rescaling: O / l at the end is exact whatever reference was
@@ -606,7 +636,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     // Softmax denominators for the epilogue warps (they finish O / l).  The previous
                     // unit's must have been read: that also keeps this slot's statistics barrier at
                     // most one phase ahead of the epilogue.
-                    if (ul > 0) {
+                    // (With three or more steps the wait is implied: this step's S was issued
+                    // behind the unit's first P V, which itself waited for that read.)
+                    if (ul > 0 && w.n < 3) {
                         ok = wait_bar(bar(BAR_O_FREE + s), (ul - 1) & 1, abort_flag, a.status, 13);
                         ok = __all_sync(0xffffffffu, ok);
                         if (!ok) break;
@@ -908,6 +940,8 @@ extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const
     a.G = p->n_q_heads / p->n_kv_heads;
     a.nsub = (a.G + 3) / 4;
     a.n_units = (int64_t)p->batch * nqb * a.Hkv * a.nsub;
+    auto inv32 = [](int32_t d) { return d == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)d); };
+    a.inv_nsub = inv32(a.nsub); a.inv_Hkv = inv32(a.Hkv); a.inv_nqb = inv32(a.nqb);
     if (a.n_units > (int64_t)0x3fffffff) return fail(PA_ERR_SHAPE, "too many work units (%lld)", (long long)a.n_units);
     a.o_is_f32 = p->o_dtype == PA_F32;
     const float scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.0f / sqrtf((float)D);
