@@ -56,7 +56,7 @@ def read_peaks():
 PREFILL_TRAFFIC = dict(
     bytes=2032551424 + 912317952,
     sources={
-        "prefill_sm100.cu": "bc1e1ff5b88e5874cffc50100f8015ca57e3f43692d0b0fb547c4188fada259d",
+        "prefill_sm100.cu": "9d515cbb0f83b5cb9e80385d943efe650dfa3571bd35d4f19124baba46c8bf0d",
         "sm100_ptx.cuh": "cc5cb63f8da5e88ddc941ca016a41fe337c2404ca754e7ea5c384e0a1552a5ca",
     },
 )

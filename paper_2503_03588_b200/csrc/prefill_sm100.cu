@@ -8,15 +8,16 @@
 //   warp 0      TMA producer: the listed K and V blocks, gathered by block index, into two rings
 //               of shared-memory tiles (128-byte swizzle); the next unit's Q tiles early in
 //               the current unit, into the second of two Q buffers
-//   warp 1      tcgen05 issuer.  S = Q K^T of step t+1 is issued as soon as the softmax warps
-//               hold S of step t in registers (one S buffer per slot), so those logits are
-//               ready when step t ends, across unit boundaries too; O += P V is issued when
-//               P has been handed over (P has its own two buffers in tensor memory)
+//   warps 1, 3  tcgen05 issuers, one per slot.  S = Q K^T of step t+1 is issued as soon as the
+//               softmax warps hold S of step t in registers (one S buffer per slot), so those
+//               logits are ready when step t ends, across unit boundaries too; O += P V is issued
+//               when P has been handed over (P has its own two buffers in tensor memory)
 //   warp 2      tensor-memory allocation
 //   warps 4-7   online softmax of slot 0 (thread = tile row = TMEM lane), LSE
-//   warps 8-11  online softmax of slot 1
-//   warps 12-15 epilogue: O / l out of tensor memory, staged in shared memory head by head,
-//               bulk tensor stores to global memory; runs beside the next unit's first steps
+//   warps 8-11  online softmax of slot 1; the two slots take turns at the exponentials
+//   warps 12-15 epilogue: O / l out of tensor memory into the finished unit's own Q buffer
+//               (swizzled for the bulk tensor stores to global memory); runs beside the next
+//               unit's first steps
 // Warps 0-3 and 12-15 give registers back (setmaxnreg) and the softmax warpgroups take them.
 // Every barrier wait is bounded; a wait that runs out records PA_ERR_TIMEOUT in the status
 // block, raises a CTA-wide abort flag and the CTA drains and exits (no trap, no endless spin).
