@@ -463,6 +463,13 @@ def run_ours(args):
 
     value = flops_all / (ms * 1e-3) / 1e12
     achieved = flops / (prefill_ms * 1e-3) / 1e12
+    # Which measured bf16 peak the kernel is held against: the burst figure while the timed region
+    # ran at full clocks (a short run), the sustained one once the median SM clock sampled during it
+    # is more than 8 % below the maximum (a long run of a kernel that draws the full board power).  Both fractions
+    # are in the line.
+    capped = clocks.get("sm_mhz") is not None and clocks["sm_mhz"] < 0.92 * clocks["sm_max_mhz"]
+    peak = peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"]
+    peak_kind = " sustained bf16 (power-capped clocks in the timed region)" if capped else " burst bf16"
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
                 ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                 data="synthetic",
@@ -472,10 +479,11 @@ def run_ours(args):
                             decode_workload=wd.name, l2="inputs larger than L2 (Q+K+V+O = 2.4 GB per step)",
                             parallelism="replicas" if world > 1 else "single"),
                 clocks=clocks,
-                roofline=dict(bound="tensor", achieved=achieved, peak=peaks["bf16_tflops"], unit="TFLOP/s",
-                              frac=achieved / peaks["bf16_tflops"], traffic=prefill_traffic(),
-                              peak_source=peaks["source"] + " burst bf16", kernel="prefill_kernel<128>",
+                roofline=dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s",
+                              frac=achieved / peak, traffic=prefill_traffic(),
+                              peak_source=peaks["source"] + peak_kind, kernel="prefill_kernel<128>",
                               kernel_ms=prefill_ms,
+                              frac_of_burst=achieved / peaks["bf16_tflops"],
                               frac_of_sustained=achieved / peaks["bf16_tflops_sustained"]),
                 prefill_32k=prefill_32k,
                 decode=dict(metric="decode_kv_gbs", value=dec_gbs, unit="GB/s", us_per_call=dec_us,
