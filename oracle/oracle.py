@@ -127,16 +127,26 @@ def block_predicate(i: int, j: int, W: int, S: int = 1, use_power: bool = True) 
     return (d < W) or (use_power and (d & (d - 1)) == 0) or (j < S)
 
 
+def block_row(i: int, W: int, S: int = 1, use_power: bool = True) -> np.ndarray:
+    """Every key block j = 0..i that block_predicate lists for query block i, ascending: the
+    predicate written out on the whole index range at once (no candidate pruning)."""
+    j = np.arange(i + 1, dtype=np.int64)
+    d = i - j
+    keep = (d < W) | (j < S)
+    if use_power:
+        keep |= (d & (d - 1)) == 0
+    return j[keep].astype(np.int32)
+
+
 def block_layout(N: int, B: int, W: int, S: int = 1,
                  use_power: bool = True) -> Tuple[np.ndarray, np.ndarray]:
-    """Block-level enumeration of every (i, j) pair; usable at large N."""
+    """Block-level enumeration of every (i, j) pair with j <= i; usable at large N."""
     nb = -(-N // B)
     row_ptr = np.zeros(nb + 1, dtype=np.int32)
     cols = []
     for i in range(nb):
-        js = [j for j in _candidate_blocks(i, W, S, use_power)
-              if block_predicate(i, j, W, S, use_power)]
-        cols.append(np.asarray(js, dtype=np.int32))
+        js = block_row(i, W, S, use_power)
+        cols.append(js)
         row_ptr[i + 1] = row_ptr[i] + len(js)
     col_idx = np.concatenate(cols) if cols else np.zeros(0, dtype=np.int32)
     return row_ptr, col_idx.astype(np.int32)
@@ -167,27 +177,12 @@ def tile_layout(N: int, B: int, W: int, S: int, T: int,
     cols = []
     for ti in range(nt):
         i = ti // r
-        js = [tj for j in _candidate_blocks(i, W, S, use_power) if block_predicate(i, j, W, S, use_power)
-              for tj in range(j * r, min((j + 1) * r, ti + 1))]
+        js = [tj for j in block_row(i, W, S, use_power)
+              for tj in range(int(j) * r, min((int(j) + 1) * r, ti + 1))]
         cols.append(np.asarray(js, dtype=np.int32))
         row_ptr[ti + 1] = row_ptr[ti] + len(js)
     col_idx = np.concatenate(cols) if cols else np.zeros(0, dtype=np.int32)
     return row_ptr, col_idx.astype(np.int32)
-
-
-def _candidate_blocks(i: int, W: int, S: int, use_power: bool):
-    """All j <= i when that is cheap; else only the j that can possibly pass (a superset of
-    sink, window and power-of-two distances), still filtered by block_predicate."""
-    if i < 4096:
-        return range(i + 1)
-    cand = set(range(min(S, i + 1)))
-    cand.update(range(max(0, i - W + 1), i + 1))
-    cand.add(i)
-    k = 1
-    while k <= i:
-        cand.add(i - k)
-        k *= 2
-    return sorted(cand)
 
 
 def block_adjacency(n_blocks: int, W: int, S: int = 1, use_power: bool = True) -> list:

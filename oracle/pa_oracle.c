@@ -37,25 +37,24 @@ static double bf16_to_double(uint16_t h)
     return (double)f;
 }
 
+/* True for 0, 1, 2, 4, 8, ...: at most one bit set. */
+static int is_zero_or_power_of_two(int64_t d) { return (d & (d - 1)) == 0; }
+
 /*
- * Algorithm 1 (Section 3.3), token level.
- *   blk_qk      = floor(q_idx / B) - floor(kv_idx / B)
- *   mask_window = blk_qk < W
- *   mask_power  = (blk_qk & (blk_qk - 1)) == 0            (true for blk_qk = 0, 1, 2, 4, 8, ...)
- *   mask_sink   = kv_idx < B                              (here: kv_idx < sink_blocks * B)
- *   mask_causal = q_idx >= kv_idx
- *   result      = mask_causal and (mask_window or mask_power or mask_sink)
- * The power term is only meaningful for blk_qk >= 0; causality makes every other case false.
+ * The mask of Algorithm 1 (Section 3.3) for one (query, key) token pair.  A key after the query
+ * is never attended.  Otherwise let d >= 0 be the distance between the B-token blocks that hold
+ * the two tokens; the key is attended when its block lies inside the local window (d < W), at a
+ * power-of-two block distance (or in the query's own block, d = 0), or among the first
+ * sink_blocks * B tokens of the sequence.
  */
 int pa_oracle_mask(int64_t q_idx, int64_t kv_idx, int64_t B, int64_t W, int64_t sink_blocks,
                    int use_power)
 {
-    if (q_idx < kv_idx) return 0; /* mask_causal */
-    int64_t blk_qk = q_idx / B - kv_idx / B;
-    int mask_window = blk_qk < W;
-    int mask_power = use_power && ((blk_qk & (blk_qk - 1)) == 0);
-    int mask_sink = kv_idx < sink_blocks * B;
-    return mask_window || mask_power || mask_sink;
+    if (kv_idx > q_idx) return 0;
+    const int64_t d = q_idx / B - kv_idx / B;
+    if (d < W) return 1;
+    if (use_power && is_zero_or_power_of_two(d)) return 1;
+    return kv_idx < sink_blocks * B;
 }
 
 /* Dense mask row of query q over kv in [0, n_keys): row[kv] in {0,1}. */

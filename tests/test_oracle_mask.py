@@ -193,6 +193,24 @@ def test_row_length_closed_form(oracle):
             assert sorted(i - j for j in row) == sorted(ds)
 
 
+def test_block_row_at_large_indices(oracle):
+    """Rows far beyond the sizes the brute force reaches: the vector form of the block predicate
+    against the scalar one on every j <= i, and against the closed-form set of distances."""
+    for (W, S) in [(5, 1), (0, 0), (9, 3), (26, 4)]:
+        for i in (4095, 4096, 4097, 5000, 8191, 8192, 16383, 16384, 70001):
+            row = oracle.block_row(i, W, S)
+            scalar = [j for j in range(i + 1) if oracle.block_predicate(i, j, W, S)]
+            assert row.tolist() == scalar, (i, W, S)
+            ds = set(range(min(max(W, 1), i + 1))) | {i - j for j in range(min(S, i + 1))}
+            k = 1
+            while k <= i:
+                ds.add(k)
+                k *= 2
+            assert sorted(i - j for j in row.tolist()) == sorted(ds), (i, W, S)
+        nopow = oracle.block_row(5000, W, S, use_power=False)
+        assert nopow.tolist() == [j for j in range(5001) if oracle.block_predicate(5000, j, W, S, False)]
+
+
 def test_active_block_counts_scale_as_n_log_n(oracle):
     """Section 4.5: O(N log N).  nnz / (nqb * log2 nqb) stays bounded and nnz < dense triangle."""
     prev = None
