@@ -48,6 +48,17 @@ const char *pa_last_error_message(void);
 /* major * 10000 + minor * 100 + patch */
 int pa_version(void);
 
+/* Environment switches (PA_VALIDATE, PA_DECODE_PATH, PA_DECODE_CLUSTER, PA_DECODE_STAGES; each is
+ * described at the call it affects) are read once, when a call first needs them.  This re-reads
+ * them; tests and measurement scripts call it after changing the environment. */
+void pa_reload_environment(void);
+
+/* Limit, in GPU clock cycles, of every bounded barrier wait inside the prefill kernel (a wait that
+ * runs out ends the kernel with PA_ERR_TIMEOUT in its status block, see pa_prefill_status).
+ * cycles <= 0 restores the default of about two seconds.  Process-wide; applies to calls made
+ * after it returns. */
+void pa_set_wait_limit_cycles(int64_t cycles);
+
 /* ------------------------------------------------------------------------------------------
  * Layout: Algorithm 1 (Section 3.3) evaluated on blocks.
  *
@@ -137,7 +148,8 @@ size_t pa_prefill_workspace_bytes(const pa_prefill_params *p);
  * Enqueues one memset and one kernel.  Errors: PA_ERR_INVALID_ARG, PA_ERR_SHAPE,
  * PA_ERR_ALIGNMENT, PA_ERR_LAYOUT (nnz < n_qblocks), PA_ERR_WORKSPACE, PA_ERR_UNSUPPORTED,
  * PA_ERR_CUDA.  Outputs are undefined after a failure.  The CSR is trusted: extents that point
- * outside col_idx would be read out of bounds.  With PA_VALIDATE=1 in the environment the call
+ * outside col_idx would be read out of bounds.  With PA_VALIDATE=1 in the environment (see
+ * pa_reload_environment) the call
  * first checks it on the device (row_ptr from 0 to nnz, extents inside col_idx, every index in
  * [0, row] and ascending within its row), synchronises the stream, and returns PA_ERR_LAYOUT with
  * the first offending row in pa_last_error_message() instead of enqueuing the kernel; do not
@@ -168,8 +180,8 @@ typedef struct {
     pa_dtype o_dtype;
 } pa_decode_params;
 
-/* Bytes of device scratch for the split-K partial results (m, l, o[head_dim] per query head
- * and chunk of the block list). */
+/* Bytes of device scratch: a 256-byte status block, then the split-K partial results (m, l,
+ * o[head_dim] per query head and chunk of the block list). */
 size_t pa_decode_workspace_bytes(const pa_decode_params *p);
 
 /* q: device bf16 [batch, n_q_heads, head_dim] contiguous.  k_cache, v_cache: device bf16 by
@@ -178,28 +190,91 @@ size_t pa_decode_workspace_bytes(const pa_decode_params *p);
  * o: device [batch, n_q_heads, head_dim] contiguous, o_dtype.  lse: device fp32
  * [batch, n_q_heads].  When a row's window, power-of-two and sink candidates number at most 32
  * (window_blocks + sink_blocks + log2 of the row count: any default-window row up to millions of
- * tokens) one kernel is enqueued: a thread-block cluster per (sequence, KV head)
- * shares the row's blocks, each CTA runs an online softmax over its blocks, and the partial
- * results are merged inside the cluster with the log-sum-exp rule
- * m = max m_c, l = sum l_c e^(m_c - m), o = sum o_c e^(m_c - m) / l; the workspace is then not
- * touched.  Otherwise two kernels are enqueued: partial attention per (sequence, KV head,
- * block) into the workspace, then the same merge.  The workspace must be given in both cases.
- * Calls that share a workspace must not overlap on the GPU.  Environment switches read on every
- * call (for tests and measurements): PA_DECODE_PATH=splitk forces the two-kernel path,
- * PA_DECODE_CLUSTER=n (1..8) sets the cluster size (default: 8 for small calls, fewer CTAs per
- * row as batch x n_kv_heads grows, down to one), PA_DECODE_STAGES=n (1..4) the number of key
- * blocks a CTA keeps in flight when it has more blocks than that. */
+ * tokens) the row kernel runs: a row's key blocks are dealt to R chunks; in each CTA a producer
+ * warp fetches the blocks of its chunk by TMA into a ring of shared-memory stages and four warps
+ * run an online softmax over them.  Small calls (batch x n_kv_heads up to about 70) are one
+ * launch in which the R CTAs of a row form a thread-block cluster and merge their results through
+ * distributed shared memory with the log-sum-exp rule
+ * m = max m_c, l = sum l_c e^(m_c - m), o = sum o_c e^(m_c - m) / l.  Larger calls run a
+ * persistent grid (two CTAs per SM) over the (row, chunk) items and, unless R is 1, a second small
+ * kernel that merges each row's R partial results from the workspace.  Rows with more candidates
+ * take two kernels: partial attention per (sequence, KV head, block) into the workspace, then
+ * the same merge.  The workspace (>= pa_decode_workspace_bytes(p), 16-byte aligned) must always
+ * be given; its first word is a status block (see pa_decode_status).
+ * Calls that share a workspace must not overlap on the GPU.  Environment switches (for tests and
+ * measurements, see pa_reload_environment): PA_DECODE_PATH=splitk forces the two-kernel path,
+ * =cluster / =persist the two forms of the row kernel; PA_DECODE_CLUSTER=n (1..8) sets R (default:
+ * for small calls enough CTAs to fill the GPU about three times, for large ones the smallest
+ * split that loads the SMs evenly); PA_DECODE_STAGES=n (1..6) the number of key blocks a CTA keeps
+ * in flight. */
 pa_status pa_decode(const pa_decode_params *p, const void *q, const void *k_cache,
                     const void *v_cache, const int32_t *cache_lens, void *o, float *lse,
                     void *workspace, size_t workspace_bytes, void *stream);
 
-/* The key-block list the decode kernel derives for one cache length, written on the device by
- * the same device function the kernel uses: out_blocks device int32[capacity], out_count
- * device int32[1].  Equals row floor((cache_len-1)/block) of pa_build_layout(cache_len, ...).
- * capacity >= 64 + window_blocks + sink_blocks is always enough. */
+/* Synchronises `stream` and reads back the status block a decode call (pa_decode, pa_decode_paged)
+ * left in `workspace`.  Returns PA_OK, PA_ERR_TIMEOUT (a bounded barrier wait inside the kernel
+ * ran out; *detail, a host pointer that may be NULL, receives a code naming the wait) or
+ * PA_ERR_CUDA. */
+pa_status pa_decode_status(const void *workspace, void *stream, int32_t *detail);
+
+/* The key-block list of one cache length as the two-kernel path derives it (ascending), written
+ * on the device by the device function that path uses: out_blocks device int32[capacity],
+ * out_count device int32[1].  Equals row floor((cache_len-1)/block) of pa_build_layout(cache_len,
+ * ...).  capacity >= 64 + window_blocks + sink_blocks is always enough. */
 pa_status pa_decode_block_list(int64_t cache_len, int32_t block, int32_t window_blocks,
                                int32_t sink_blocks, int32_t *out_blocks, int32_t *out_count,
                                int32_t capacity, void *stream);
+
+/* The key-block SET of one cache length as the single-launch kernel derives it: that kernel
+ * enumerates window, power-of-two and sink candidates one per lane and does not sort them (the
+ * order of the keys does not matter for Eq. (1)).  Written by the kernel's own device function in
+ * lane order: out_blocks device int32[capacity >= 32], out_count device int32[1].  As a set it
+ * equals row floor((cache_len-1)/block) of pa_build_layout(cache_len, ...), without duplicates.
+ * PA_ERR_SHAPE when the candidates number more than 32 (such rows take the two-kernel path). */
+pa_status pa_decode_row_block_set(int64_t cache_len, int32_t block, int32_t window_blocks,
+                                  int32_t sink_blocks, int32_t *out_blocks, int32_t *out_count,
+                                  int32_t capacity, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Decode against a paged KV cache (Section 4.5 measures 16K-128K-token inputs followed by 1024
+ * decoding steps; Section 4.1: the same pattern in both phases).  Keys and values live in a pool
+ * of pages of `block` (= 64) tokens, [n_pages, block, n_kv_heads, head_dim] by strides
+ * (k.batch / v.batch is the PAGE stride, .seq the token stride inside a page, .head the head
+ * stride).  block_table[b, j] (device int32 [batch, max_blocks_per_seq]) is the page that holds
+ * tokens [64 j, 64 j + 64) of sequence b, so a key block of the mask is exactly one page.  The
+ * caller owns the pool and the table and decides which pages a sequence gets; the library
+ * allocates nothing.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    int32_t batch, n_q_heads, n_kv_heads, head_dim; /* head_dim in {64, 128}; group <= 8    */
+    int32_t block, window_blocks, sink_blocks;      /* block = page size, must be 64        */
+    int32_t n_pages;                                /* pages in the pool                    */
+    int32_t max_blocks_per_seq;                     /* row length of block_table            */
+    float softmax_scale;                            /* 0 => 1 / sqrt(head_dim)              */
+    pa_strides k, v;                                /* pool strides: page, token, head      */
+    pa_dtype o_dtype;
+} pa_paged_params;
+
+size_t pa_decode_paged_workspace_bytes(const pa_paged_params *p);
+
+/* As pa_decode, with the key blocks fetched through block_table.  cache_lens[b] in
+ * [1, 64 * max_blocks_per_seq].  A table entry outside [0, n_pages) does not fault: on the
+ * single-launch path that page reads as zeros, on the two-kernel path it is clamped into the
+ * pool; the sequence's result is then meaningless. */
+pa_status pa_decode_paged(const pa_paged_params *p, const void *q, const void *k_pool,
+                          const void *v_pool, const int32_t *block_table,
+                          const int32_t *cache_lens, void *o, float *lse, void *workspace,
+                          size_t workspace_bytes, void *stream);
+
+/* Appends one token per sequence: k_new, v_new (device bf16 [batch, n_kv_heads, head_dim]
+ * contiguous) are written at position cache_lens[b] (the page block_table[b, cache_lens[b] / 64],
+ * slot cache_lens[b] mod 64) and cache_lens[b] (device int32, read and written) grows by one.
+ * A sequence whose table has no page for that position (position beyond 64 * max_blocks_per_seq,
+ * or an entry outside [0, n_pages)) is left unchanged: nothing written, length kept.  Two small
+ * kernels are enqueued on `stream`. */
+pa_status pa_kv_append(const pa_paged_params *p, const void *k_new, const void *v_new,
+                       void *k_pool, void *v_pool, const int32_t *block_table,
+                       int32_t *cache_lens, void *stream);
 
 /* ------------------------------------------------------------------------------------------
  * Decode without any allocation.  (The paper has no counterpart to this entry point; it exists
@@ -210,21 +285,26 @@ pa_status pa_decode_block_list(int64_t cache_len, int32_t block, int32_t window_
  * runtime owns every byte of the device and hands out none, and real-time serving loops in which
  * an allocation (which may synchronise the device or fail) is forbidden once warm-up is over.
  * pa_decode asks such callers for a workspace they have no means to provide.  pa_decode_static
- * computes exactly what pa_decode computes, but keeps the split-K partial results in an array of
- * PA_DECODE_STATIC_SCRATCH_BYTES bytes that is part of the library image.  Every GPU on which
- * the library's code gets loaded carries that array until the process exits.
+ * computes exactly what pa_decode computes, but keeps the workspace (the status block and, on the
+ * two-kernel path, the split-K partial results) in an array of PA_DECODE_STATIC_SCRATCH_BYTES
+ * bytes that is part of the library image.  Every GPU on which the library's code gets loaded
+ * carries that array until the process exits.
  *
  * Arguments q, k_cache, v_cache, cache_lens, o, lse and stream: as for pa_decode.
- *   - Limit: pa_decode_workspace_bytes(p) must not exceed PA_DECODE_STATIC_SCRATCH_BYTES,
- *     otherwise PA_ERR_WORKSPACE is returned (with a message giving both numbers) and nothing is
- *     launched.  The batch-8, 28-head, head_dim-128, 128K-token workload needs about 2 MB.
+ *   - Limit: a problem that takes the two-kernel path (long windows, or PA_DECODE_PATH=splitk)
+ *     needs pa_decode_workspace_bytes(p) bytes of the array; beyond
+ *     PA_DECODE_STATIC_SCRATCH_BYTES the call returns PA_ERR_WORKSPACE (with a message giving both
+ *     numbers) and launches nothing.  The batch-8, 28-head, head_dim-128, 128K-token workload
+ *     would need about 2 MB there.  A problem that takes the single-launch path uses only the
+ *     256-byte status block, whatever its size.
  *   - The call itself performs no device allocation or free, and calls no library that does.
  *   - The first call on each device looks up the array's device address (a one-time set-up that
  *     loads the library's device code if it is not loaded yet).  Make that first call during
  *     start-up, outside any stream capture.
  *   - All calls on one device share the one array, and it still holds the previous call's
- *     partial results when the next call starts.  Nothing in it has to start at zero: each call
- *     overwrites every entry it later reads.  Because the array is shared, two calls that run
+ *     status and partial results when the next call starts.  The status word is cleared by the
+ *     kernels themselves at their start; nothing else has to start at zero: each call overwrites
+ *     every entry it later reads.  Because the array is shared, two calls that run
  *     on the GPU at the same time (different streams, or different host threads) overwrite each
  *     other's partial results; issue them on one stream or order them yourself.
  * ------------------------------------------------------------------------------------------ */

@@ -20,9 +20,12 @@ PA_BF16, PA_F32 = 0, 1
 STATUS_NAMES = ["PA_OK", "PA_ERR_INVALID_ARG", "PA_ERR_SHAPE", "PA_ERR_ALIGNMENT", "PA_ERR_LAYOUT",
                 "PA_ERR_WORKSPACE", "PA_ERR_UNSUPPORTED", "PA_ERR_CUDA", "PA_ERR_TIMEOUT"]
 
-EXPORTS = ["pa_status_string", "pa_last_error_message", "pa_version", "pa_layout_size",
-           "pa_build_layout", "pa_tile_layout_size", "pa_build_tile_layout", "pa_prefill_workspace_bytes", "pa_prefill", "pa_prefill_status",
-           "pa_decode_workspace_bytes", "pa_decode", "pa_decode_block_list", "pa_decode_static"]
+EXPORTS = ["pa_status_string", "pa_last_error_message", "pa_version", "pa_reload_environment",
+           "pa_set_wait_limit_cycles", "pa_layout_size", "pa_build_layout", "pa_tile_layout_size",
+           "pa_build_tile_layout", "pa_prefill_workspace_bytes", "pa_prefill", "pa_prefill_status",
+           "pa_decode_workspace_bytes", "pa_decode", "pa_decode_status", "pa_decode_block_list",
+           "pa_decode_row_block_set", "pa_decode_paged_workspace_bytes", "pa_decode_paged", "pa_kv_append",
+           "pa_decode_static"]
 
 
 class PaError(RuntimeError):
@@ -49,6 +52,14 @@ class pa_decode_params(ctypes.Structure):
                 ("sink_blocks", ctypes.c_int32), ("max_len", ctypes.c_int64),
                 ("softmax_scale", ctypes.c_float), ("k", pa_strides), ("v", pa_strides),
                 ("o_dtype", ctypes.c_int)]
+
+
+class pa_paged_params(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("block", ctypes.c_int32), ("window_blocks", ctypes.c_int32),
+                ("sink_blocks", ctypes.c_int32), ("n_pages", ctypes.c_int32),
+                ("max_blocks_per_seq", ctypes.c_int32), ("softmax_scale", ctypes.c_float),
+                ("k", pa_strides), ("v", pa_strides), ("o_dtype", ctypes.c_int)]
 
 
 def _load() -> ctypes.CDLL:
@@ -86,6 +97,21 @@ def _load() -> ctypes.CDLL:
     lib.pa_decode_block_list.argtypes = [i64, i32, i32, i32, vp, vp, i32, vp]
     lib.pa_decode_static.restype = ctypes.c_int
     lib.pa_decode_static.argtypes = [ctypes.POINTER(pa_decode_params), vp, vp, vp, vp, vp, vp, vp]
+    lib.pa_reload_environment.restype = None
+    lib.pa_reload_environment.argtypes = []
+    lib.pa_set_wait_limit_cycles.restype = None
+    lib.pa_set_wait_limit_cycles.argtypes = [i64]
+    lib.pa_decode_status.restype = ctypes.c_int
+    lib.pa_decode_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+    lib.pa_decode_row_block_set.restype = ctypes.c_int
+    lib.pa_decode_row_block_set.argtypes = [i64, i32, i32, i32, vp, vp, i32, vp]
+    lib.pa_decode_paged_workspace_bytes.restype = ctypes.c_size_t
+    lib.pa_decode_paged_workspace_bytes.argtypes = [ctypes.POINTER(pa_paged_params)]
+    lib.pa_decode_paged.restype = ctypes.c_int
+    lib.pa_decode_paged.argtypes = [ctypes.POINTER(pa_paged_params), vp, vp, vp, vp, vp, vp, vp, vp,
+                                    ctypes.c_size_t, vp]
+    lib.pa_kv_append.restype = ctypes.c_int
+    lib.pa_kv_append.argtypes = [ctypes.POINTER(pa_paged_params), vp, vp, vp, vp, vp, vp, vp]
     return lib
 
 
@@ -116,6 +142,14 @@ def pa_version() -> int:
 
 def pa_status_string(status: int) -> str:
     return lib.pa_status_string(status).decode()
+
+
+def pa_reload_environment() -> None:
+    lib.pa_reload_environment()
+
+
+def pa_set_wait_limit_cycles(cycles: int) -> None:
+    lib.pa_set_wait_limit_cycles(int(cycles))
 
 
 def pa_layout_size(seq_len: int, block: int, window_blocks: int, sink_blocks: int) -> Tuple[int, int]:
@@ -237,6 +271,65 @@ def pa_decode_block_list(cache_len: int, block: int, window_blocks: int, sink_bl
                                     capacity, _stream()))
     n = int(cnt.item())
     return out[:n].clone()
+
+
+def pa_decode_status(workspace: torch.Tensor) -> int:
+    """Synchronises the current stream; raises PaError if the decode kernel recorded a timeout."""
+    detail = ctypes.c_int32(0)
+    _check(lib.pa_decode_status(_ptr(workspace), _stream(), ctypes.byref(detail)))
+    return int(detail.value)
+
+
+def pa_decode_row_block_set(cache_len: int, block: int, window_blocks: int, sink_blocks: int,
+                            device="cuda") -> torch.Tensor:
+    """The single-launch decode kernel's (unsorted) key-block set for one cache length."""
+    out = torch.full((32,), -1, dtype=torch.int32, device=device)
+    cnt = torch.zeros(1, dtype=torch.int32, device=device)
+    _check(lib.pa_decode_row_block_set(cache_len, block, window_blocks, sink_blocks, _ptr(out), _ptr(cnt), 32,
+                                       _stream()))
+    n = int(cnt.item())
+    return out[:n].clone()
+
+
+def paged_params(q, k_pool, v_pool, block_table, window_blocks: int, sink_blocks: int, block: int = 64,
+                 softmax_scale: float = 0.0, o_dtype=torch.bfloat16) -> pa_paged_params:
+    """q [batch, Hq, D]; pools [n_pages, block, Hkv, D]; block_table int32 [batch, max_blocks]."""
+    batch, hq, d = q.shape
+    assert k_pool.shape[1] == block and block_table.dtype == torch.int32 and block_table.is_contiguous()
+    return pa_paged_params(batch, hq, k_pool.shape[2], d, block, window_blocks, sink_blocks, k_pool.shape[0],
+                           block_table.shape[1], float(softmax_scale), _strides4(k_pool), _strides4(v_pool),
+                           PA_F32 if o_dtype == torch.float32 else PA_BF16)
+
+
+def pa_decode_paged_workspace_bytes(params: pa_paged_params) -> int:
+    return int(lib.pa_decode_paged_workspace_bytes(ctypes.byref(params)))
+
+
+def pa_decode_paged(q, k_pool, v_pool, block_table, cache_lens, window_blocks: int, sink_blocks: int, o=None,
+                    lse=None, workspace=None, block: int = 64, softmax_scale: float = 0.0, o_dtype=torch.bfloat16):
+    """pa_decode against a pool of 64-token pages.  Returns (o, lse, workspace)."""
+    batch, hq, d = q.shape
+    if o is None:
+        o = torch.empty((batch, hq, d), dtype=o_dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty((batch, hq), dtype=torch.float32, device=q.device)
+    params = paged_params(q, k_pool, v_pool, block_table, window_blocks, sink_blocks, block, softmax_scale, o.dtype)
+    if workspace is None:
+        workspace = torch.empty(max(pa_decode_paged_workspace_bytes(params), 16), dtype=torch.uint8, device=q.device)
+    assert cache_lens.dtype == torch.int32 and q.is_contiguous() and o.is_contiguous()
+    _check(lib.pa_decode_paged(ctypes.byref(params), _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(block_table),
+                               _ptr(cache_lens), _ptr(o), _ptr(lse), _ptr(workspace), workspace.numel(), _stream()))
+    return o, lse, workspace
+
+
+def pa_kv_append(k_new, v_new, k_pool, v_pool, block_table, cache_lens, block: int = 64) -> None:
+    """k_new, v_new [batch, Hkv, D] go to position cache_lens[b] of each sequence; cache_lens grows by one."""
+    batch, hkv, d = k_new.shape
+    assert k_new.is_contiguous() and v_new.is_contiguous() and cache_lens.dtype == torch.int32
+    params = pa_paged_params(batch, hkv, hkv, d, block, 0, 0, k_pool.shape[0], block_table.shape[1], 0.0,
+                             _strides4(k_pool), _strides4(v_pool), PA_BF16)
+    _check(lib.pa_kv_append(ctypes.byref(params), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool),
+                            _ptr(block_table), _ptr(cache_lens), _stream()))
 
 
 PA_DECODE_STATIC_SCRATCH_BYTES = 4 << 20

@@ -1,4 +1,5 @@
-// Shared host-side helpers of the library: error reporting and argument checks.
+// Shared host-side helpers of the library: error reporting, argument checks, and the small
+// per-process caches (device properties, environment switches) that keep repeated calls cheap.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -14,8 +15,33 @@ void clear_error();
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// PA_OK if the current device is an sm_100 part, else PA_ERR_UNSUPPORTED / PA_ERR_CUDA.
-pa_status require_sm100();
+constexpr int kMaxDevices = 64;
+
+// Properties of the current device, looked up once per device and process.
+struct DeviceInfo {
+    int device, sms, cc_major;
+};
+// PA_OK with *out filled in if the current device is an sm_100 part, else PA_ERR_UNSUPPORTED /
+// PA_ERR_CUDA.
+pa_status current_sm100_device(DeviceInfo *out);
+
+// One-time per-device set-up steps (kernel attributes) are keyed by these slots.
+enum DeviceOnce : int { ONCE_PREFILL_ATTR = 0, ONCE_DECODE_ATTR, ONCE_BACKWARD_ATTR, ONCE_COUNT };
+// True exactly once per (device, slot); the caller then performs the step and, if it fails, calls
+// device_once_reset so that a later call tries again.
+bool device_once_begin(int device, DeviceOnce slot);
+void device_once_reset(int device, DeviceOnce slot);
+
+// Environment switches (for tests and measurements).  They are read when the library first needs
+// them and again on pa_reload_environment().
+struct EnvSwitches {
+    int decode_path;     // PA_DECODE_PATH: 0 unset, 1 splitk, 2 cluster, 3 persistent
+    int decode_cluster;  // PA_DECODE_CLUSTER=1..8 chunks per row, 0 = chosen from the problem size
+    int decode_stages;   // PA_DECODE_STAGES=1..8, 0 = chosen from the problem size
+    int decode_ctas_per_sm;  // PA_DECODE_CTAS_PER_SM=n: size of the persistent grid (default 2 per SM)
+    int validate;        // PA_VALIDATE=1
+};
+EnvSwitches env_switches();
 
 #define PA_CUDA_OK(expr)                                                                    \
     do {                                                                                    \

@@ -26,8 +26,11 @@
 #include <math.h>
 #include <stdlib.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 
 // Registers per thread by role: 4 control warps, 8 softmax warps, 4 epilogue warps share the
 // CTA's 16 x 128.
@@ -50,7 +53,7 @@ constexpr uint32_t kTmemCols = 512;    // slot s: S at columns 128 s, P buffers 
 // A step's row sum above this limit sends the step through the exact path (new reference).
 constexpr float kSumLimit = 1048576.0f;  // 2^20
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logits: rescale O only when the row max grows by more
-constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
+constexpr long long kWaitCycles = 4000000000ll;  // default limit of a barrier wait: ~2 s at 2 GHz
 
 struct PrefillArgs {
     const int32_t *row_ptr, *col_idx;
@@ -62,6 +65,7 @@ struct PrefillArgs {
     int32_t nqb, batch, Hq, Hkv, G, nsub, o_is_f32;
     uint32_t inv_nsub, inv_Hkv, inv_nqb;  // floor(2^32 / d) of the three divisors of a unit index
     float scale_log2;
+    long long wait_cycles;  // limit of every barrier wait, in clock cycles
 };
 
 template <int D>
@@ -139,27 +143,6 @@ __device__ __forceinline__ Unit decode_unit(const PrefillArgs &a, uint32_t u)
     return r;
 }
 
-// Bounded mbarrier wait.  Returns false after a timeout (recorded once) or once another thread
-// of the CTA has raised the abort flag.
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                         int32_t *status, int code)
-{
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    uint32_t it = 0;
-    while (true) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
-        if ((++it & 63u) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) break;
-        }
-    }
-    if (atomicCAS(status, 0, (int)PA_ERR_TIMEOUT) == 0) status[1] = code;
-    *abort_flag = 1;
-    __threadfence_block();
-    return false;
-}
-
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -175,6 +158,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + SM::kBars + BAR_COUNT * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::kBars + BAR_COUNT * 8 + 8);
     auto bar = [&](uint32_t idx) { return bars + idx * 8u; };
+    // Every barrier wait is bounded by the launch's cycle limit.
+    auto wait_bar = [&](uint32_t b_, uint32_t parity, volatile int *flag, int32_t *status, int code) {
+        return ptx::mbar_wait_bounded(b_, parity, flag, status, code, a.wait_cycles, (int)PA_ERR_TIMEOUT);
+    };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -789,46 +776,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
 // ---------------------------------------------------------------------------------- host side
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
-                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
-                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static pa_status get_encode_fn(EncodeTiledFn *out)
-{
-    static EncodeTiledFn cached = nullptr;
-    if (!cached) {
-        void *fn = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        PA_CUDA_OK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
-        if (qres != cudaDriverEntryPointSuccess || !fn)
-            return fail(PA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
-        cached = reinterpret_cast<EncodeTiledFn>(fn);
-    }
-    *out = cached;
-    return PA_OK;
-}
-
-// Tensor map over a bf16 [batch, seq, head, D] tensor with dimensions ordered
-// (feature, token, head, batch) so that a box of `box_heads` heads x 64 tokens x 64 features
-// lands in shared memory as rows head * 64 + token of 128 bytes each (128-byte swizzle).
-static pa_status make_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int D, int64_t N,
-                          int heads, int batch, const pa_strides &s, int box_heads, const char *what)
-{
-    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)heads, (cuuint64_t)batch};
-    const cuuint64_t strides[3] = {(cuuint64_t)s.seq * 2, (cuuint64_t)s.head * 2,
-                                   (cuuint64_t)(s.batch > 0 ? s.batch : s.seq * N) * 2};
-    const cuuint32_t box[4] = {64, 64, (cuuint32_t)box_heads, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims,
-                           strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS)
-        return fail(PA_ERR_CUDA, "cuTensorMapEncodeTiled failed for %s (CUresult %d)", what, (int)r);
-    return PA_OK;
-}
-
 static pa_status check_strides(const pa_strides &s, int D, const char *what)
 {
     if (s.seq < D || s.head < D || s.batch < 0)
@@ -862,6 +809,9 @@ static pa_status check_prefill(const pa_prefill_params *p)
 
 constexpr size_t kPrefillWorkspace = 256;
 
+// Limit of the kernel's barrier waits in clock cycles (0: the default); set by pa_set_wait_limit_cycles.
+static std::atomic<long long> g_wait_cycles{0};
+
 // Optional check of a caller's CSR (PA_VALIDATE=1): one thread per row.  The first violation
 // found is recorded as (kind, row) in check[0..1]: 1 row_ptr does not start at 0 / end at nnz,
 // 2 row extent negative or beyond nnz, 3 block index outside [0, row], 4 indices not ascending.
@@ -888,6 +838,11 @@ __global__ void validate_csr_kernel(const int32_t *row_ptr, const int32_t *col_i
 
 }  // namespace pa
 
+extern "C" void pa_set_wait_limit_cycles(int64_t cycles)
+{
+    pa::g_wait_cycles.store(cycles > 0 ? (long long)cycles : 0, std::memory_order_relaxed);
+}
+
 extern "C" size_t pa_prefill_workspace_bytes(const pa_prefill_params *p)
 {
     (void)p;
@@ -913,17 +868,22 @@ extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const
     if (!workspace || workspace_bytes < kPrefillWorkspace)
         return fail(PA_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", kPrefillWorkspace, workspace_bytes);
     if (!aligned16(workspace)) return fail(PA_ERR_ALIGNMENT, "workspace must be 16-byte aligned");
-    if (pa_status s = require_sm100()) return s;
+    DeviceInfo dev;
+    if (pa_status s = current_sm100_device(&dev)) return s;
 
-    EncodeTiledFn enc = nullptr;
-    if (pa_status s = get_encode_fn(&enc)) return s;
+    // Tensor maps (cached per buffer and shape): a Q box holds the two heads of a tile, K, V and O
+    // boxes one head.
     CUtensorMap tmQ, tmK, tmV, tmO;
     const int D = p->head_dim;
-    if (pa_status s = make_map(enc, &tmQ, q, D, p->seq_len, p->n_q_heads, p->batch, p->q, 2, "q")) return s;
-    if (pa_status s = make_map(enc, &tmK, k, D, p->seq_len, p->n_kv_heads, p->batch, p->k, 1, "k")) return s;
-    if (pa_status s = make_map(enc, &tmV, v, D, p->seq_len, p->n_kv_heads, p->batch, p->v, 1, "v")) return s;
+    auto map_of = [&](const void *base, int heads, const pa_strides &st, int box_heads, const char *what, CUtensorMap *m) {
+        const TensorMapKey key = {base, p->seq_len, st.seq, st.head, st.batch, dev.device, D, heads, p->batch, box_heads, kBlk};
+        return get_tensor_map(key, what, m);
+    };
+    if (pa_status s = map_of(q, p->n_q_heads, p->q, 2, "q", &tmQ)) return s;
+    if (pa_status s = map_of(k, p->n_kv_heads, p->k, 1, "k", &tmK)) return s;
+    if (pa_status s = map_of(v, p->n_kv_heads, p->v, 1, "v", &tmV)) return s;
     if (p->o_dtype == PA_BF16) {
-        if (pa_status s = make_map(enc, &tmO, o, D, p->seq_len, p->n_q_heads, p->batch, p->o, 1, "o")) return s;
+        if (pa_status s = map_of(o, p->n_q_heads, p->o, 1, "o", &tmO)) return s;
     } else {
         tmO = tmQ;  // fp32 output is written from registers; the map is not used
     }
@@ -948,18 +908,16 @@ extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const
     const float scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.0f / sqrtf((float)D);
     a.scale_log2 = scale * 1.4426950408889634f;
 
-    int dev = 0, sms = 0;
-    PA_CUDA_OK(cudaGetDevice(&dev));
-    PA_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    const unsigned grid = (unsigned)(a.n_units < sms ? a.n_units : sms);
+    const long long wait_cycles = g_wait_cycles.load(std::memory_order_relaxed);
+    a.wait_cycles = wait_cycles > 0 ? wait_cycles : kWaitCycles;
+    const unsigned grid = (unsigned)(a.n_units < dev.sms ? a.n_units : dev.sms);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     PA_CUDA_OK(cudaMemsetAsync(workspace, 0, kPrefillWorkspace, st));
     {
         // PA_VALIDATE=1: check the CSR on the device before the attention kernel is enqueued.  This
         // synchronises the stream (so not during stream capture) and is meant for bring-up: a CSR
         // whose extents point outside col_idx would otherwise be read out of bounds.
-        const char *e = getenv("PA_VALIDATE");
-        if (e && e[0] == '1') {
+        if (env_switches().validate) {
             int32_t *check = static_cast<int32_t *>(workspace) + 32;
             validate_csr_kernel<<<(unsigned)((nqb + 127) / 128), 128, 0, st>>>(row_ptr, col_idx, (int32_t)nqb, nnz, check);
             PA_CUDA_OK(cudaGetLastError());
@@ -972,15 +930,20 @@ extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const
                 return fail(PA_ERR_LAYOUT, "CSR check: %s (row %d)", what[found[0]], (int)found[1]);
         }
     }
-    if (D == 128) {
-        PA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)SmemMap<128>::kAlloc));
-        prefill_kernel<128><<<grid, kThreads, SmemMap<128>::kAlloc, st>>>(tmQ, tmK, tmV, tmO, a);
-    } else {
-        PA_CUDA_OK(cudaFuncSetAttribute(prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)SmemMap<64>::kAlloc));
-        prefill_kernel<64><<<grid, kThreads, SmemMap<64>::kAlloc, st>>>(tmQ, tmK, tmV, tmO, a);
+    if (device_once_begin(dev.device, ONCE_PREFILL_ATTR)) {
+        const cudaError_t e1 = cudaFuncSetAttribute(prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    (int)SmemMap<128>::kAlloc);
+        const cudaError_t e2 = cudaFuncSetAttribute(prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    (int)SmemMap<64>::kAlloc);
+        if (e1 != cudaSuccess || e2 != cudaSuccess) {
+            device_once_reset(dev.device, ONCE_PREFILL_ATTR);
+            return fail(PA_ERR_CUDA, "cudaFuncSetAttribute failed: %s", cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
+        }
     }
+    if (D == 128)
+        prefill_kernel<128><<<grid, kThreads, SmemMap<128>::kAlloc, st>>>(tmQ, tmK, tmV, tmO, a);
+    else
+        prefill_kernel<64><<<grid, kThreads, SmemMap<64>::kAlloc, st>>>(tmQ, tmK, tmV, tmO, a);
     PA_CUDA_OK(cudaGetLastError());
     return PA_OK;
 }

@@ -62,6 +62,29 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// Bounded mbarrier wait shared by the kernels.  Spins on try_wait for at most `limit` clock
+// cycles.  Returns false after a timeout, which it records once in status[0] (error code) and
+// status[1] (an id naming the wait), or once another thread of the CTA has raised the abort flag;
+// a timeout raises the flag, so that every role of the CTA leaves its loop and the CTA ends.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                                  int32_t *status, int code, long long limit, int timeout_status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t it = 0;
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++it & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > limit) break;
+        }
+    }
+    if (atomicCAS(status, 0, timeout_status) == 0) status[1] = code;
+    *abort_flag = 1;
+    __threadfence_block();
+    return false;
+}
+
 // ---------------------------------------------------------------- TMA (no multicast anywhere)
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *m)
 {
@@ -153,45 +176,12 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         : "memory");
 }
 
-// Waits for the tensor-memory loads issued so far; the registers they fill are passed through so
-// that no use of them can be scheduled before the wait.
-__device__ __forceinline__ void tmem_wait_ld_into(uint32_t (&r)[64])
-{
-    asm volatile(
-        "tcgen05.wait::ld.sync.aligned;\n"
-        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
-          "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]),
-          "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]),
-          "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-        :
-        : "memory");
-    asm volatile(
-        ""
-        : "+r"(r[32]), "+r"(r[33]), "+r"(r[34]), "+r"(r[35]), "+r"(r[36]), "+r"(r[37]), "+r"(r[38]),
-          "+r"(r[39]), "+r"(r[40]), "+r"(r[41]), "+r"(r[42]), "+r"(r[43]), "+r"(r[44]), "+r"(r[45]),
-          "+r"(r[46]), "+r"(r[47]), "+r"(r[48]), "+r"(r[49]), "+r"(r[50]), "+r"(r[51]), "+r"(r[52]),
-          "+r"(r[53]), "+r"(r[54]), "+r"(r[55]), "+r"(r[56]), "+r"(r[57]), "+r"(r[58]), "+r"(r[59]),
-          "+r"(r[60]), "+r"(r[61]), "+r"(r[62]), "+r"(r[63])
-        :
-        : "memory");
-}
-
 // ---------------------------------------------------------------- tcgen05 MMA
-// Shared-memory operand descriptor, 128-byte swizzle, tile base 1024-byte aligned.
+// Shared-memory operand descriptors (128-byte swizzle, tile base 1024-byte aligned) are built by
+// the kernels from their two 32-bit words:
 //   bits  0-13 start address >> 4      bits 16-29 leading byte offset >> 4
 //   bits 32-45 stride byte offset >> 4 bits 46-47 descriptor version (1 on sm_100)
 //   bits 61-63 swizzle mode (2 = 128 B)
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_bytes,
-                                                    uint32_t sbo_bytes)
-{
-    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
 
 // Instruction descriptor for kind::f16 with bf16 operands and fp32 accumulation.
 //   bits 4-5 D format (1 = f32), 7-9 A format (1 = bf16), 10-12 B format (1 = bf16),
@@ -202,19 +192,9 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N, int b_mn_maj
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// D[tmem] (+)= A[smem] * B[smem]; issued by one thread.
-__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
-                                        uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// Same with each descriptor given as its low and high 32-bit words (the high word of a tile's
-// descriptor is constant, so advancing along K is one 32-bit add on the low word).
+// D[tmem] (+)= A[smem] * B[smem]; issued by one thread.  Each descriptor is given as its low and
+// high 32-bit words (the high word of a tile's descriptor is constant, so advancing along K is
+// one 32-bit add on the low word).
 __device__ __forceinline__ void umma_ss_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
                                              uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
                                              uint32_t accumulate)
@@ -290,13 +270,6 @@ __device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi)
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
-__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b)
-{
-    uint32_t r;
-    asm("max.bf16x2 %0, %1, %2;\n" : "=r"(r) : "r"(a), "r"(b));
-    return r;
-}
-
 // Register reallocation between warpgroups (all four warps of a warpgroup execute it).
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc()
@@ -314,6 +287,25 @@ __device__ __forceinline__ float ex2(float x)
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
     return y;
+}
+
+// Four 8 x 8 matrices of 16-bit elements from shared memory (lanes 8 i .. 8 i + 7 give the row
+// addresses of matrix i); lane (g, t) = (lane / 4, lane % 4) receives elements 2t, 2t + 1 of row g
+// of each matrix, or of its transpose with the .trans form.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr)
+                 : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2,
+                                                  uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr)
+                 : "memory");
 }
 
 }  // namespace ptx

@@ -31,3 +31,19 @@ def oracle():
 
     _oracle.build()
     return _oracle
+
+
+@pytest.fixture
+def pa_env(monkeypatch):
+    """Sets PA_* environment switches for one test and makes the library re-read them (it reads
+    the environment once); the previous state comes back, and is re-read, afterwards."""
+    import paper_2503_03588_b200 as pa
+
+    def set_env(**kv):
+        for key, val in kv.items():
+            monkeypatch.setenv(key, val)
+        pa.pa_reload_environment()
+
+    yield set_env
+    monkeypatch.undo()
+    pa.pa_reload_environment()

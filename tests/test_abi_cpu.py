@@ -110,8 +110,9 @@ def test_argument_validation_happens_before_any_launch(pa, oracle):
     dgood = pa.pa_decode_params(2, 4, 2, 128, 64, 5, 1, 4096, 0.0, s, s, pa.PA_BF16)
     # one (o[128], m, l) slot per query head and chunk; chunks = the longest block list of any row
     rp_ref, _ = oracle.block_layout(4096, 64, 5, 1)
-    chunks = pa.pa_decode_workspace_bytes(dgood) // (2 * 4 * 130 * 4)
-    assert pa.pa_decode_workspace_bytes(dgood) == 2 * 4 * chunks * 130 * 4
+    # a 256-byte status block, then one (o[128], m, l) slot per query head and chunk
+    chunks = (pa.pa_decode_workspace_bytes(dgood) - 256) // (2 * 4 * 130 * 4)
+    assert pa.pa_decode_workspace_bytes(dgood) == 256 + 2 * 4 * chunks * 130 * 4
     assert chunks == int(np.diff(rp_ref).max()) == 9
     dbad = pa.pa_decode_params.from_buffer_copy(dgood); dbad.n_q_heads = 40
     assert pa.pa_decode_workspace_bytes(dbad) == 0
@@ -120,4 +121,20 @@ def test_argument_validation_happens_before_any_launch(pa, oracle):
     st = pa.lib.pa_decode(ctypes.byref(dgood), p, p, p, p, p, p, p, 16, null)
     assert pa.pa_status_string(st) == "PA_ERR_WORKSPACE"
     st = pa.lib.pa_decode_block_list(0, 64, 5, 1, p, p, 64, null)
+    assert pa.pa_status_string(st) == "PA_ERR_INVALID_ARG"
+    st = pa.lib.pa_decode_row_block_set(4096, 64, 40, 1, p, p, 64, null)   # more than 32 candidates
+    assert pa.pa_status_string(st) == "PA_ERR_SHAPE"
+    st = pa.lib.pa_decode_row_block_set(4096, 64, 5, 1, p, p, 8, null)     # capacity below one warp
+    assert pa.pa_status_string(st) == "PA_ERR_INVALID_ARG"
+
+    sp = pa.pa_strides(64 * 2 * 128, 2 * 128, 128)
+    pgood = pa.pa_paged_params(2, 4, 2, 128, 64, 5, 1, 100, 64, 0.0, sp, sp, pa.PA_BF16)
+    assert pa.pa_decode_paged_workspace_bytes(pgood) == pa.pa_decode_workspace_bytes(dgood)  # 64 blocks = 4096 tokens
+    pbad = pa.pa_paged_params.from_buffer_copy(pgood); pbad.n_pages = 0
+    assert pa.pa_decode_paged_workspace_bytes(pbad) == 0
+    st = pa.lib.pa_decode_paged(ctypes.byref(pgood), p, p, p, 0, p, p, p, p, 10**6, null)
+    assert pa.pa_status_string(st) == "PA_ERR_INVALID_ARG"                 # null block table
+    st = pa.lib.pa_kv_append(ctypes.byref(pgood), p, p, p, p, p, 0, null)
+    assert pa.pa_status_string(st) == "PA_ERR_INVALID_ARG"                 # null cache_lens
+    st = pa.lib.pa_decode_status(0, null, None)
     assert pa.pa_status_string(st) == "PA_ERR_INVALID_ARG"

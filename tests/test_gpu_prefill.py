@@ -214,10 +214,10 @@ def test_repeated_launches_agree_bit_for_bit(pa):
     assert torch.equal(o0, o1) and torch.equal(lse0, lse1)
 
 
-def test_csr_check_switch_rejects_malformed_layouts(pa, monkeypatch):
+def test_csr_check_switch_rejects_malformed_layouts(pa, pa_env):
     """PA_VALIDATE=1 makes pa_prefill check the caller's CSR on the device before any attention
     work: each kind of violation comes back as PA_ERR_LAYOUT, and a good layout still runs."""
-    monkeypatch.setenv("PA_VALIDATE", "1")
+    pa_env(PA_VALIDATE="1")
     N, Hq, Hkv, D = 1024, 4, 2, 64
     Q = si.bf16_randn((1, N, Hq, D), 51).cuda()
     K = si.bf16_randn((1, N, Hkv, D), 52).cuda()
