@@ -83,6 +83,28 @@ pa_status pa_build_layout(int64_t seq_len, int32_t block, int32_t window_blocks,
                           int32_t sink_blocks, int32_t *row_ptr, int32_t *col_idx,
                           int64_t col_capacity, void *stream);
 
+/* The sliding-window comparison pattern of Section 3.2 / Section 4.1 ("Baseline": a local window
+ * plus initial sink tokens; the paper's setting is a 9-block window and 1 sink block): Algorithm 1
+ * without its power-of-two term, i.e. key block j is listed for query block i exactly when j <= i
+ * and ( i - j < window_blocks  or  j < sink_blocks ).  window_blocks >= 1 is required so that the
+ * diagonal block is listed (PA_ERR_INVALID_ARG otherwise); everything else as pa_layout_size /
+ * pa_build_layout.  The CSR runs through pa_prefill like any other causal layout. */
+pa_status pa_window_layout_size(int64_t seq_len, int32_t block, int32_t window_blocks,
+                                int32_t sink_blocks, int32_t *n_qblocks, int64_t *nnz);
+pa_status pa_build_window_layout(int64_t seq_len, int32_t block, int32_t window_blocks,
+                                 int32_t sink_blocks, int32_t *row_ptr, int32_t *col_idx,
+                                 int64_t col_capacity, void *stream);
+
+/* Receptive field of a layout seen as a directed graph over blocks (Section 3.1; Appendix A):
+ * counts[k-1] = |B_k|, the number of blocks that block `start` reaches within k steps along the
+ * edges block -> listed key block, itself included, for k = 1 .. max_steps.  Appendix A's
+ * theoretical accuracy is |B_k| / n_blocks with start = the last block (10/128 for the sliding
+ * window of its worked example).  Host only: row_ptr [n_blocks + 1], col_idx and counts
+ * [max_steps] are HOST pointers; nothing is launched.  Errors: PA_ERR_INVALID_ARG, PA_ERR_LAYOUT
+ * (an index outside [0, n_blocks) or a negative row extent). */
+pa_status pa_reach_counts(const int32_t *row_ptr, const int32_t *col_idx, int32_t n_blocks,
+                          int32_t start, int32_t max_steps, int64_t *counts);
+
 /* Tile layouts: the same mask listed at the granularity of the attention kernel.
  *
  * The paper's efficiency runs use 256-token blocks (Section 4.1, "Implementation"), the kernels
@@ -115,9 +137,10 @@ pa_status pa_build_tile_layout(int64_t seq_len, int32_t block, int32_t window_bl
  *   kv <= q inside the diagonal block (Algorithm 1's causal term), kv < seq_len;
  *   LSE[b,h,q] = ln sum_kv exp(s_kv);   O[b,q,h,:] = sum_kv exp(s_kv - LSE) V[b,kv,hk,:].
  *
- * The kernel accepts ANY causal CSR whose rows are ascending, end with the diagonal block
- * (col == row) and hold only cols <= row: the PowerAttention layout, dense causal, sliding
- * window.  It applies token-level causality to the diagonal pair and the seq_len bound itself.
+ * The kernel accepts ANY causal CSR whose rows are ascending and hold only cols <= row: the
+ * PowerAttention layout, dense causal, sliding window.  It applies token-level causality to the
+ * diagonal pair (col == row, which if listed is the row's last entry) and the seq_len bound
+ * itself.  A row may be empty: its query tokens get O = 0 and LSE = -inf.
  * Arithmetic: bf16 operands, fp32 accumulation (tensor cores), fp32 softmax; O rounded to
  * bf16 or kept fp32; LSE fp32.
  * ------------------------------------------------------------------------------------------ */
@@ -146,7 +169,7 @@ size_t pa_prefill_workspace_bytes(const pa_prefill_params *p);
  * o: device, o_dtype, strides p->o.  lse: device fp32 [batch, n_q_heads, seq_len] contiguous.
  * workspace: device, >= pa_prefill_workspace_bytes(p); cleared by the call itself.
  * Enqueues one memset and one kernel.  Errors: PA_ERR_INVALID_ARG, PA_ERR_SHAPE,
- * PA_ERR_ALIGNMENT, PA_ERR_LAYOUT (nnz < n_qblocks), PA_ERR_WORKSPACE, PA_ERR_UNSUPPORTED,
+ * PA_ERR_ALIGNMENT, PA_ERR_LAYOUT (nnz outside [0, 2^31)), PA_ERR_WORKSPACE, PA_ERR_UNSUPPORTED,
  * PA_ERR_CUDA.  Outputs are undefined after a failure.  The CSR is trusted: extents that point
  * outside col_idx would be read out of bounds.  With PA_VALIDATE=1 in the environment (see
  * pa_reload_environment) the call
@@ -157,6 +180,22 @@ size_t pa_prefill_workspace_bytes(const pa_prefill_params *p);
 pa_status pa_prefill(const pa_prefill_params *p, const void *q, const void *k, const void *v,
                      const int32_t *row_ptr, const int32_t *col_idx, int64_t nnz, void *o,
                      float *lse, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Variable-length batch: the sequences are packed one after the other along the token axis
+ * (Algorithm 1's mask takes no batch argument: every sequence uses the same layout, cut off at
+ * its own length).  q [total_tokens, n_q_heads, head_dim], k, v [total_tokens, n_kv_heads,
+ * head_dim] by the .seq and .head strides of p (the .batch strides are ignored); cu_seqlens:
+ * device int32 [p->batch + 1], ascending, cu_seqlens[0] = 0, cu_seqlens[batch] = total_tokens:
+ * sequence b owns tokens [cu_seqlens[b], cu_seqlens[b+1]).  p->seq_len is the length of the longest
+ * sequence (an upper bound is fine; query tokens of a sequence beyond it get no output), and the
+ * CSR has at least ceil(p->seq_len / block) rows: row i serves query block i of every sequence.
+ * o as q (n_q_heads heads); lse: device fp32 [n_q_heads, total_tokens].  A sequence's last block is
+ * written row by row so that the next sequence's rows stay untouched; empty sequences are allowed.
+ * Everything else as pa_prefill. */
+pa_status pa_prefill_varlen(const pa_prefill_params *p, const void *q, const void *k, const void *v,
+                            const int32_t *cu_seqlens, int64_t total_tokens, const int32_t *row_ptr,
+                            const int32_t *col_idx, int64_t nnz, void *o, float *lse, void *workspace,
+                            size_t workspace_bytes, void *stream);
 
 /* Synchronises `stream` and reads back the status block a pa_prefill call left in `workspace`.
  * Returns PA_OK, PA_ERR_TIMEOUT (a bounded barrier wait inside the kernel ran out; *detail, a

@@ -21,8 +21,9 @@ STATUS_NAMES = ["PA_OK", "PA_ERR_INVALID_ARG", "PA_ERR_SHAPE", "PA_ERR_ALIGNMENT
                 "PA_ERR_WORKSPACE", "PA_ERR_UNSUPPORTED", "PA_ERR_CUDA", "PA_ERR_TIMEOUT"]
 
 EXPORTS = ["pa_status_string", "pa_last_error_message", "pa_version", "pa_reload_environment",
-           "pa_set_wait_limit_cycles", "pa_layout_size", "pa_build_layout", "pa_tile_layout_size",
-           "pa_build_tile_layout", "pa_prefill_workspace_bytes", "pa_prefill", "pa_prefill_status",
+           "pa_set_wait_limit_cycles", "pa_layout_size", "pa_build_layout", "pa_window_layout_size",
+           "pa_build_window_layout", "pa_reach_counts", "pa_tile_layout_size",
+           "pa_build_tile_layout", "pa_prefill_workspace_bytes", "pa_prefill", "pa_prefill_varlen", "pa_prefill_status",
            "pa_decode_workspace_bytes", "pa_decode", "pa_decode_status", "pa_decode_block_list",
            "pa_decode_row_block_set", "pa_decode_paged_workspace_bytes", "pa_decode_paged", "pa_kv_append",
            "pa_decode_static"]
@@ -77,6 +78,12 @@ def _load() -> ctypes.CDLL:
     lib.pa_layout_size.argtypes = [i64, i32, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i64)]
     lib.pa_build_layout.restype = ctypes.c_int
     lib.pa_build_layout.argtypes = [i64, i32, i32, i32, vp, vp, i64, vp]
+    lib.pa_window_layout_size.restype = ctypes.c_int
+    lib.pa_window_layout_size.argtypes = [i64, i32, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i64)]
+    lib.pa_build_window_layout.restype = ctypes.c_int
+    lib.pa_build_window_layout.argtypes = [i64, i32, i32, i32, vp, vp, i64, vp]
+    lib.pa_reach_counts.restype = ctypes.c_int
+    lib.pa_reach_counts.argtypes = [vp, vp, i32, i32, i32, vp]
     lib.pa_tile_layout_size.restype = ctypes.c_int
     lib.pa_tile_layout_size.argtypes = [i64, i32, i32, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i64)]
     lib.pa_build_tile_layout.restype = ctypes.c_int
@@ -86,6 +93,9 @@ def _load() -> ctypes.CDLL:
     lib.pa_prefill.restype = ctypes.c_int
     lib.pa_prefill.argtypes = [ctypes.POINTER(pa_prefill_params), vp, vp, vp, vp, vp, i64, vp, vp, vp,
                                ctypes.c_size_t, vp]
+    lib.pa_prefill_varlen.restype = ctypes.c_int
+    lib.pa_prefill_varlen.argtypes = [ctypes.POINTER(pa_prefill_params), vp, vp, vp, vp, i64, vp, vp, i64, vp, vp, vp,
+                                      ctypes.c_size_t, vp]
     lib.pa_prefill_status.restype = ctypes.c_int
     lib.pa_prefill_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     lib.pa_decode_workspace_bytes.restype = ctypes.c_size_t
@@ -173,6 +183,38 @@ def pa_build_layout(seq_len: int, block: int, window_blocks: int, sink_blocks: i
     return row_ptr, col_idx
 
 
+def pa_window_layout_size(seq_len: int, block: int, window_blocks: int, sink_blocks: int) -> Tuple[int, int]:
+    nqb, nnz = ctypes.c_int32(0), ctypes.c_int64(0)
+    _check(lib.pa_window_layout_size(seq_len, block, window_blocks, sink_blocks, ctypes.byref(nqb), ctypes.byref(nnz)))
+    return int(nqb.value), int(nnz.value)
+
+
+def pa_build_window_layout(seq_len: int, block: int, window_blocks: int, sink_blocks: int,
+                           row_ptr: Optional[torch.Tensor] = None, col_idx: Optional[torch.Tensor] = None,
+                           device="cuda"):
+    """Sliding-window layout (window + sink blocks, no power-of-two term) as int32 device tensors."""
+    nqb, nnz = pa_window_layout_size(seq_len, block, window_blocks, sink_blocks)
+    if row_ptr is None:
+        row_ptr = torch.empty(nqb + 1, dtype=torch.int32, device=device)
+    if col_idx is None:
+        col_idx = torch.empty(nnz, dtype=torch.int32, device=device)
+    _check(lib.pa_build_window_layout(seq_len, block, window_blocks, sink_blocks, _ptr(row_ptr), _ptr(col_idx),
+                                      col_idx.numel(), _stream()))
+    return row_ptr, col_idx
+
+
+def pa_reach_counts(row_ptr, col_idx, start: int, max_steps: int):
+    """|B_k| for k = 1..max_steps from a HOST CSR (numpy int32 arrays or CPU tensors)."""
+    import numpy as np
+
+    rp = np.ascontiguousarray(np.asarray(row_ptr, dtype=np.int32))
+    ci = np.ascontiguousarray(np.asarray(col_idx, dtype=np.int32))
+    out = np.zeros(max_steps, dtype=np.int64)
+    _check(lib.pa_reach_counts(rp.ctypes.data_as(ctypes.c_void_p), ci.ctypes.data_as(ctypes.c_void_p), len(rp) - 1,
+                               start, max_steps, out.ctypes.data_as(ctypes.c_void_p)))
+    return out.tolist()
+
+
 def pa_tile_layout_size(seq_len: int, block: int, window_blocks: int, sink_blocks: int,
                         tile: int = 64) -> Tuple[int, int]:
     nqt, nnz = ctypes.c_int32(0), ctypes.c_int64(0)
@@ -223,6 +265,27 @@ def pa_prefill(q, k, v, row_ptr, col_idx, o=None, lse=None, workspace=None, bloc
     _check(lib.pa_prefill(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(row_ptr), _ptr(col_idx),
                           col_idx.numel() if nnz is None else nnz, _ptr(o), _ptr(lse), _ptr(workspace),
                           workspace.numel(), _stream()))
+    return o, lse, workspace
+
+
+def pa_prefill_varlen(q, k, v, cu_seqlens, max_seq_len: int, row_ptr, col_idx, o=None, lse=None, workspace=None,
+                      block: int = 64, softmax_scale: float = 0.0, o_dtype=torch.bfloat16):
+    """Packed sequences: q [total, Hq, D], k, v [total, Hkv, D] bf16, cu_seqlens int32 [batch + 1] on the
+    device.  Returns (o [total, Hq, D], lse [Hq, total], workspace)."""
+    total, hq, d = q.shape
+    assert q.stride(2) == 1 and k.stride(2) == 1 and v.stride(2) == 1 and cu_seqlens.dtype == torch.int32
+    if o is None:
+        o = torch.empty((total, hq, d), dtype=o_dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty((hq, total), dtype=torch.float32, device=q.device)
+    st = lambda t: pa_strides(0, t.stride(0), t.stride(1))
+    params = pa_prefill_params(cu_seqlens.numel() - 1, hq, k.shape[1], d, max_seq_len, block, float(softmax_scale),
+                               st(q), st(k), st(v), st(o), PA_F32 if o.dtype == torch.float32 else PA_BF16)
+    if workspace is None:
+        workspace = torch.empty(max(pa_prefill_workspace_bytes(params), 16), dtype=torch.uint8, device=q.device)
+    _check(lib.pa_prefill_varlen(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(cu_seqlens), total,
+                                 _ptr(row_ptr), _ptr(col_idx), col_idx.numel(), _ptr(o), _ptr(lse), _ptr(workspace),
+                                 workspace.numel(), _stream()))
     return o, lse, workspace
 
 

@@ -1,14 +1,16 @@
 // pa_layout_size / pa_build_layout: the block-sparse CSR of Algorithm 1 (Section 3.3).
+#include <vector>
+
 #include "common.cuh"
 #include "layout_rule.cuh"
 
 namespace pa {
 
-__global__ void layout_count_kernel(int32_t nqb, int32_t W, int32_t S, int32_t *row_ptr)
+__global__ void layout_count_kernel(int32_t nqb, int32_t W, int32_t S, int32_t *row_ptr, bool power)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0) row_ptr[0] = 0;
-    if (i < nqb) row_ptr[i + 1] = row_length(i, W, S);
+    if (i < nqb) row_ptr[i + 1] = row_length(i, W, S, power);
 }
 
 // In-place inclusive scan of row_ptr[1 .. nqb] by one block, tile by tile with a running carry.
@@ -52,11 +54,11 @@ struct StoreCols {
 };
 
 __global__ void layout_fill_kernel(int32_t nqb, int32_t W, int32_t S, const int32_t *row_ptr,
-                                   int32_t *col_idx)
+                                   int32_t *col_idx, bool power)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= nqb) return;
-    for_each_key_block(i, W, S, StoreCols{col_idx + row_ptr[i]});
+    for_each_key_block(i, W, S, StoreCols{col_idx + row_ptr[i]}, power);
 }
 
 // Tile layouts: the mask's block holds r tiles of the attention kernel.  Algorithm 1's window,
@@ -107,42 +109,106 @@ static pa_status check_layout_args(int64_t seq_len, int32_t block, int32_t W, in
 
 }  // namespace pa
 
-extern "C" pa_status pa_layout_size(int64_t seq_len, int32_t block, int32_t window_blocks,
-                                    int32_t sink_blocks, int32_t *n_qblocks, int64_t *nnz)
+namespace pa {
+
+static pa_status layout_size(int64_t seq_len, int32_t block, int32_t W, int32_t S, bool power, int32_t *n_qblocks,
+                             int64_t *nnz)
 {
-    using namespace pa;
-    clear_error();
-    if (pa_status s = check_layout_args(seq_len, block, window_blocks, sink_blocks)) return s;
+    if (pa_status s = check_layout_args(seq_len, block, W, S)) return s;
+    if (!power && W < 1)
+        return fail(PA_ERR_INVALID_ARG, "a sliding-window layout needs window_blocks >= 1 (the diagonal block)");
     if (!n_qblocks || !nnz) return fail(PA_ERR_INVALID_ARG, "n_qblocks and nnz must be non-null");
     const int64_t nqb = (seq_len + block - 1) / block;
     if (nqb >= INT32_MAX) return fail(PA_ERR_SHAPE, "n_qblocks %lld does not fit in int32", (long long)nqb);
     int64_t total = 0;
-    for (int64_t i = 0; i < nqb; ++i) total += row_length(i, window_blocks, sink_blocks);
+    for (int64_t i = 0; i < nqb; ++i) total += row_length(i, W, S, power);
     if (total > INT32_MAX) return fail(PA_ERR_SHAPE, "nnz %lld does not fit in int32", (long long)total);
     *n_qblocks = (int32_t)nqb;
     *nnz = total;
     return PA_OK;
 }
 
-extern "C" pa_status pa_build_layout(int64_t seq_len, int32_t block, int32_t window_blocks,
-                                     int32_t sink_blocks, int32_t *row_ptr, int32_t *col_idx,
-                                     int64_t col_capacity, void *stream)
+static pa_status build_layout(int64_t seq_len, int32_t block, int32_t W, int32_t S, bool power, int32_t *row_ptr,
+                              int32_t *col_idx, int64_t col_capacity, void *stream)
 {
-    using namespace pa;
-    clear_error();
     int32_t nqb = 0;
     int64_t nnz = 0;
-    if (pa_status s = pa_layout_size(seq_len, block, window_blocks, sink_blocks, &nqb, &nnz)) return s;
+    if (pa_status s = layout_size(seq_len, block, W, S, power, &nqb, &nnz)) return s;
     if (!row_ptr || !col_idx) return fail(PA_ERR_INVALID_ARG, "row_ptr and col_idx must be non-null");
     if (col_capacity < nnz)
         return fail(PA_ERR_LAYOUT, "col_capacity %lld < nnz %lld", (long long)col_capacity, (long long)nnz);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int threads = 256;
     const unsigned blocks = (unsigned)((nqb + threads - 1) / threads);
-    layout_count_kernel<<<blocks, threads, 0, st>>>(nqb, window_blocks, sink_blocks, row_ptr);
+    layout_count_kernel<<<blocks, threads, 0, st>>>(nqb, W, S, row_ptr, power);
     layout_scan_kernel<<<1, 1024, 0, st>>>(nqb, row_ptr);
-    layout_fill_kernel<<<blocks, threads, 0, st>>>(nqb, window_blocks, sink_blocks, row_ptr, col_idx);
+    layout_fill_kernel<<<blocks, threads, 0, st>>>(nqb, W, S, row_ptr, col_idx, power);
     PA_CUDA_OK(cudaGetLastError());
+    return PA_OK;
+}
+
+}  // namespace pa
+
+extern "C" pa_status pa_layout_size(int64_t seq_len, int32_t block, int32_t window_blocks,
+                                    int32_t sink_blocks, int32_t *n_qblocks, int64_t *nnz)
+{
+    pa::clear_error();
+    return pa::layout_size(seq_len, block, window_blocks, sink_blocks, true, n_qblocks, nnz);
+}
+
+extern "C" pa_status pa_build_layout(int64_t seq_len, int32_t block, int32_t window_blocks,
+                                     int32_t sink_blocks, int32_t *row_ptr, int32_t *col_idx,
+                                     int64_t col_capacity, void *stream)
+{
+    pa::clear_error();
+    return pa::build_layout(seq_len, block, window_blocks, sink_blocks, true, row_ptr, col_idx, col_capacity, stream);
+}
+
+extern "C" pa_status pa_window_layout_size(int64_t seq_len, int32_t block, int32_t window_blocks,
+                                           int32_t sink_blocks, int32_t *n_qblocks, int64_t *nnz)
+{
+    pa::clear_error();
+    return pa::layout_size(seq_len, block, window_blocks, sink_blocks, false, n_qblocks, nnz);
+}
+
+extern "C" pa_status pa_build_window_layout(int64_t seq_len, int32_t block, int32_t window_blocks,
+                                            int32_t sink_blocks, int32_t *row_ptr, int32_t *col_idx,
+                                            int64_t col_capacity, void *stream)
+{
+    pa::clear_error();
+    return pa::build_layout(seq_len, block, window_blocks, sink_blocks, false, row_ptr, col_idx, col_capacity, stream);
+}
+
+extern "C" pa_status pa_reach_counts(const int32_t *row_ptr, const int32_t *col_idx, int32_t n_blocks,
+                                     int32_t start, int32_t max_steps, int64_t *counts)
+{
+    using namespace pa;
+    clear_error();
+    if (!row_ptr || !col_idx || !counts) return fail(PA_ERR_INVALID_ARG, "row_ptr, col_idx and counts must be non-null");
+    if (n_blocks < 1 || start < 0 || start >= n_blocks || max_steps < 1)
+        return fail(PA_ERR_INVALID_ARG, "need n_blocks >= 1, 0 <= start < n_blocks, max_steps >= 1");
+    // Breadth-first search from `start` over the edges block -> listed key block, level by level.
+    std::vector<int32_t> depth((size_t)n_blocks, -1), frontier{start}, next;
+    depth[(size_t)start] = 0;
+    int64_t reached = 1;
+    for (int32_t k = 1; k <= max_steps; ++k) {
+        next.clear();
+        for (int32_t u : frontier) {
+            const int32_t lo = row_ptr[u], hi = row_ptr[u + 1];
+            if (lo < 0 || hi < lo) return fail(PA_ERR_LAYOUT, "row %d has a negative extent", u);
+            for (int32_t e = lo; e < hi; ++e) {
+                const int32_t v = col_idx[e];
+                if (v < 0 || v >= n_blocks) return fail(PA_ERR_LAYOUT, "row %d lists block %d outside [0, %d)", u, v, n_blocks);
+                if (depth[(size_t)v] < 0) {
+                    depth[(size_t)v] = k;
+                    next.push_back(v);
+                    ++reached;
+                }
+            }
+        }
+        counts[k - 1] = reached;
+        frontier.swap(next);
+    }
     return PA_OK;
 }
 

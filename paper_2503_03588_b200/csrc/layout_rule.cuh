@@ -14,15 +14,17 @@ namespace pa {
 // Calls emit(pos, j) for every listed key block j of query block i in ascending order and
 // returns the row length.  i >= 0, W >= 0, S >= 0.  Index is int64_t, or int32_t where the block
 // indices are known to fit (the decode kernel: a cheaper walk on its critical path).
+// `power` false drops the power-of-two run: the sliding-window pattern (local window plus sink
+// blocks, Section 3.2 / Section 4.1 "Baseline"), for which W >= 1 keeps the diagonal block listed.
 template <typename Index, typename Emit>
-__host__ __device__ inline int for_each_key_block_t(Index i, int32_t W, int32_t S, Emit emit)
+__host__ __device__ inline int for_each_key_block_t(Index i, int32_t W, int32_t S, Emit emit, bool power = true)
 {
     const Index w_eff = W > 1 ? (Index)W : (Index)1;
     const Index sink_end = (Index)S < i + 1 ? (Index)S : i + 1;  // sink run [0, sink_end)
     Index js = 0;                                                // sink cursor
     Index jw = i - w_eff + 1 > 0 ? i - w_eff + 1 : 0;            // window cursor .. i
     Index pw = 0;                                                // current power distance
-    if (i >= 1) {
+    if (power && i >= 1) {
         pw = 1;
         while (pw <= i / 2) pw *= 2;                             // largest 2^k <= i
     }
@@ -45,18 +47,18 @@ __host__ __device__ inline int for_each_key_block_t(Index i, int32_t W, int32_t 
 }
 
 template <typename Emit>
-__host__ __device__ inline int for_each_key_block(int64_t i, int32_t W, int32_t S, Emit emit)
+__host__ __device__ inline int for_each_key_block(int64_t i, int32_t W, int32_t S, Emit emit, bool power = true)
 {
-    return for_each_key_block_t<int64_t>(i, W, S, emit);
+    return for_each_key_block_t<int64_t>(i, W, S, emit, power);
 }
 
 struct NoEmit {
     __host__ __device__ void operator()(int, int64_t) const {}
 };
 
-__host__ __device__ inline int row_length(int64_t i, int32_t W, int32_t S)
+__host__ __device__ inline int row_length(int64_t i, int32_t W, int32_t S, bool power = true)
 {
-    return for_each_key_block(i, W, S, NoEmit());
+    return for_each_key_block(i, W, S, NoEmit(), power);
 }
 
 }  // namespace pa

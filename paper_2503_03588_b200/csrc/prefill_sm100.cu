@@ -57,11 +57,13 @@ constexpr long long kWaitCycles = 4000000000ll;  // default limit of a barrier w
 
 struct PrefillArgs {
     const int32_t *row_ptr, *col_idx;
+    const int32_t *cu_seqlens;  // variable-length batch: [batch + 1] token offsets of the packed sequences; else null
     void *o;
     float *lse;
     int32_t *status;  // [0] error code, [1] detail
     int64_t o_sb, o_ss, o_sh;
-    int64_t N, n_units;
+    int64_t lse_sb, lse_sh;  // LSE strides (batch, head); the token stride is 1
+    int64_t N, n_units;     // N: sequence length (variable-length batch: the longest one, which sizes the unit grid)
     int32_t nqb, batch, Hq, Hkv, G, nsub, o_is_f32;
     uint32_t inv_nsub, inv_Hkv, inv_nqb;  // floor(2^32 / d) of the three divisors of a unit index
     float scale_log2;
@@ -109,6 +111,10 @@ enum : uint32_t {
 
 struct Unit {
     int32_t b, hk, i, sub, rs, n;
+    // Where the unit's sequence lives: batch coordinate of the tensor maps, offset of its first
+    // token along their token axis, its length.  (Equal-length batch: b, 0, N.  Packed
+    // variable-length batch: 0, cu_seqlens[b], cu_seqlens[b + 1] - cu_seqlens[b].)
+    int32_t bt, tok0, len;
 };
 
 // u / d and u % d with inv = floor(2^32 / d) (2^32 - 1 for d = 1): the high product falls short of
@@ -140,6 +146,16 @@ __device__ __forceinline__ Unit decode_unit(const PrefillArgs &a, uint32_t u)
     r.i = a.nqb - 1 - (int32_t)rem;  // long rows first
     r.rs = __ldg(a.row_ptr + r.i);
     r.n = __ldg(a.row_ptr + r.i + 1) - r.rs;
+    if (a.cu_seqlens) {
+        r.bt = 0;
+        r.tok0 = __ldg(a.cu_seqlens + r.b);
+        r.len = __ldg(a.cu_seqlens + r.b + 1) - r.tok0;
+        if ((int64_t)r.i * kBlk >= r.len) r.n = 0;  // the sequence ends before this query block: nothing to do
+    } else {
+        r.bt = r.b;
+        r.tok0 = 0;
+        r.len = (int32_t)a.N;
+    }
     return r;
 }
 
@@ -243,8 +259,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 for (int s = 0; s < 2; ++s)
                     for (int dh = 0; dh < DH; ++dh)
                         ptx::tma_load_4d(smem_base + SM::kQ + qb * SM::kQBuf + s * SM::kQSlot + dh * SM::kQSub, &tmQ,
-                                         bar(BAR_Q_FULL + qb), dh * 64, w.i * kBlk,
-                                         w.hk * a.G + w.sub * 4 + 2 * s, w.b);
+                                         bar(BAR_Q_FULL + qb), dh * 64, w.tok0 + w.i * kBlk,
+                                         w.hk * a.G + w.sub * 4 + 2 * s, w.bt);
                 return true;
             };
             Unit w, wn;
@@ -264,7 +280,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     ptx::mbar_expect_tx(bar(BAR_K_FULL + ks), SM::kBlkTile);
                     for (int dh = 0; dh < DH; ++dh)
                         ptx::tma_load_4d(smem_base + SM::kK + ks * SM::kBlkTile + dh * SM::kBlkSub, &tmK,
-                                         bar(BAR_K_FULL + ks), dh * 64, j * kBlk, w.hk, w.b);
+                                         bar(BAR_K_FULL + ks), dh * 64, w.tok0 + j * kBlk, w.hk, w.bt);
                     if (kc >= (uint32_t)kVStages) {
                         ok = wait_bar(bar(BAR_V_EMPTY + vs), (kc / kVStages - 1) & 1, abort_flag, a.status, 3);
                         if (!ok) break;
@@ -272,7 +288,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     ptx::mbar_expect_tx(bar(BAR_V_FULL + vs), SM::kBlkTile);
                     for (int dh = 0; dh < DH; ++dh)
                         ptx::tma_load_4d(smem_base + SM::kV + vs * SM::kBlkTile + dh * SM::kBlkSub, &tmV,
-                                         bar(BAR_V_FULL + vs), dh * 64, j * kBlk, w.hk, w.b);
+                                         bar(BAR_V_FULL + vs), dh * 64, w.tok0 + j * kBlk, w.hk, w.bt);
                     j = jn;
                     // The next unit's Q goes where the unit before this one kept its Q and then
                     // staged its output, which leaves during this unit's first steps: the request
@@ -466,7 +482,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const int head_local = w.sub * 4 + 2 * s + (row >> 6);
             const int head = w.hk * a.G + head_local;
             const int64_t tok = (int64_t)w.i * kBlk + qrow;
-            const bool valid = head_local < a.G && tok < a.N;
+            const bool valid = head_local < a.G && tok < w.len;
             // Algorithm 1's causal term acts inside the diagonal pair (col == row) only; rows end
             // with that block.
             const bool last_is_diag = w.n > 0 && lastcol == w.i;
@@ -634,7 +650,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     reinterpret_cast<float *>(smem + SM::kStats)[s * 128 + row] = l;
                     __threadfence_block();
                     // LSE = ln sum exp(s) = (m + log2 l) ln 2.
-                    if (valid) a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = (m + log2f(l)) * 0.6931471805599453f;
+                    if (valid) a.lse[w.b * a.lse_sb + head * a.lse_sh + w.tok0 + tok] = (m + log2f(l)) * 0.6931471805599453f;
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(bar(BAR_ML_READY + s));
                 }
@@ -666,15 +682,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             for (int s = 0; s < 2; ++s) {
                 const int head_local = w.sub * 4 + 2 * s + (row >> 6);
                 const int head = w.hk * a.G + head_local;
-                const bool valid = head_local < a.G && tok < a.N;
-                const int64_t obase = w.b * a.o_sb + tok * a.o_ss + (int64_t)head * a.o_sh;
+                const bool valid = head_local < a.G && tok < w.len;
+                const int64_t obase = w.bt * a.o_sb + (w.tok0 + tok) * a.o_ss + (int64_t)head * a.o_sh;
                 if (w.n <= 0) {  // empty row: defined outputs, no barrier traffic
                     if (valid) {
                         for (int c = 0; c < D; ++c) {
                             if (a.o_is_f32) reinterpret_cast<float *>(a.o)[obase + c] = 0.f;
                             else reinterpret_cast<__nv_bfloat16 *>(a.o)[obase + c] = __float2bfloat16_rn(0.f);
                         }
-                        a.lse[((int64_t)w.b * a.Hq + head) * a.N + tok] = -INFINITY;
+                        a.lse[w.b * a.lse_sb + head * a.lse_sh + w.tok0 + tok] = -INFINITY;
                     }
                     continue;
                 }
@@ -710,6 +726,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     // Head 2 s + (row >> 6) of the unit: two boxes of 64 tokens x 128 bytes (one per
                     // 64-feature half); 16-byte chunk j of token t sits at chunk position j ^ (t & 7).
                     const uint32_t rbase = stage + (uint32_t)(2 * s + (row >> 6)) * SM::kOHead + (uint32_t)qrow * 128u;
+                    // A packed sequence's last block may reach into the next sequence's rows, which a
+                    // box store would overwrite: its rows are written one by one from the registers.
+                    const bool ragged = a.cu_seqlens != nullptr && (int64_t)(w.i + 1) * kBlk > w.len;
 #pragma unroll
                     for (int ch = 0; ch < D / 32; ++ch) {
                         uint32_t orr[32];
@@ -731,6 +750,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                                                         __uint_as_float(orr[8 * k + 2 * e + 1]) * inv);
                             const uint32_t dst = rbase + (uint32_t)(c >> 3) * 8192u + ((uint32_t)((c & 7) ^ (qrow & 7)) << 4);
                             ptx::st_shared_v4(dst, pk[0], pk[1], pk[2], pk[3]);
+                            if (ragged && valid)
+                                *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(a.o) + obase + 8 * c) =
+                                    make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         }
                     }
                     ptx::fence_proxy_async_smem();
@@ -745,10 +767,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     if (store_thread) {
                         for (int hh = 0; hh < 2; ++hh) {
                             const int hl = w.sub * 4 + 2 * s + hh;
-                            if (hl >= a.G) continue;  // the padding head of an odd group
+                            if (hl >= a.G || ragged) continue;  // the padding head of an odd group; rows already written
                             for (int dh = 0; dh < DH; ++dh)
                                 ptx::tma_store_4d(&tmO, stage + (uint32_t)(2 * s + hh) * SM::kOHead + (uint32_t)dh * 8192u,
-                                                  dh * 64, w.i * kBlk, w.hk * a.G + hl, w.b);
+                                                  dh * 64, w.tok0 + w.i * kBlk, w.hk * a.G + hl, w.bt);
                         }
                         ptx::bulk_commit_group();
                     }
@@ -849,22 +871,26 @@ extern "C" size_t pa_prefill_workspace_bytes(const pa_prefill_params *p)
     return pa::kPrefillWorkspace;
 }
 
-extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const void *k,
-                                const void *v, const int32_t *row_ptr, const int32_t *col_idx,
-                                int64_t nnz, void *o, float *lse, void *workspace,
+namespace pa {
+
+// The launch behind pa_prefill (cu_seqlens null) and pa_prefill_varlen (packed sequences:
+// p->seq_len is the longest one, tokens run over [0, total_tokens)).
+static pa_status launch_prefill(const pa_prefill_params *p, const void *q, const void *k, const void *v,
+                                const int32_t *cu_seqlens, int64_t total_tokens, const int32_t *row_ptr,
+                                const int32_t *col_idx, int64_t nnz, void *o, float *lse, void *workspace,
                                 size_t workspace_bytes, void *stream)
 {
-    using namespace pa;
-    clear_error();
     if (pa_status s = check_prefill(p)) return s;
+    const bool varlen = cu_seqlens != nullptr;
+    if (varlen && (total_tokens < 1 || total_tokens > ((int64_t)1 << 30)))
+        return fail(PA_ERR_INVALID_ARG, "total_tokens must be in [1, 2^30]");
     if (!q || !k || !v || !row_ptr || !col_idx || !o || !lse)
         return fail(PA_ERR_INVALID_ARG, "q, k, v, row_ptr, col_idx, o and lse must be non-null");
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o))
         return fail(PA_ERR_ALIGNMENT, "q, k, v and o must be 16-byte aligned");
     const int64_t nqb = (p->seq_len + kBlk - 1) / kBlk;
-    if (nnz < nqb)
-        return fail(PA_ERR_LAYOUT, "nnz %lld < n_qblocks %lld: every row lists its diagonal block",
-                    (long long)nnz, (long long)nqb);
+    if (nnz < 0 || nnz > (int64_t)INT32_MAX)
+        return fail(PA_ERR_LAYOUT, "nnz %lld is outside [0, 2^31)", (long long)nnz);
     if (!workspace || workspace_bytes < kPrefillWorkspace)
         return fail(PA_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", kPrefillWorkspace, workspace_bytes);
     if (!aligned16(workspace)) return fail(PA_ERR_ALIGNMENT, "workspace must be 16-byte aligned");
@@ -876,7 +902,9 @@ extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const
     CUtensorMap tmQ, tmK, tmV, tmO;
     const int D = p->head_dim;
     auto map_of = [&](const void *base, int heads, const pa_strides &st, int box_heads, const char *what, CUtensorMap *m) {
-        const TensorMapKey key = {base, p->seq_len, st.seq, st.head, st.batch, dev.device, D, heads, p->batch, box_heads, kBlk};
+        // (packed sequences: one "batch" entry of total_tokens tokens)
+        const TensorMapKey key = {base, varlen ? total_tokens : p->seq_len, st.seq, st.head, varlen ? 0 : st.batch, dev.device, D,
+                                  heads, varlen ? 1 : p->batch, box_heads, kBlk};
         return get_tensor_map(key, what, m);
     };
     if (pa_status s = map_of(q, p->n_q_heads, p->q, 2, "q", &tmQ)) return s;
@@ -891,10 +919,14 @@ extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const
     PrefillArgs a;
     a.row_ptr = row_ptr;
     a.col_idx = col_idx;
+    a.cu_seqlens = cu_seqlens;
     a.o = o;
     a.lse = lse;
     a.status = static_cast<int32_t *>(workspace);
     a.o_sb = p->o.batch; a.o_ss = p->o.seq; a.o_sh = p->o.head;
+    // LSE: [batch, Hq, seq_len], or [Hq, total_tokens] for packed sequences.
+    a.lse_sb = varlen ? 0 : (int64_t)p->n_q_heads * p->seq_len;
+    a.lse_sh = varlen ? total_tokens : p->seq_len;
     a.N = p->seq_len;
     a.nqb = (int32_t)nqb;
     a.batch = p->batch; a.Hq = p->n_q_heads; a.Hkv = p->n_kv_heads;
@@ -946,6 +978,28 @@ extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const
         prefill_kernel<64><<<grid, kThreads, SmemMap<64>::kAlloc, st>>>(tmQ, tmK, tmV, tmO, a);
     PA_CUDA_OK(cudaGetLastError());
     return PA_OK;
+}
+
+}  // namespace pa
+
+extern "C" pa_status pa_prefill(const pa_prefill_params *p, const void *q, const void *k,
+                                const void *v, const int32_t *row_ptr, const int32_t *col_idx,
+                                int64_t nnz, void *o, float *lse, void *workspace,
+                                size_t workspace_bytes, void *stream)
+{
+    pa::clear_error();
+    return pa::launch_prefill(p, q, k, v, nullptr, 0, row_ptr, col_idx, nnz, o, lse, workspace, workspace_bytes, stream);
+}
+
+extern "C" pa_status pa_prefill_varlen(const pa_prefill_params *p, const void *q, const void *k, const void *v,
+                                       const int32_t *cu_seqlens, int64_t total_tokens, const int32_t *row_ptr,
+                                       const int32_t *col_idx, int64_t nnz, void *o, float *lse, void *workspace,
+                                       size_t workspace_bytes, void *stream)
+{
+    pa::clear_error();
+    if (!cu_seqlens) return pa::fail(PA_ERR_INVALID_ARG, "cu_seqlens must be non-null");
+    return pa::launch_prefill(p, q, k, v, cu_seqlens, total_tokens, row_ptr, col_idx, nnz, o, lse, workspace,
+                              workspace_bytes, stream);
 }
 
 extern "C" pa_status pa_prefill_status(const void *workspace, void *stream, int32_t *detail)

@@ -104,7 +104,7 @@ def test_argument_validation_happens_before_any_launch(pa, oracle):
     assert prefill_status(bad) == "PA_ERR_ALIGNMENT"
     assert prefill_status(good, q=0) == "PA_ERR_INVALID_ARG"
     assert prefill_status(good, q=p + 4) == "PA_ERR_ALIGNMENT"
-    assert prefill_status(good, nnz=3) == "PA_ERR_LAYOUT"
+    assert prefill_status(good, nnz=-1) == "PA_ERR_LAYOUT"
     assert prefill_status(good, ws_bytes=8) == "PA_ERR_WORKSPACE"
 
     dgood = pa.pa_decode_params(2, 4, 2, 128, 64, 5, 1, 4096, 0.0, s, s, pa.PA_BF16)
@@ -138,3 +138,52 @@ def test_argument_validation_happens_before_any_launch(pa, oracle):
     assert pa.pa_status_string(st) == "PA_ERR_INVALID_ARG"                 # null cache_lens
     st = pa.lib.pa_decode_status(0, null, None)
     assert pa.pa_status_string(st) == "PA_ERR_INVALID_ARG"
+
+
+def test_window_layout_size_matches_oracle(pa, oracle):
+    """Sliding window (window + sink blocks, no power-of-two term), Section 4.1 "Baseline"."""
+    for N in (1, 64, 65, 2048, 4096 + 17, 32768):
+        for W in (1, 4, 9):
+            for S in (0, 1, 3):
+                nqb, nnz = pa.pa_window_layout_size(N, 64, W, S)
+                rp, ci = oracle.block_layout(N, 64, W, S, use_power=False)
+                assert nqb == len(rp) - 1 and nnz == int(rp[-1]) == len(ci), (N, W, S)
+    with pytest.raises(pa.PaError, match="PA_ERR_INVALID_ARG"):
+        pa.pa_window_layout_size(4096, 64, 0, 1)      # no window: the diagonal block would be missing
+
+
+def _read_golden(name):
+    out = {}
+    with open(os.path.join(ROOT, "tests", "golden", name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                key, *vals = line.split()
+                out[key] = [int(v) for v in vals]
+    return out
+
+
+def test_reach_counts_against_the_paper_and_the_oracle(pa, oracle):
+    """pa_reach_counts (host BFS over a CSR) on the layouts of the appendix's setting: |B_1| = 10 of
+    128 blocks for the 9 + 1 sliding window (Appendix A), the default pattern's 10-block budget and
+    full coverage within six steps (Section 4.1, Section 4.3), and the oracle's BFS everywhere."""
+    g = _read_golden("sliding_window_B1.txt")
+    n, W, S = g["n_blocks"][0], g["window_blocks"][0], g["sink_blocks"][0]
+    rp, ci = oracle.block_layout(n * 256, 256, W, S, use_power=False)
+    counts = pa.pa_reach_counts(rp, ci, n - 1, 20)
+    assert counts[0] == g["alpha1_numerator"][0] == len(g["B1"])
+    assert counts == oracle.reach_counts(oracle.block_adjacency(n, W, S, use_power=False), n - 1, 20)
+    d = _read_golden("power_attention_default.txt")
+    n, W, S = d["n_blocks"][0], d["window_blocks"][0], d["sink_blocks"][0]
+    rp, ci = oracle.block_layout(n * 256, 256, W, S)
+    counts = pa.pa_reach_counts(rp, ci, n - 1, 8)
+    assert counts[0] == d["last_row_blocks"][0]
+    assert counts[d["full_coverage_layers_at_most"][0] - 1] == n and counts[d["full_coverage_layers_at_most"][0] - 2] < n
+    assert counts == oracle.reach_counts(oracle.block_adjacency(n, W, S), n - 1, 8)
+    for start in (0, 1, 77):
+        assert pa.pa_reach_counts(rp, ci, start, 5) == oracle.reach_counts(oracle.block_adjacency(n, W, S), start, 5)
+    bad = ci.copy(); bad[-1] = n
+    with pytest.raises(pa.PaError, match="PA_ERR_LAYOUT"):
+        pa.pa_reach_counts(rp, bad, n - 1, 3)
+    with pytest.raises(pa.PaError, match="PA_ERR_INVALID_ARG"):
+        pa.pa_reach_counts(rp, ci, n, 3)

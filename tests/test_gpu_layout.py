@@ -76,3 +76,23 @@ def test_decode_block_list_is_the_layout_row(pa, oracle):
             got = pa.pa_decode_block_list(L, 64, W, S).cpu().numpy()
             rp, ci = oracle.block_layout(L, 64, W, S)
             np.testing.assert_array_equal(got, ci[rp[-2]:rp[-1]])
+
+
+def test_window_layout_bit_exact(pa, oracle):
+    """pa_build_window_layout (window + sink, no power-of-two term) against the oracle's
+    enumeration, against token-level brute force, and at the paper's 9 + 1 setting."""
+    for N in (1, 64, 65, 640, 4096 + 17, 70000):
+        for W in (1, 4, 9):
+            for S in (0, 1, 3):
+                rp, ci = pa.pa_build_window_layout(N, 64, W, S)
+                rp_ref, ci_ref = oracle.block_layout(N, 64, W, S, use_power=False)
+                np.testing.assert_array_equal(rp.cpu().numpy(), rp_ref)
+                np.testing.assert_array_equal(ci.cpu().numpy(), ci_ref)
+    for (N, B, W, S) in [(700, 8, 3, 1), (513, 4, 2, 2)]:
+        rp, ci = pa.pa_build_window_layout(N, B, W, S)
+        rp_ref, ci_ref = oracle.block_layout_from_tokens(N, B, W, S, use_power=False)
+        np.testing.assert_array_equal(rp.cpu().numpy(), rp_ref)
+        np.testing.assert_array_equal(ci.cpu().numpy(), ci_ref)
+    rp, ci = pa.pa_build_window_layout(128 * 256, 256, 9, 1)
+    assert (ci[int(rp[-2]):].cpu().numpy() + 1).tolist() == [1, 120, 121, 122, 123, 124, 125, 126, 127, 128]
+    assert pa.pa_reach_counts(rp.cpu().numpy(), ci.cpu().numpy(), 127, 1) == [10]

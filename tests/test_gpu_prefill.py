@@ -258,3 +258,164 @@ def test_strided_output_is_written_only_inside_its_view(pa, oracle, o_dtype):
     outside = torch.ones_like(big, dtype=torch.bool)
     outside[:, :N, 1:1 + Hq] = False
     assert bool((big[outside] == 7.0).all()), "elements outside the output view were overwritten"
+
+
+@pytest.mark.parametrize("o_dtype", [torch.bfloat16, torch.float32])
+def test_variable_length_batch(pa, oracle, o_dtype):
+    """Sequences of 1, 63, 64, 65, 0, 5000 and 32768 tokens packed into one call (Algorithm 1 takes no
+    batch argument: one layout serves them all).  Oracle side: one sequence at a time.  The output
+    buffer has sentinel rows behind the last token and every sequence's neighbours are checked
+    by the element-wise comparison itself (a box store over a ragged last block would show there)."""
+    Hq, Hkv, D, W, S = 8, 2, 128, 5, 1
+    lens = [1, 63, 64, 65, 0, 5000, 32768]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    total = int(cu[-1])
+    Q = si.bf16_randn((total, Hq, D), 801)
+    K = si.bf16_randn((total, Hkv, D), 802, 2.0)
+    V = si.bf16_randn((total, Hkv, D), 803)
+    rp, ci = pa.pa_build_layout(max(lens), 64, W, S)
+    big = torch.full((total + 70, Hq, D), 7.0, dtype=o_dtype, device="cuda")
+    o, lse, ws = pa.pa_prefill_varlen(Q.cuda(), K.cuda(), V.cuda(), torch.as_tensor(cu).cuda(), max(lens), rp, ci,
+                                      o=big[:total], o_dtype=o_dtype)
+    pa.pa_prefill_status(ws)
+    assert bool((big[total:] == 7.0).all()), "rows behind the last sequence were overwritten"
+    for b, n in enumerate(lens):
+        if n == 0:
+            continue
+        a, e = int(cu[b]), int(cu[b + 1])
+        o_ref, lse_ref, _ = oracle.prefill(Q[None, a:e], K[None, a:e], V[None, a:e], 64, W, S)
+        compare(o[None, a:e], lse[None, :, a:e], o_ref, lse_ref, f"sequence {b} of {n} tokens")
+
+
+def test_variable_length_batch_equals_one_call_per_sequence(pa):
+    """Bit for bit: the packed call and separate pa_prefill calls run the same arithmetic per row."""
+    Hq, Hkv, D, W, S = 28, 4, 128, 5, 1
+    lens = [3000, 130, 4096, 777]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    total = int(cu[-1])
+    Q, K, V = (si.bf16_randn((total, h, D), 810 + i).cuda() for i, h in enumerate((Hq, Hkv, Hkv)))
+    rp, ci = pa.pa_build_layout(max(lens), 64, W, S)
+    o, lse, ws = pa.pa_prefill_varlen(Q, K, V, torch.as_tensor(cu).cuda(), max(lens), rp, ci)
+    pa.pa_prefill_status(ws)
+    for b, n in enumerate(lens):
+        a, e = int(cu[b]), int(cu[b + 1])
+        rp1, ci1 = pa.pa_build_layout(n, 64, W, S)
+        o1, lse1, ws1 = pa.pa_prefill(Q[None, a:e], K[None, a:e], V[None, a:e], rp1, ci1)
+        pa.pa_prefill_status(ws1)
+        assert torch.equal(o1[0], o[a:e]) and torch.equal(lse1[0], lse[:, a:e])
+
+
+def test_rows_the_layout_leaves_empty(pa, oracle):
+    """A caller's CSR may list nothing for a query block: its rows get O = 0 and LSE = -inf, the
+    other rows are untouched by it (oracle: the dense token mask that the CSR stands for)."""
+    N, Hq, Hkv, D = 700, 8, 2, 128
+    nqb = (N + 63) // 64
+    rp_full, ci_full = oracle.block_layout(N, 64, 5, 1)
+    empty = {0, 3, 4, nqb - 1}
+    rows = [[] if i in empty else ci_full[rp_full[i]:rp_full[i + 1]].tolist() for i in range(nqb)]
+    rp = np.concatenate([[0], np.cumsum([len(r) for r in rows])]).astype(np.int32)
+    ci = np.asarray([j for r in rows for j in r], dtype=np.int32)
+    dense = np.zeros((N, N), dtype=bool)
+    for i, r in enumerate(rows):
+        for j in r:
+            dense[i * 64:(i + 1) * 64, j * 64:(j + 1) * 64] = True
+    dense &= np.tril(np.ones((N, N), dtype=bool))
+    Q, K, V = si.bf16_randn((1, N, Hq, D), 821), si.bf16_randn((1, N, Hkv, D), 822), si.bf16_randn((1, N, Hkv, D), 823)
+    o, lse, ws = pa.pa_prefill(Q.cuda(), K.cuda(), V.cuda(), torch.as_tensor(rp).cuda(), torch.as_tensor(ci).cuda())
+    pa.pa_prefill_status(ws)
+    o_ref, lse_ref, cnt = oracle.prefill(Q, K, V, 64, 5, 1, dense=dense)
+    dead = np.array([q // 64 in empty for q in range(N)])
+    assert (cnt[dead] == 0).all() and (cnt[~dead] > 0).all()
+    assert (o[0, dead] == 0).all() and torch.isinf(lse[0, :, dead]).all() and (lse[0, :, dead] < 0).all()
+    live = torch.as_tensor(np.nonzero(~dead)[0]).cuda()
+    compare(o[:, live], lse[:, :, live], o_ref[:, ~dead], lse_ref[:, :, ~dead], "rows beside empty ones")
+
+
+def test_batch_of_two_at_32k_on_sampled_rows(pa, oracle):
+    """Batch 2 at the 32K workload's shape: the unit grid spans both batch entries."""
+    w = si.PREFILL_32K
+    Q = si.bf16_randn((2, w.seq_len, w.n_q_heads, w.head_dim), 831)
+    K = si.bf16_randn((2, w.seq_len, w.n_kv_heads, w.head_dim), 832, 2.0)
+    V = si.bf16_randn((2, w.seq_len, w.n_kv_heads, w.head_dim), 833)
+    o, lse = _gpu_prefill(pa, Q, K, V, w.window_blocks, w.sink_blocks)
+    rows = _sampled_rows(w.seq_len, np.random.default_rng(834), n_random=40)
+    o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, w.window_blocks, w.sink_blocks, rows=rows)
+    ridx = torch.as_tensor(rows).cuda()
+    compare(o[:, ridx], lse[:, :, ridx], o_ref, lse_ref, "batch 2 at 32K")
+
+
+def test_head_dim_64_at_32k_on_sampled_rows(pa, oracle):
+    N, Hq, Hkv, D = 32768, 16, 4, 64
+    Q, K, V = si.bf16_randn((1, N, Hq, D), 841), si.bf16_randn((1, N, Hkv, D), 842, 2.0), si.bf16_randn((1, N, Hkv, D), 843)
+    o, lse = _gpu_prefill(pa, Q, K, V, 5, 1)
+    rows = _sampled_rows(N, np.random.default_rng(844), n_random=64)
+    o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, 5, 1, rows=rows)
+    ridx = torch.as_tensor(rows).cuda()
+    compare(o[:, ridx], lse[:, :, ridx], o_ref, lse_ref, "head_dim 64 at 32K")
+
+
+def _row_matched_window(rp_pa):
+    """The sweep's comparison layout: row i lists block 0 and its most recent blocks, as many as
+    the PowerAttention row has (so both layouts have the same number of active block pairs)."""
+    cols, cnts = [], np.diff(rp_pa)
+    for i, cnt in enumerate(cnts):
+        recent = list(range(max(1, i - (int(cnt) - 1) + 1), i + 1))
+        row = sorted(set([0] + recent))
+        lo = max(1, i - (int(cnt) - 1) + 1)
+        while len(row) < min(int(cnt), i + 1):      # early rows where the sink falls inside the window
+            lo -= 1
+            row = sorted(set(row + [lo]))
+        cols.append(row)
+    rp = np.concatenate([[0], np.cumsum([len(c) for c in cols])]).astype(np.int32)
+    return rp, np.asarray([j for c in cols for j in c], dtype=np.int32), cols
+
+
+def test_sweep_lengths_and_comparison_masks_on_sampled_rows(pa, oracle):
+    """The sequence-length sweep's other points, each at its own size on sampled rows: 256K with the
+    PowerAttention layout and with the row-matched sliding window, 16K with dense causal, and the
+    short ends (4K, 8K, 64K) with the PowerAttention layout."""
+    for N in (4096, 8192, 65536):
+        w = si.sweep_workload(N)
+        Q, K, V = si.prefill_inputs(w)
+        o, lse = _gpu_prefill(pa, Q, K, V, w.window_blocks, w.sink_blocks)
+        rows = _sampled_rows(N, np.random.default_rng(w.seed), n_random=32)
+        o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, w.window_blocks, w.sink_blocks, rows=rows)
+        ridx = torch.as_tensor(rows).cuda()
+        compare(o[:, ridx], lse[:, :, ridx], o_ref, lse_ref, w.name)
+    # dense causal at 16K: the window covers every block
+    w = si.sweep_workload(16384)
+    Q, K, V = si.prefill_inputs(w)
+    nqb = w.seq_len // 64
+    rp, ci = oracle.block_layout(w.seq_len, 64, nqb, 0, use_power=False)
+    assert int(rp[-1]) == nqb * (nqb + 1) // 2
+    o, lse = _gpu_prefill(pa, Q, K, V, nqb, 0, layout=(torch.as_tensor(rp).cuda(), torch.as_tensor(ci).cuda()))
+    rows = _sampled_rows(w.seq_len, np.random.default_rng(w.seed), n_random=16)
+    o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, nqb, 0, use_power=False, rows=rows)
+    ridx = torch.as_tensor(rows).cuda()
+    compare(o[:, ridx], lse[:, :, ridx], o_ref, lse_ref, "dense causal at 16K")
+    del Q, K, V, o, lse
+    # 256K: the PowerAttention layout, then the row-matched window (per row: sink + a window of cnt - 1 blocks)
+    w = si.sweep_workload(262144)
+    Q, K, V = si.prefill_inputs(w)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    rp_pa, ci_pa = pa.pa_build_layout(w.seq_len, 64, w.window_blocks, w.sink_blocks)
+    o, lse, ws = pa.pa_prefill(Qd, Kd, Vd, rp_pa, ci_pa)
+    pa.pa_prefill_status(ws)
+    rows = _sampled_rows(w.seq_len, np.random.default_rng(w.seed), n_random=24)
+    o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, w.window_blocks, w.sink_blocks, rows=rows, heads=list(range(0, 28, 3)))
+    ridx = torch.as_tensor(rows).cuda()
+    hidx = torch.arange(0, 28, 3).cuda()
+    compare(o[:, ridx][:, :, hidx], lse[:, hidx][:, :, ridx], o_ref, lse_ref, "256K PowerAttention")
+    rp_w, ci_w, cols = _row_matched_window(rp_pa.cpu().numpy())
+    assert int(rp_w[-1]) == int(rp_pa[-1])
+    o, lse, ws = pa.pa_prefill(Qd, Kd, Vd, torch.as_tensor(rp_w).cuda(), torch.as_tensor(ci_w).cuda(), o=o, lse=lse, workspace=ws)
+    pa.pa_prefill_status(ws)
+    by_w = {}
+    for q in rows:
+        i = q // 64
+        by_w.setdefault(len(cols[i]) - (1 if i >= len(cols[i]) else 0), []).append(q)   # window width in blocks
+    for wblocks, qs in by_w.items():
+        # rows whose window does not reach block 0 are "sink + window"; early rows are plain causal windows
+        o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, wblocks, 1, use_power=False, rows=qs, heads=[0, 13, 27])
+        qidx, hsel = torch.as_tensor(qs).cuda(), torch.tensor([0, 13, 27]).cuda()
+        compare(o[:, qidx][:, :, hsel], lse[:, hsel][:, :, qidx], o_ref, lse_ref, f"256K row-matched window of {wblocks}")
