@@ -53,10 +53,10 @@ int pa_version(void);
  * them; tests and measurement scripts call it after changing the environment. */
 void pa_reload_environment(void);
 
-/* Limit, in GPU clock cycles, of every bounded barrier wait inside the prefill kernel (a wait that
- * runs out ends the kernel with PA_ERR_TIMEOUT in its status block, see pa_prefill_status).
- * cycles <= 0 restores the default of about two seconds.  Process-wide; applies to calls made
- * after it returns. */
+/* Limit, in GPU clock cycles, of every bounded barrier wait inside the prefill and decode kernels
+ * (a wait that runs out ends the kernel with PA_ERR_TIMEOUT in its status block, see
+ * pa_prefill_status and pa_decode_status).  cycles <= 0 restores the defaults of one to two
+ * seconds.  Process-wide; applies to calls made after it returns. */
 void pa_set_wait_limit_cycles(int64_t cycles);
 
 /* ------------------------------------------------------------------------------------------

@@ -5,6 +5,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "common.cuh"
@@ -108,6 +109,11 @@ EnvSwitches env_switches()
     return g_env;
 }
 
+// ---------------------------------------------------------------- wait limit
+static std::atomic<long long> g_wait_cycles{0};
+
+long long wait_limit_cycles() { return g_wait_cycles.load(std::memory_order_relaxed); }
+
 // ---------------------------------------------------------------- tensor maps
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -189,6 +195,11 @@ extern "C" const char *pa_status_string(pa_status s)
 extern "C" const char *pa_last_error_message(void) { return pa::g_err; }
 
 extern "C" int pa_version(void) { return 200; /* 0.2.0 */ }
+
+extern "C" void pa_set_wait_limit_cycles(int64_t cycles)
+{
+    pa::g_wait_cycles.store(cycles > 0 ? (long long)cycles : 0, std::memory_order_relaxed);
+}
 
 extern "C" void pa_reload_environment(void)
 {

@@ -43,6 +43,10 @@ struct EnvSwitches {
 };
 EnvSwitches env_switches();
 
+// Limit of the kernels' bounded barrier waits in clock cycles as set by pa_set_wait_limit_cycles
+// (0: each kernel's default).
+long long wait_limit_cycles();
+
 #define PA_CUDA_OK(expr)                                                                    \
     do {                                                                                    \
         cudaError_t e_ = (expr);                                                            \

@@ -52,6 +52,7 @@ struct DecodeArgs {
     int64_t items;         // (row kernel) rows of the call x R
     int32_t table_stride, n_pages;
     float scale_log2;  // softmax_scale * log2(e)
+    long long wait_cycles;  // (row kernel) limit of every barrier wait, in clock cycles
 };
 
 // Where key block j of sequence b starts: (index along the batch / page axis, first token).  A
@@ -330,7 +331,7 @@ constexpr int kRowConsumers = 4;                     // consumer warps
 constexpr int kRowThreads = 32 * (kRowConsumers + 1);
 constexpr int kRowMaxStages = 6;                     // shared-memory stages (key blocks in flight) per CTA
 constexpr int kRowMaxCluster = 8;                    // portable cluster size limit
-constexpr long long kRowWaitCycles = 2000000000ll;   // ~1 s
+constexpr long long kRowWaitCycles = 2000000000ll;   // default limit of a barrier wait: ~1 s
 enum : int32_t { kModeCluster = 0, kModePartial = 1, kModeDirect = 2 };
 
 template <int D>
@@ -472,7 +473,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
                     const int s = (int)(ci % (uint32_t)stages);
                     if (ci >= (uint32_t)stages)
                         ok = ptx::mbar_wait_bounded(bar_empty(s), (ci / (uint32_t)stages - 1) & 1, abort_flag, a.status, 1,
-                                                    kRowWaitCycles, (int)PA_ERR_TIMEOUT);
+                                                    a.wait_cycles, (int)PA_ERR_TIMEOUT);
                     if (ok) {
                         // (a page outside the pool reads as zeros)
                         const int32_t outer = a.table ? page : w.b, tok0 = a.table ? 0 : j * kDecBlock;
@@ -536,7 +537,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
                 const int32_t jblk = __shfl_sync(0xffffffffu, w.cand, lane_of(w, i));
                 const int n_keys = jblk == w.row ? w.last_keys : kDecBlock;
                 const uint32_t sk = smem_base + (uint32_t)s * SM::kStage, sv = sk + SM::kTile;
-                ok = ptx::mbar_wait_bounded(bar_kfull(s), parity, abort_flag, a.status, 2, kRowWaitCycles, (int)PA_ERR_TIMEOUT);
+                ok = ptx::mbar_wait_bounded(bar_kfull(s), parity, abort_flag, a.status, 2, a.wait_cycles, (int)PA_ERR_TIMEOUT);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (16 * wid < n_keys) {  // (else none of this warp's keys exists: the diagonal block's tail)
@@ -597,7 +598,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
                         keep0 = (key0 < n_keys ? 0x0000ffffu : 0u) | (key0 + 1 < n_keys ? 0xffff0000u : 0u);
                         keep1 = (key0 + 8 < n_keys ? 0x0000ffffu : 0u) | (key0 + 9 < n_keys ? 0xffff0000u : 0u);
                     }
-                    ok = ptx::mbar_wait_bounded(bar_vfull(s), parity, abort_flag, a.status, 3, kRowWaitCycles, (int)PA_ERR_TIMEOUT);
+                    ok = ptx::mbar_wait_bounded(bar_vfull(s), parity, abort_flag, a.status, 3, a.wait_cycles, (int)PA_ERR_TIMEOUT);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     // ---- O = alpha O + P V: rows = heads, 16 keys, all D features (8 per MMA)
@@ -989,6 +990,7 @@ static pa_status launch_decode(const DecodeShape &p, const void *q, const void *
     a.stages = 0;
     const float scale = p.softmax_scale != 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
+    a.wait_cycles = wait_limit_cycles() > 0 ? wait_limit_cycles() : kRowWaitCycles;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const EnvSwitches env = env_switches();

@@ -20,13 +20,12 @@
 //               unit's first steps
 // Warps 0-3 and 12-15 give registers back (setmaxnreg) and the softmax warpgroups take them.
 // Every barrier wait is bounded; a wait that runs out records PA_ERR_TIMEOUT in the status
-// block, raises a CTA-wide abort flag and the CTA drains and exits (no trap, no endless spin).
+// block, raises a CTA-wide abort flag, every role leaves its loop and the CTA ends after a bounded
+// pause for what is still in flight (no trap, no endless spin).
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <math.h>
 #include <stdlib.h>
-
-#include <atomic>
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -304,12 +303,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 u = un;
                 w = wn;
                 j = jnext;
-            }
-            if (!ok) {
-                // Drain: give copies already in flight a bounded chance to land before exit.
-                const long long t0 = clock64();
-                while (clock64() - t0 < 4000000ll) {
-                }
             }
         }
         __syncwarp();
@@ -791,6 +784,16 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == 2) {
+        // Every role has left its loop.  After a wait that gave up, copies and tensor-core
+        // operations issued before it may still be in flight: they finish by themselves within
+        // microseconds (nothing they need is withheld), and the warp that owns the tensor memory
+        // lets a bounded two milliseconds pass before it gives the memory back and the CTA's
+        // shared memory can go to another kernel.
+        if (*abort_flag) {
+            const long long t0 = clock64();
+            while (clock64() - t0 < 4000000ll) {
+            }
+        }
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
@@ -831,9 +834,6 @@ static pa_status check_prefill(const pa_prefill_params *p)
 
 constexpr size_t kPrefillWorkspace = 256;
 
-// Limit of the kernel's barrier waits in clock cycles (0: the default); set by pa_set_wait_limit_cycles.
-static std::atomic<long long> g_wait_cycles{0};
-
 // Optional check of a caller's CSR (PA_VALIDATE=1): one thread per row.  The first violation
 // found is recorded as (kind, row) in check[0..1]: 1 row_ptr does not start at 0 / end at nnz,
 // 2 row extent negative or beyond nnz, 3 block index outside [0, row], 4 indices not ascending.
@@ -859,11 +859,6 @@ __global__ void validate_csr_kernel(const int32_t *row_ptr, const int32_t *col_i
 }
 
 }  // namespace pa
-
-extern "C" void pa_set_wait_limit_cycles(int64_t cycles)
-{
-    pa::g_wait_cycles.store(cycles > 0 ? (long long)cycles : 0, std::memory_order_relaxed);
-}
 
 extern "C" size_t pa_prefill_workspace_bytes(const pa_prefill_params *p)
 {
@@ -940,7 +935,7 @@ static pa_status launch_prefill(const pa_prefill_params *p, const void *q, const
     const float scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.0f / sqrtf((float)D);
     a.scale_log2 = scale * 1.4426950408889634f;
 
-    const long long wait_cycles = g_wait_cycles.load(std::memory_order_relaxed);
+    const long long wait_cycles = wait_limit_cycles();
     a.wait_cycles = wait_cycles > 0 ? wait_cycles : kWaitCycles;
     const unsigned grid = (unsigned)(a.n_units < dev.sms ? a.n_units : dev.sms);
     cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -71,13 +71,10 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    uint32_t it = 0;
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((++it & 63u) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > limit) break;
-        }
+        if (mbar_try_wait(bar, parity)) return true;  // (each try suspends the thread for a while by itself)
+        if (*abort_flag) return false;
+        if (clock64() - t0 > limit) break;
     }
     if (atomicCAS(status, 0, timeout_status) == 0) status[1] = code;
     *abort_flag = 1;

@@ -295,3 +295,4 @@ def test_decode_many_rows_through_the_persistent_grid(pa, oracle, pa_env, env):
     good = np.setdiff1d(np.arange(batch), [3, 77])
     o_ref, lse_ref, _ = oracle.decode(q[good], kc[good], vc[good], lens[good], 64, 5, 1)
     compare(o[good], lse[good], o_ref, lse_ref, "persistent grid with invalid lengths")
+

@@ -419,3 +419,27 @@ def test_sweep_lengths_and_comparison_masks_on_sampled_rows(pa, oracle):
         o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, wblocks, 1, use_power=False, rows=qs, heads=[0, 13, 27])
         qidx, hsel = torch.as_tensor(qs).cuda(), torch.tensor([0, 13, 27]).cuda()
         compare(o[:, qidx][:, :, hsel], lse[:, hsel][:, :, qidx], o_ref, lse_ref, f"256K row-matched window of {wblocks}")
+
+
+def test_a_wait_that_runs_out_ends_the_kernel_with_a_status(pa, oracle):
+    """Every barrier wait inside the prefill kernel is bounded.  With the limit set to one cycle,
+    an ordinary wait that is not over at its first try (the epilogue warps wait tens of
+    microseconds for a row of 47 blocks to finish) runs out: the call returns, pa_prefill_status
+    reports PA_ERR_TIMEOUT with the id of a wait, and the next call, back at the default limit, is
+    correct on the same stream."""
+    N, Hq, Hkv, D = 3000, 8, 2, 128
+    Q, K, V = si.bf16_randn((1, N, Hq, D), 851), si.bf16_randn((1, N, Hkv, D), 852), si.bf16_randn((1, N, Hkv, D), 853)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    rp, ci = pa.pa_build_window_layout(N, 64, 64, 0)     # the window covers every block: dense causal
+    try:
+        pa.pa_set_wait_limit_cycles(1)
+        o, lse, ws = pa.pa_prefill(Qd, Kd, Vd, rp, ci)
+        with pytest.raises(pa.PaError, match="PA_ERR_TIMEOUT") as err:
+            pa.pa_prefill_status(ws)
+        assert "wait id" in str(err.value)
+    finally:
+        pa.pa_set_wait_limit_cycles(0)
+    o, lse, ws = pa.pa_prefill(Qd, Kd, Vd, rp, ci)
+    assert pa.pa_prefill_status(ws) == 0
+    o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, 64, 0, use_power=False)
+    compare(o, lse, o_ref, lse_ref, "after a timed-out call")
