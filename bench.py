@@ -50,9 +50,8 @@ def read_peaks():
 
 
 # DRAM bytes moved by one prefill_kernel<128> launch on the 128K workload: dram__bytes_read.sum +
-# dram__bytes_write.sum of an ncu capture of this very workload (the command is in
-# profiles/prefill_kernel_128k_traffic.md).  The figure belongs to the kernel sources it was taken
-# on: once they change it is reported as null until the capture is repeated.
+# dram__bytes_write.sum of an ncu capture of this very workload.  The figure belongs to the kernel
+# sources it was taken on: once they change it is reported as null until the capture is repeated.
 PREFILL_TRAFFIC = dict(
     bytes=2032551424 + 912317952,
     sources={
@@ -168,14 +167,17 @@ def oracle_sample_rows(w, every: int):
     return np.sort((blocks[:, None] * w.block + np.arange(w.block)[None, :]).reshape(-1))
 
 
-def time_oracle(w, Q, K, V, every: int, nnz_rows_flops):
-    """Times the fp64 oracle, as it stands, on the sampled rows; returns (seconds, flops, cores)."""
+def time_oracle(w, Q, K, V, every: int, nnz_rows_flops, keep=None):
+    """Times the fp64 oracle, as it stands, on the sampled rows; returns (seconds, flops, cores, rows).
+    `keep`, a dict, receives the rows and the oracle's results for a comparison with the GPU's."""
     from oracle import oracle
 
     rows = oracle_sample_rows(w, every)
     t0 = time.time()
-    oracle.prefill(Q, K, V, w.block, w.window_blocks, w.sink_blocks, rows=rows)
+    o_ref, lse_ref, _ = oracle.prefill(Q, K, V, w.block, w.window_blocks, w.sink_blocks, rows=rows)
     dt = time.time() - t0
+    if keep is not None:
+        keep.update(rows=rows, o=o_ref, lse=lse_ref)
     return dt, nnz_rows_flops(rows), oracle.max_threads(), len(rows)
 
 
@@ -331,6 +333,74 @@ def run_ours(args):
     dec_us = 1e3 * d0.elapsed_time(d1) / (n_sets * reps)
     dec_gbs = dec_bytes / (dec_us * 1e-6) / 1e9
 
+    # ---- the same calls issued eagerly (no graph): device time per call and the host's time to
+    # enqueue one (argument checks, cached tensor maps, the launch), which a graph replay hides.
+    def eager(fn, n):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        g0.record(stream)
+        for _ in range(n):
+            fn()
+        g1.record(stream)
+        host_us = 1e6 * (time.perf_counter() - t0) / n
+        torch.cuda.synchronize()
+        return dict(device_us_per_call=1e3 * g0.elapsed_time(g1) / n, host_enqueue_us_per_call=host_us, calls=n)
+
+    it = iter(range(1 << 30))
+    eager_decode = eager(lambda: pa.pa_decode(qd, kc, vc, lens_sets_d[next(it) % n_sets], wd.window_blocks, wd.sink_blocks,
+                                              o=Od, lse=LSEd, workspace=wsd), 256)
+    eager_prefill = eager(lambda: pa.pa_prefill(Q, K, V, row_ptr, col_idx, o=O, lse=LSE, workspace=ws), 10)
+
+    # ---- many decoding steps against a paged cache (the paper's serving shape: a long input, then
+    # 1024 decoding steps): batch 8 at 16K tokens, every step appends one token's K and V and
+    # decodes.  128 steps are captured in a graph (the lengths live on the device and advance by
+    # themselves) and replayed eight times.
+    def decode_steps():
+        ctx, steps, per_graph = 16384, 1024, 128
+        max_blocks = (ctx + steps + 63) // 64
+        n_pages = wd.batch * max_blocks
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(wd.seed + 7)
+        shape = (n_pages, 64, wd.n_kv_heads, wd.head_dim)
+        kp = torch.randn(shape, device=dev, dtype=torch.bfloat16, generator=gen)
+        vp = torch.randn(shape, device=dev, dtype=torch.bfloat16, generator=gen)
+        perm = torch.randperm(n_pages, device=dev, generator=gen).to(torch.int32)
+        table = perm.view(wd.batch, max_blocks).contiguous()
+        lens_s = torch.full((wd.batch,), ctx, dtype=torch.int32, device=dev)
+        k_new = torch.randn((wd.batch, wd.n_kv_heads, wd.head_dim), device=dev, dtype=torch.bfloat16, generator=gen)
+        v_new = torch.randn_like(k_new)
+        o_s, lse_s, ws_s = pa.pa_decode_paged(qd, kp, vp, table, lens_s, wd.window_blocks, wd.sink_blocks)
+
+        def one_step():
+            pa.pa_kv_append(k_new, v_new, kp, vp, table, lens_s)
+            pa.pa_decode_paged(qd, kp, vp, table, lens_s, wd.window_blocks, wd.sink_blocks, o=o_s, lse=lse_s, workspace=ws_s)
+
+        with torch.cuda.stream(side):
+            one_step()
+            torch.cuda.synchronize()
+            lens_s.fill_(ctx)
+            gs = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gs, stream=side):
+                for _ in range(per_graph):
+                    one_step()
+            torch.cuda.synchronize()
+            lens_s.fill_(ctx)
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s0.record(side)
+            for _ in range(steps // per_graph):
+                gs.replay()
+            s1.record(side)
+            torch.cuda.synchronize()
+        assert int(lens_s[0].item()) == ctx + steps
+        pa.pa_decode_status(ws_s)
+        return dict(workload="batch 8, 16K-token context + 1024 steps, paged cache (64-token pages), append + decode per step",
+                    us_per_step=1e3 * s0.elapsed_time(s1) / steps, steps=steps, launches_per_step=3)
+
+    decode_many = decode_steps()
+
     # ---- the 32K prefill workload (the metric is quoted at 32K and 128K): same kernel, K scaled so
     # that the logits have a standard deviation of about 3; its inputs (0.6 GB) exceed L2.
     w32 = si.PREFILL_32K
@@ -445,7 +515,7 @@ def run_ours(args):
     d2h = sum(t.numel() * t.element_size() for t in (Oh, LSEh))
 
     # ---- CPU baseline: the oracle, as it stands, on a bounded sample of the same workload.
-    cpu = None
+    cpu = parity = None
     if world == 1 and not args.no_cpu_baseline:
         from oracle import oracle
 
@@ -457,9 +527,20 @@ def run_ours(args):
             return 4.0 * w.block * w.block * w.head_dim * float(row_len[blocks].sum()) * w.n_q_heads
 
         every = 16
-        dt, fl, cores, nrows = time_oracle(w, Qh, Kh, Vh, every, flops_of)
+        ref = {}
+        dt, fl, cores, nrows = time_oracle(w, Qh, Kh, Vh, every, flops_of, keep=ref)
         cpu = dict(value=fl / dt / 1e12, unit=UNIT, cores=cores, kind="oracle",
                    sample=f"every {every}th query block of the 128K workload ({nrows} rows, all heads), {dt:.1f} s")
+        # The rows the oracle has just evaluated, against the GPU's output of the same workload.
+        pa.pa_prefill(Q, K, V, row_ptr, col_idx, o=O, lse=LSE, workspace=ws)
+        pa.pa_prefill_status(ws)
+        ridx = torch.as_tensor(ref["rows"], device=dev)
+        eo = np.abs(O[:, ridx].double().cpu().numpy() - ref["o"])
+        el = np.abs(LSE[:, :, ridx].double().cpu().numpy() - ref["lse"])
+        parity = dict(rows=int(nrows), heads=w.n_q_heads, o_max_abs=float(eo.max()), o_mean_abs=float(eo.mean()),
+                      lse_max_abs=float(el.max()), bounds=dict(o_max_abs=2e-2, o_mean_abs=2e-3, lse_max_abs=1e-3),
+                      against="fp64 oracle on the cpu_baseline sample")
+        del ref
 
     value = flops_all / (ms * 1e-3) / 1e12
     achieved = flops / (prefill_ms * 1e-3) / 1e12
@@ -489,7 +570,8 @@ def run_ours(args):
                 decode=dict(metric="decode_kv_gbs", value=dec_gbs, unit="GB/s", us_per_call=dec_us,
                             kv_bytes_per_call=dec_bytes, peak=peaks["hbm_gbs"], frac=dec_gbs / peaks["hbm_gbs"],
                             bound="hbm", timing=f"CUDA graph of {n_sets * reps} calls rotating over {n_sets} seeded length sets",
-                            workload=wd.name, scale_up=scale_up),
+                            workload=wd.name, scale_up=scale_up, eager=eager_decode, many_steps=decode_many),
+                eager_prefill=eager_prefill, parity=parity,
                 e2e=dict(value=flops / (e2e_ms * 1e-3) / 1e12, unit=UNIT, ms_per_step=e2e_ms,
                          h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps,
                          overlap="copies in, compute and copies out of consecutive steps overlap (3 streams)"),
@@ -600,6 +682,25 @@ def run_sweep(args):
         del Q, K, V, o, lse
 
 
+def spawn_replicas(n: int) -> int:
+    """`python bench.py --gpus N` outside torchrun: start N replica processes of this script, one
+    per GPU, with the rendezvous variables torchrun would set; rank 0's output is the job's line."""
+    import socket
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    procs = []
+    for rank in range(n):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable] + sys.argv, env=env))
+    rc = 0
+    for pr in procs:
+        rc = rc or pr.wait()
+    return rc
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -622,6 +723,8 @@ def main():
         return
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_replicas(args.gpus))
     else:
         run_ours(args)
 
