@@ -53,10 +53,10 @@ def read_peaks():
 # dram__bytes_write.sum of an ncu capture of this very workload.  The figure belongs to the kernel
 # sources it was taken on: once they change it is reported as null until the capture is repeated.
 PREFILL_TRAFFIC = dict(
-    bytes=2032551424 + 912317952,
+    bytes=2046557440 + 913454336,
     sources={
-        "prefill_sm100.cu": "9d515cbb0f83b5cb9e80385d943efe650dfa3571bd35d4f19124baba46c8bf0d",
-        "sm100_ptx.cuh": "cc5cb63f8da5e88ddc941ca016a41fe337c2404ca754e7ea5c384e0a1552a5ca",
+        "prefill_sm100.cu": "a66e37af1b7b790bc81f8584f4395104207c2cba82d053d09e8013ec9ed257bf",
+        "sm100_ptx.cuh": "f0dd47ba76fa3fd147120ccffa5c14e4d442cb67ae25aedcff0959f1dbb6ad64",
     },
 )
 
@@ -596,6 +596,22 @@ def run_case(args):
         for _ in range(args.steps):
             pa.pa_prefill(Q, K, V, rp, ci, o=o, lse=lse, workspace=ws)
         pa.pa_prefill_status(ws)
+    elif args.case == "decode_persist":
+        # The persistent form of the decode row kernel on a case small enough for a full-set capture:
+        # batch 96 (384 rows), 16K-token caches (1.6 GB), lengths uniform in [8192, 16384].
+        wd = si.DECODE_B8
+        batch, max_len = 96, 16384
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(wd.seed + 96)
+        kc = torch.randn((batch, max_len, wd.n_kv_heads, wd.head_dim), device=dev, dtype=torch.bfloat16, generator=gen)
+        vc = torch.randn((batch, max_len, wd.n_kv_heads, wd.head_dim), device=dev, dtype=torch.bfloat16, generator=gen)
+        qd = torch.randn((batch, wd.n_q_heads, wd.head_dim), device=dev, dtype=torch.bfloat16, generator=gen)
+        lens = np.random.Generator(np.random.PCG64(wd.lens_seed + 96)).integers(max_len // 2, max_len + 1, size=batch)
+        lens_d = torch.as_tensor(lens, dtype=torch.int32, device=dev)
+        o, lse, ws = pa.pa_decode(qd, kc, vc, lens_d, wd.window_blocks, wd.sink_blocks)
+        for _ in range(args.steps):
+            pa.pa_decode(qd, kc, vc, lens_d, wd.window_blocks, wd.sink_blocks, o=o, lse=lse, workspace=ws)
+        pa.pa_decode_status(ws)
     else:
         wd = si.DECODE_B8
         qd, kc, vc, lens = si.decode_inputs(wd)
@@ -709,7 +725,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode-scale-up", action="store_true", help="skip the batch-64/256 decode lines")
-    ap.add_argument("--case", default=None, choices=["prefill32k", "decode"],
+    ap.add_argument("--case", default=None, choices=["prefill32k", "decode", "decode_persist"],
                     help="run only a small single-kernel case (for profiler captures)")
     ap.add_argument("--sweep", action="store_true", help="sequence-length sweep with comparison layouts")
     ap.add_argument("--sweep-max-len", type=int, default=262144)
