@@ -3,7 +3,7 @@
 Python face of ``pa_oracle.c`` (fp64, dense token-level mask, Eq. (1) row by row) plus the
 graph-side checks of the paper: brute-force block layout from the token mask, the block-level
 predicate for large sizes, and breadth-first reachability over the mask seen as a DAG
-(Section 3.1; Appendix A; Appendix B).
+(Section 3.1; Appendix A; Appendix B); and the gradients of Eq. (1) for the backward pass.
 
 The product library never imports this module; this module never imports the product.
 Every function here is pinned by ``tests/test_oracle_*.py``; none is "parity unpinned".
@@ -52,6 +52,9 @@ def _load():
         lib.pa_oracle_decode.argtypes = [_p, _p, _p, _p, _i64, _i64, _i64, _i64, _i64,
                                          ctypes.c_double, _i64, _i64, _i64, ctypes.c_int, _p, _p,
                                          _p, ctypes.c_int]
+        lib.pa_oracle_backward.restype = None
+        lib.pa_oracle_backward.argtypes = [_p, _p, _p, _p, _i64, _i64, _i64, _i64, _i64, ctypes.c_double, _i64, _i64,
+                                           _i64, ctypes.c_int, _p, _p, _p, _p, ctypes.c_int]
         lib.pa_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -294,3 +297,27 @@ def decode(q, Kc, Vc, lens, B: int, W: int, S: int = 1, scale: Optional[float] =
                          float(scale), B, W, S, int(use_power), _ptr(O), _ptr(LSE), _ptr(cnt),
                          int(threads))
     return O, LSE, cnt
+
+
+def backward(Q, K, V, dO, B: int, W: int, S: int = 1, scale: Optional[float] = None, use_power: bool = True,
+             dense: Optional[np.ndarray] = None, threads: int = 0):
+    """Gradients of Eq. (1) under Algorithm 1's mask (or an explicit dense [N, N] mask) for an
+    upstream gradient dO of the output: returns (dQ [batch, N, Hq, D], dK, dV [batch, N, Hkv, D]) fp64.
+    Inputs bf16 as in `prefill`; O(N^2) pair evaluations, for small N."""
+    lib = _load()
+    q, k, v, g = _bf16_bits(Q), _bf16_bits(K), _bf16_bits(V), _bf16_bits(dO)
+    batch, N, Hq, D = q.shape
+    Hkv = k.shape[2]
+    assert k.shape == (batch, N, Hkv, D) and v.shape == k.shape and g.shape == q.shape and Hq % Hkv == 0
+    if scale is None:
+        scale = 1.0 / float(np.sqrt(D))
+    dm = None
+    if dense is not None:
+        dm = np.ascontiguousarray(dense.astype(np.uint8))
+        assert dm.shape == (N, N)
+    dQ = np.zeros(q.shape, dtype=np.float64)
+    dK = np.zeros(k.shape, dtype=np.float64)
+    dV = np.zeros(k.shape, dtype=np.float64)
+    lib.pa_oracle_backward(_ptr(q), _ptr(k), _ptr(v), _ptr(g), batch, N, Hq, Hkv, D, float(scale), B, W, S,
+                           int(use_power), _ptr(dm), _ptr(dQ), _ptr(dK), _ptr(dV), int(threads))
+    return dQ, dK, dV

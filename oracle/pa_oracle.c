@@ -199,3 +199,108 @@ int pa_oracle_max_threads(void)
     return 1;
 #endif
 }
+
+/*
+ * Backward of Eq. (1) (the paper trains with the mask, Section 4.1; it prints no gradient formulas,
+ * these follow from differentiating Eq. (1)).  For one query row i with attended set A, weights
+ * p_j = softmax_A(scale <q, k_j>) and output o = sum_j p_j v_j, and an upstream gradient g = dL/do:
+ *     dL/dv_j  = p_j g
+ *     dL/dp_j  = <g, v_j>
+ *     dL/ds_j  = p_j (dL/dp_j - sum_k p_k dL/dp_k)          (softmax over A)
+ *     dL/dq    = scale sum_j dL/ds_j k_j
+ *     dL/dk_j  = scale dL/ds_j q
+ * dK and dV sum over the query rows that attend to key j and over the query heads that share its
+ * KV head.  Two plain passes, neither with any blocking: rows (dQ, and the per-row log-sum-exp and
+ * sum_k p_k dL/dp_k), then keys (dK, dV), each re-evaluating the mask predicate pair by pair.
+ * Q, dO [batch, N, Hq, D]; K, V [batch, N, Hkv, D] bf16 bit patterns; outputs fp64, same shapes.
+ */
+void pa_oracle_backward(const uint16_t *Q, const uint16_t *K, const uint16_t *V, const uint16_t *dO,
+                        int64_t batch, int64_t N, int64_t Hq, int64_t Hkv, int64_t D, double scale,
+                        int64_t B, int64_t W, int64_t sink_blocks, int use_power,
+                        const uint8_t *dense_mask, double *dQ, double *dK, double *dV, int n_threads)
+{
+    const int64_t G = Hq / Hkv;
+    double *lse = (double *)malloc((size_t)(batch * Hq * N) * sizeof(double));
+    double *dsum = (double *)malloc((size_t)(batch * Hq * N) * sizeof(double));
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#endif
+#pragma omp parallel
+    {
+        double *s = (double *)malloc((size_t)N * sizeof(double));
+        double *dp = (double *)malloc((size_t)N * sizeof(double));
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t t = 0; t < batch * Hq * N; ++t) {
+            const int64_t b = t / (Hq * N), h = (t / N) % Hq, i = t % N, hk = h / G;
+            const uint16_t *q = Q + ((b * N + i) * Hq + h) * D;
+            const uint16_t *g = dO + ((b * N + i) * Hq + h) * D;
+            double m = -INFINITY;
+            for (int64_t j = 0; j < N; ++j) {
+                const int on = dense_mask ? dense_mask[i * N + j] : pa_oracle_mask(i, j, B, W, sink_blocks, use_power);
+                s[j] = -INFINITY;
+                if (!on) continue;
+                const uint16_t *k = K + ((b * N + j) * Hkv + hk) * D;
+                const uint16_t *v = V + ((b * N + j) * Hkv + hk) * D;
+                double acc = 0.0, gv = 0.0;
+                for (int64_t d = 0; d < D; ++d) {
+                    acc += bf16_to_double(q[d]) * bf16_to_double(k[d]);
+                    gv += bf16_to_double(g[d]) * bf16_to_double(v[d]);
+                }
+                s[j] = acc * scale;
+                dp[j] = gv;
+                if (s[j] > m) m = s[j];
+            }
+            double l = 0.0, pd = 0.0;
+            for (int64_t j = 0; j < N; ++j)
+                if (s[j] != -INFINITY) l += exp(s[j] - m);
+            double *dq = dQ + ((b * N + i) * Hq + h) * D;
+            for (int64_t d = 0; d < D; ++d) dq[d] = 0.0;
+            if (l == 0.0) { /* empty row: no gradient flows */
+                lse[t] = INFINITY;
+                dsum[t] = 0.0;
+                continue;
+            }
+            for (int64_t j = 0; j < N; ++j)
+                if (s[j] != -INFINITY) pd += exp(s[j] - m) / l * dp[j];
+            for (int64_t j = 0; j < N; ++j) {
+                if (s[j] == -INFINITY) continue;
+                const double ds = exp(s[j] - m) / l * (dp[j] - pd);
+                const uint16_t *k = K + ((b * N + j) * Hkv + hk) * D;
+                for (int64_t d = 0; d < D; ++d) dq[d] += scale * ds * bf16_to_double(k[d]);
+            }
+            lse[t] = m + log(l);
+            dsum[t] = pd;
+        }
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t t = 0; t < batch * Hkv * N; ++t) {
+            const int64_t b = t / (Hkv * N), hk = (t / N) % Hkv, j = t % N;
+            const uint16_t *k = K + ((b * N + j) * Hkv + hk) * D;
+            const uint16_t *v = V + ((b * N + j) * Hkv + hk) * D;
+            double *dk = dK + ((b * N + j) * Hkv + hk) * D;
+            double *dv = dV + ((b * N + j) * Hkv + hk) * D;
+            for (int64_t d = 0; d < D; ++d) dk[d] = dv[d] = 0.0;
+            for (int64_t h = hk * G; h < (hk + 1) * G; ++h)
+                for (int64_t i = 0; i < N; ++i) {
+                    const int on = dense_mask ? dense_mask[i * N + j] : pa_oracle_mask(i, j, B, W, sink_blocks, use_power);
+                    if (!on) continue;
+                    const uint16_t *q = Q + ((b * N + i) * Hq + h) * D;
+                    const uint16_t *g = dO + ((b * N + i) * Hq + h) * D;
+                    double acc = 0.0, gv = 0.0;
+                    for (int64_t d = 0; d < D; ++d) {
+                        acc += bf16_to_double(q[d]) * bf16_to_double(k[d]);
+                        gv += bf16_to_double(g[d]) * bf16_to_double(v[d]);
+                    }
+                    const double p = exp(acc * scale - lse[(b * Hq + h) * N + i]);
+                    const double ds = p * (gv - dsum[(b * Hq + h) * N + i]);
+                    for (int64_t d = 0; d < D; ++d) {
+                        dv[d] += p * bf16_to_double(g[d]);
+                        dk[d] += scale * ds * bf16_to_double(q[d]);
+                    }
+                }
+        }
+        free(s);
+        free(dp);
+    }
+    free(lse);
+    free(dsum);
+}

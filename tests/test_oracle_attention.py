@@ -184,3 +184,65 @@ def test_bf16_widening_is_exact(oracle):
     Q = torch.ones((1, 1, 1, D), dtype=torch.bfloat16)
     O, _, _ = oracle.prefill(Q, Q.clone(), V, 4, 1, 1)
     np.testing.assert_array_equal(O[0, 0, 0], _f64(vals))
+
+
+# ------------------------------------------------------------------ backward of Eq. (1)
+
+def _autograd_reference(Q, K, V, dO, mask, scale):
+    """dQ, dK, dV of softmax-over-the-mask attention by torch's fp64 autograd on the dense form."""
+    import torch
+
+    q = Q.double().clone().requires_grad_(True)
+    k = K.double().clone().requires_grad_(True)
+    v = V.double().clone().requires_grad_(True)
+    G = q.shape[2] // k.shape[2]
+    kk, vv = k.repeat_interleave(G, dim=2), v.repeat_interleave(G, dim=2)
+    s = torch.einsum("bqhd,bkhd->bhqk", q, kk) * scale
+    s = s.masked_fill(~torch.as_tensor(mask)[None, None], float("-inf"))
+    o = torch.einsum("bhqk,bkhd->bqhd", torch.softmax(s, dim=-1), vv)
+    (o * dO.double()).sum().backward()
+    return q.grad.numpy(), k.grad.numpy(), v.grad.numpy()
+
+
+@pytest.mark.parametrize("N,Hq,Hkv,D,B,W,S,use_power", [
+    (200, 4, 2, 16, 8, 2, 1, True),        # window + powers + sink, grouped heads, ragged tail
+    (130, 3, 1, 8, 16, 0, 0, True),        # pure power-of-two pattern, a group of three
+    (96, 2, 2, 32, 4, 3, 2, False),        # sliding window with two sink blocks
+    (64, 2, 1, 8, 64, 5, 1, True),         # one block: plain causal attention
+])
+def test_backward_matches_autograd_on_the_dense_form(oracle, N, Hq, Hkv, D, B, W, S, use_power):
+    """The oracle's gradients against torch autograd (fp64) through a dense masked softmax: a
+    dropped term, a wrong sign, a missing scale or a wrong head grouping fails here."""
+    import synth_inputs as si
+
+    Q, K, V = si.bf16_randn((2, N, Hq, D), 7), si.bf16_randn((2, N, Hkv, D), 8, 2.0), si.bf16_randn((2, N, Hkv, D), 9)
+    dO = si.bf16_randn((2, N, Hq, D), 10)
+    scale = 0.37
+    dq, dk, dv = oracle.backward(Q, K, V, dO, B, W, S, scale=scale, use_power=use_power)
+    rq, rk, rv = _autograd_reference(Q, K, V, dO, oracle.dense_mask(N, B, W, S, use_power), scale)
+    for got, ref in ((dq, rq), (dk, rk), (dv, rv)):
+        assert np.abs(got - ref).max() <= 1e-10 * max(1.0, np.abs(ref).max())
+    # an explicit dense mask gives the same
+    dq2, dk2, dv2 = oracle.backward(Q, K, V, dO, B, W, S, scale=scale, dense=oracle.dense_mask(N, B, W, S, use_power))
+    assert np.abs(dq2 - dq).max() == 0 and np.abs(dk2 - dk).max() == 0 and np.abs(dv2 - dv).max() == 0
+
+
+def test_backward_closed_forms(oracle):
+    """What the calculus fixes without any reference: a constant upstream gradient per row gives
+    dS = 0 when V is constant (dP equal for every key), hence dQ = dK = 0 and dV_j = sum of the
+    weights that land on key j times dO; and the gradients of a single-key row are those of o = v."""
+    import synth_inputs as si
+
+    N, Hq, Hkv, D, B = 96, 2, 1, 8, 8
+    Q, K = si.bf16_randn((1, N, Hq, D), 21), si.bf16_randn((1, N, Hkv, D), 22)
+    vrow = si.bf16_randn((D,), 23)
+    V = vrow.expand(1, N, Hkv, D).contiguous()
+    dO = si.bf16_randn((1, N, Hq, D), 24)
+    dq, dk, dv = oracle.backward(Q, K, V, dO, B, 2, 1)
+    assert np.abs(dq).max() < 1e-12 and np.abs(dk).max() < 1e-12
+    # column sums of the weights: sum_j dV_j = sum_i dO_i (each row's weights sum to one)
+    assert np.abs(dv[0, :, 0].sum(axis=0) - dO[0].double().numpy().sum(axis=(0, 1))).max() < 1e-9
+    # row 0 attends to key 0 only: o_0 = v_0, so dV_0 gets dO_0 of every head in full
+    Vr = si.bf16_randn((1, N, Hkv, D), 25)
+    dq, dk, dv = oracle.backward(Q, K, Vr, dO, B, 2, 1)
+    assert np.abs(dq[0, 0]).max() < 1e-12            # a one-key softmax has no gradient in its logit
