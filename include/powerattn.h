@@ -203,6 +203,31 @@ pa_status pa_prefill_varlen(const pa_prefill_params *p, const void *q, const voi
 pa_status pa_prefill_status(const void *workspace, void *stream, int32_t *detail);
 
 /* ------------------------------------------------------------------------------------------
+ * Backward of the prefill (the paper trains with its mask, Section 4.1 "Implementation"; it prints no
+ * gradient formulas: these are the derivatives of Eq. (1)).  With P = exp(s - LSE) on the attended
+ * pairs and dO the gradient of the output:
+ *   delta_q = <dO_q, O_q>;   dV_kv = sum_q P dO_q;   dS = P (<dO_q, V_kv> - delta_q);
+ *   dQ_q = softmax_scale sum_kv dS K_kv;   dK_kv = softmax_scale sum_q dS Q_q,
+ * dK and dV summed over the query heads of the KV head's group as well.
+ *
+ * p, q, k, v, row_ptr, col_idx, nnz: as given to pa_prefill (o_dtype must be PA_BF16); o, lse: what
+ * pa_prefill returned; d_o: device bf16 with the strides of o.  dq: device fp32 [batch, seq_len,
+ * n_q_heads, head_dim] contiguous; dk, dv: device fp32 [batch, seq_len, n_kv_heads, head_dim]
+ * contiguous (cleared by the call).  workspace: device, 256-byte aligned,
+ * >= pa_prefill_backward_workspace_bytes(p, nnz) (the row sums delta and the transposed layout).
+ * Two memsets and seven kernels are enqueued.  S and P are recomputed tile by tile on the warp-level
+ * tensor-core MMA (bf16 operands, fp32 accumulation).  A key block that many query blocks list (a
+ * sink block is listed by all) is spread over several CTAs that add their parts with fp32 atomics,
+ * so dk and dv of such blocks may differ in the last bits from run to run.
+ * Errors: as pa_prefill.
+ * ------------------------------------------------------------------------------------------ */
+size_t pa_prefill_backward_workspace_bytes(const pa_prefill_params *p, int64_t nnz);
+pa_status pa_prefill_backward(const pa_prefill_params *p, const void *q, const void *k, const void *v,
+                              const void *o, const float *lse, const void *d_o, const int32_t *row_ptr,
+                              const int32_t *col_idx, int64_t nnz, float *dq, float *dk, float *dv,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
+/* ------------------------------------------------------------------------------------------
  * Decode: one query token per sequence against its KV cache (Section 4.1: the same pattern in
  * prefilling and decoding).  cache_lens[b] counts the cached keys INCLUDING the current token,
  * so the query sits at position p = cache_lens[b] - 1, attends to itself, and its key blocks

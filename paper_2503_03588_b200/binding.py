@@ -24,6 +24,7 @@ EXPORTS = ["pa_status_string", "pa_last_error_message", "pa_version", "pa_reload
            "pa_set_wait_limit_cycles", "pa_layout_size", "pa_build_layout", "pa_window_layout_size",
            "pa_build_window_layout", "pa_reach_counts", "pa_tile_layout_size",
            "pa_build_tile_layout", "pa_prefill_workspace_bytes", "pa_prefill", "pa_prefill_varlen", "pa_prefill_status",
+           "pa_prefill_backward_workspace_bytes", "pa_prefill_backward",
            "pa_decode_workspace_bytes", "pa_decode", "pa_decode_status", "pa_decode_block_list",
            "pa_decode_row_block_set", "pa_decode_paged_workspace_bytes", "pa_decode_paged", "pa_kv_append",
            "pa_decode_static"]
@@ -96,6 +97,11 @@ def _load() -> ctypes.CDLL:
     lib.pa_prefill_varlen.restype = ctypes.c_int
     lib.pa_prefill_varlen.argtypes = [ctypes.POINTER(pa_prefill_params), vp, vp, vp, vp, i64, vp, vp, i64, vp, vp, vp,
                                       ctypes.c_size_t, vp]
+    lib.pa_prefill_backward_workspace_bytes.restype = ctypes.c_size_t
+    lib.pa_prefill_backward_workspace_bytes.argtypes = [ctypes.POINTER(pa_prefill_params), i64]
+    lib.pa_prefill_backward.restype = ctypes.c_int
+    lib.pa_prefill_backward.argtypes = [ctypes.POINTER(pa_prefill_params), vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp,
+                                        vp, vp, ctypes.c_size_t, vp]
     lib.pa_prefill_status.restype = ctypes.c_int
     lib.pa_prefill_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     lib.pa_decode_workspace_bytes.restype = ctypes.c_size_t
@@ -287,6 +293,31 @@ def pa_prefill_varlen(q, k, v, cu_seqlens, max_seq_len: int, row_ptr, col_idx, o
                                  _ptr(row_ptr), _ptr(col_idx), col_idx.numel(), _ptr(o), _ptr(lse), _ptr(workspace),
                                  workspace.numel(), _stream()))
     return o, lse, workspace
+
+
+def pa_prefill_backward(q, k, v, o, lse, d_o, row_ptr, col_idx, dq=None, dk=None, dv=None, workspace=None,
+                        block: int = 64, softmax_scale: float = 0.0):
+    """Gradients of pa_prefill: q, k, v, o (bf16) and lse as in the forward call, d_o bf16 with o's
+    strides.  Returns (dq, dk, dv, workspace), fp32 contiguous, allocated here when not passed in."""
+    batch, seq, hq, d = q.shape
+    hkv = k.shape[2]
+    assert d_o.stride() == o.stride() and o.dtype == torch.bfloat16 and d_o.dtype == torch.bfloat16
+    if dq is None:
+        dq = torch.empty((batch, seq, hq, d), dtype=torch.float32, device=q.device)
+    if dk is None:
+        dk = torch.empty((batch, seq, hkv, d), dtype=torch.float32, device=q.device)
+    if dv is None:
+        dv = torch.empty((batch, seq, hkv, d), dtype=torch.float32, device=q.device)
+    params = prefill_params(q, k, v, o, block, softmax_scale)
+    nnz = col_idx.numel()
+    if workspace is None:
+        workspace = torch.empty(int(lib.pa_prefill_backward_workspace_bytes(ctypes.byref(params), nnz)) + 256,
+                                dtype=torch.uint8, device=q.device)
+    ws_ptr = (workspace.data_ptr() + 255) & ~255
+    _check(lib.pa_prefill_backward(ctypes.byref(params), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o),
+                                   _ptr(row_ptr), _ptr(col_idx), nnz, _ptr(dq), _ptr(dk), _ptr(dv),
+                                   ctypes.c_void_p(ws_ptr), workspace.numel() - (ws_ptr - workspace.data_ptr()), _stream()))
+    return dq, dk, dv, workspace
 
 
 def pa_prefill_status(workspace: torch.Tensor) -> int:

@@ -26,7 +26,7 @@ struct DeviceInfo {
 pa_status current_sm100_device(DeviceInfo *out);
 
 // One-time per-device set-up steps (kernel attributes) are keyed by these slots.
-enum DeviceOnce : int { ONCE_PREFILL_ATTR = 0, ONCE_DECODE_ATTR, ONCE_BACKWARD_ATTR, ONCE_COUNT };
+enum DeviceOnce : int { ONCE_PREFILL_ATTR = 0, ONCE_DECODE_ATTR, ONCE_BACKWARD_ATTR, ONCE_BACKWARD_ATTR_64, ONCE_COUNT };
 // True exactly once per (device, slot); the caller then performs the step and, if it fails, calls
 // device_once_reset so that a later call tries again.
 bool device_once_begin(int device, DeviceOnce slot);
