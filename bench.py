@@ -423,7 +423,26 @@ def run_ours(args):
     prefill_32k = dict(workload=w32.name, active_block_pairs=int(ci32.numel()), ms=ms32,
                        value=flops32 / (ms32 * 1e-3) / 1e12, unit=UNIT,
                        frac=flops32 / (ms32 * 1e-3) / 1e12 / peaks["bf16_tflops"], launches=n32)
-    del Q32, K32, V32, o32, lse32
+    # ---- the backward pass on the same 32K workload (dO drawn on the device; values do not matter
+    # for time): 10 * 64 * 64 * head_dim FLOP per listed block pair and query head (five products).
+    gen32 = torch.Generator(device=dev)
+    gen32.manual_seed(w32.seed + 9)
+    dO32 = torch.randn(o32.shape, device=dev, dtype=torch.bfloat16, generator=gen32)
+    dq32, dk32, dv32, wsb32 = pa.pa_prefill_backward(Q32, K32, V32, o32, lse32, dO32, rp32, ci32)
+    torch.cuda.synchronize()
+    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    nb = 5
+    b0.record(stream)
+    for _ in range(nb):
+        pa.pa_prefill_backward(Q32, K32, V32, o32, lse32, dO32, rp32, ci32, dq=dq32, dk=dk32, dv=dv32, workspace=wsb32)
+    b1.record(stream)
+    torch.cuda.synchronize()
+    msb = b0.elapsed_time(b1) / nb
+    backward_32k = dict(workload=w32.name, ms=msb, value=2.5 * flops32 / (msb * 1e-3) / 1e12, unit=UNIT,
+                        frac=2.5 * flops32 / (msb * 1e-3) / 1e12 / peaks["bf16_tflops"], bound="tensor",
+                        flops_per_pair_head=10 * w32.block * w32.block * w32.head_dim, launches=nb,
+                        kernels="delta, transposed layout (3), dQ, dK/dV: warp-level MMA (mma.sync), fp32 outputs")
+    del Q32, K32, V32, o32, lse32, dO32, dq32, dk32, dv32
 
     # ---- decode scale-up (labelled, beside the batch-8 figure): the same per-sequence pattern at
     # larger batches, where one call moves enough bytes to outlast its launch.  Caches are drawn on
@@ -566,7 +585,7 @@ def run_ours(args):
                               kernel_ms=prefill_ms,
                               frac_of_burst=achieved / peaks["bf16_tflops"],
                               frac_of_sustained=achieved / peaks["bf16_tflops_sustained"]),
-                prefill_32k=prefill_32k,
+                prefill_32k=prefill_32k, backward_32k=backward_32k,
                 decode=dict(metric="decode_kv_gbs", value=dec_gbs, unit="GB/s", us_per_call=dec_us,
                             kv_bytes_per_call=dec_bytes, peak=peaks["hbm_gbs"], frac=dec_gbs / peaks["hbm_gbs"],
                             bound="hbm", timing=f"CUDA graph of {n_sets * reps} calls rotating over {n_sets} seeded length sets",

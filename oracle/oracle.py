@@ -54,7 +54,7 @@ def _load():
                                          _p, ctypes.c_int]
         lib.pa_oracle_backward.restype = None
         lib.pa_oracle_backward.argtypes = [_p, _p, _p, _p, _i64, _i64, _i64, _i64, _i64, ctypes.c_double, _i64, _i64,
-                                           _i64, ctypes.c_int, _p, _p, _p, _p, ctypes.c_int]
+                                           _i64, ctypes.c_int, _p, _p, _i64, _p, _p, _p, ctypes.c_int]
         lib.pa_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -300,10 +300,11 @@ def decode(q, Kc, Vc, lens, B: int, W: int, S: int = 1, scale: Optional[float] =
 
 
 def backward(Q, K, V, dO, B: int, W: int, S: int = 1, scale: Optional[float] = None, use_power: bool = True,
-             dense: Optional[np.ndarray] = None, threads: int = 0):
+             dense: Optional[np.ndarray] = None, threads: int = 0, key_rows: Optional[Sequence[int]] = None):
     """Gradients of Eq. (1) under Algorithm 1's mask (or an explicit dense [N, N] mask) for an
     upstream gradient dO of the output: returns (dQ [batch, N, Hq, D], dK, dV [batch, N, Hkv, D]) fp64.
-    Inputs bf16 as in `prefill`; O(N^2) pair evaluations, for small N."""
+    Inputs bf16 as in `prefill`.  dQ is always computed for every row; `key_rows` restricts dK and dV
+    to those key positions (the other rows stay zero), which keeps long sequences affordable."""
     lib = _load()
     q, k, v, g = _bf16_bits(Q), _bf16_bits(K), _bf16_bits(V), _bf16_bits(dO)
     batch, N, Hq, D = q.shape
@@ -318,6 +319,8 @@ def backward(Q, K, V, dO, B: int, W: int, S: int = 1, scale: Optional[float] = N
     dQ = np.zeros(q.shape, dtype=np.float64)
     dK = np.zeros(k.shape, dtype=np.float64)
     dV = np.zeros(k.shape, dtype=np.float64)
+    kr = None if key_rows is None else np.ascontiguousarray(np.asarray(key_rows, dtype=np.int64))
     lib.pa_oracle_backward(_ptr(q), _ptr(k), _ptr(v), _ptr(g), batch, N, Hq, Hkv, D, float(scale), B, W, S,
-                           int(use_power), _ptr(dm), _ptr(dQ), _ptr(dK), _ptr(dV), int(threads))
+                           int(use_power), _ptr(dm), _ptr(kr), 0 if kr is None else len(kr), _ptr(dQ), _ptr(dK),
+                           _ptr(dV), int(threads))
     return dQ, dK, dV

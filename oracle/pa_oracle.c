@@ -213,12 +213,17 @@ int pa_oracle_max_threads(void)
  * KV head.  Two plain passes, neither with any blocking: rows (dQ, and the per-row log-sum-exp and
  * sum_k p_k dL/dp_k), then keys (dK, dV), each re-evaluating the mask predicate pair by pair.
  * Q, dO [batch, N, Hq, D]; K, V [batch, N, Hkv, D] bf16 bit patterns; outputs fp64, same shapes.
+ * k_rows (n_krows of them; NULL = every key) restricts the second pass to those key positions: the
+ * other rows of dK and dV are left as they are.  The first pass always covers every query row, since
+ * a key's gradient needs the log-sum-exp of every row that attends to it.
  */
 void pa_oracle_backward(const uint16_t *Q, const uint16_t *K, const uint16_t *V, const uint16_t *dO,
                         int64_t batch, int64_t N, int64_t Hq, int64_t Hkv, int64_t D, double scale,
                         int64_t B, int64_t W, int64_t sink_blocks, int use_power,
-                        const uint8_t *dense_mask, double *dQ, double *dK, double *dV, int n_threads)
+                        const uint8_t *dense_mask, const int64_t *k_rows, int64_t n_krows, double *dQ,
+                        double *dK, double *dV, int n_threads)
 {
+    const int64_t n_keys_out = k_rows ? n_krows : N;
     const int64_t G = Hq / Hkv;
     double *lse = (double *)malloc((size_t)(batch * Hq * N) * sizeof(double));
     double *dsum = (double *)malloc((size_t)(batch * Hq * N) * sizeof(double));
@@ -272,8 +277,9 @@ void pa_oracle_backward(const uint16_t *Q, const uint16_t *K, const uint16_t *V,
             dsum[t] = pd;
         }
 #pragma omp for schedule(dynamic, 4)
-        for (int64_t t = 0; t < batch * Hkv * N; ++t) {
-            const int64_t b = t / (Hkv * N), hk = (t / N) % Hkv, j = t % N;
+        for (int64_t t = 0; t < batch * Hkv * n_keys_out; ++t) {
+            const int64_t b = t / (Hkv * n_keys_out), hk = (t / n_keys_out) % Hkv;
+            const int64_t j = k_rows ? k_rows[t % n_keys_out] : t % n_keys_out;
             const uint16_t *k = K + ((b * N + j) * Hkv + hk) * D;
             const uint16_t *v = V + ((b * N + j) * Hkv + hk) * D;
             double *dk = dK + ((b * N + j) * Hkv + hk) * D;

@@ -71,3 +71,24 @@ def test_backward_sink_column_spread_over_many_ctas(pa, oracle):
 
 def test_backward_sliding_window_layout(pa, oracle):
     _run(pa, oracle, 1100, 8, 2, 128, 4, 1, use_power=False, seed=6)
+
+
+def test_backward_at_16k_on_sampled_keys(pa, oracle):
+    """A sweep-sized case: 16K tokens with the 7B-like heads.  The oracle evaluates dQ on every row
+    (its first pass covers them all anyway) and dK, dV on sampled key positions: the sink block (its
+    column is spread over eight CTAs), block boundaries, power-of-two distances and a random draw."""
+    N, Hq, Hkv, D, W, S = 16384, 28, 4, 128, 5, 1
+    Q, K, V = si.bf16_randn((1, N, Hq, D), 1101), si.bf16_randn((1, N, Hkv, D), 1102), si.bf16_randn((1, N, Hkv, D), 1103)
+    dO = si.bf16_randn((1, N, Hq, D), 1104)
+    rp, ci = pa.pa_build_layout(N, 64, W, S)
+    Qd, Kd, Vd, dOd = Q.cuda(), K.cuda(), V.cuda(), dO.cuda()
+    o, lse, ws = pa.pa_prefill(Qd, Kd, Vd, rp, ci)
+    pa.pa_prefill_status(ws)
+    dq, dk, dv, _ = pa.pa_prefill_backward(Qd, Kd, Vd, o, lse, dOd, rp, ci)
+    torch.cuda.synchronize()
+    keys = sorted({0, 1, 63, 64, 65, N - 1, N - 64, N - 65, 8191, 8192, 12288 + 17}
+                  | {int(x) for x in np.random.default_rng(1105).integers(0, N, 24)})
+    rq, rk, rv = oracle.backward(Q, K, V, dO, 64, W, S, key_rows=keys)
+    kidx = torch.as_tensor(keys).cuda()
+    print("16K backward (max, mean):", _compare(dq, rq, "dQ 16K"), _compare(dk[:, kidx], rk[:, keys], "dK 16K"),
+          _compare(dv[:, kidx], rv[:, keys], "dV 16K"))

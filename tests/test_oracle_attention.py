@@ -246,3 +246,18 @@ def test_backward_closed_forms(oracle):
     Vr = si.bf16_randn((1, N, Hkv, D), 25)
     dq, dk, dv = oracle.backward(Q, K, Vr, dO, B, 2, 1)
     assert np.abs(dq[0, 0]).max() < 1e-12            # a one-key softmax has no gradient in its logit
+
+
+def test_backward_key_subset_equals_the_full_pass(oracle):
+    import synth_inputs as si
+
+    N, Hq, Hkv, D = 150, 4, 2, 16
+    Q, K, V = si.bf16_randn((1, N, Hq, D), 31), si.bf16_randn((1, N, Hkv, D), 32), si.bf16_randn((1, N, Hkv, D), 33)
+    dO = si.bf16_randn((1, N, Hq, D), 34)
+    dq, dk, dv = oracle.backward(Q, K, V, dO, 8, 2, 1)
+    keys = [0, 7, 8, 77, 149]
+    dq2, dk2, dv2 = oracle.backward(Q, K, V, dO, 8, 2, 1, key_rows=keys)
+    assert np.array_equal(dq, dq2)
+    assert np.array_equal(dk[:, keys], dk2[:, keys]) and np.array_equal(dv[:, keys], dv2[:, keys])
+    rest = np.setdiff1d(np.arange(N), keys)
+    assert not dk2[:, rest].any() and not dv2[:, rest].any()
