@@ -238,6 +238,17 @@ def run_ours(args):
     Q, K, V = Qh.to(dev), Kh.to(dev), Vh.to(dev)
     nqb, nnz = pa.pa_layout_size(w.seq_len, w.block, w.window_blocks, w.sink_blocks)
     flops = block_pair_flops(nnz, w)
+    if args.shard_heads and world > 1:
+        # Strong scaling without an exchange step: each rank takes whole KV heads and their query
+        # heads of the same problem (at most n_kv_heads ranks have work).
+        from paper_2503_03588_b200.sharding import shard_prefill_tensors
+
+        part = shard_prefill_tensors(Q, K, V, world, rank)
+        if part is None:
+            Q, K, V, flops = Q[:, :, :7], K[:, :, :1], V[:, :, :1], 0.0   # an idle rank repeats rank 0's slice, uncounted
+        else:
+            Q, K, V, _ = part
+            flops *= Q.shape[2] / w.n_q_heads
     row_ptr = torch.empty(nqb + 1, dtype=torch.int32, device=dev)
     col_idx = torch.empty(nnz, dtype=torch.int32, device=dev)
     O = torch.empty_like(Q)
@@ -571,13 +582,14 @@ def run_ours(args):
     peak = peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"]
     peak_kind = " sustained bf16 (power-capped clocks in the timed region)" if capped else " burst bf16"
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
-                ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                ms_per_step=ms, higher_is_better=True,
+                scaling="strong" if (args.shard_heads and world > 1) else "weak", vs_baseline=None, dtype="bf16",
                 data="synthetic",
                 config=dict(workload=w.name, seq_len=w.seq_len, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads,
                             head_dim=w.head_dim, block=w.block, window_blocks=w.window_blocks,
                             sink_blocks=w.sink_blocks, active_block_pairs=nnz, step="layout+prefill+decode",
                             decode_workload=wd.name, l2="inputs larger than L2 (Q+K+V+O = 2.4 GB per step)",
-                            parallelism="replicas" if world > 1 else "single"),
+                            parallelism=("kv_head_shards" if args.shard_heads else "replicas") if world > 1 else "single"),
                 clocks=clocks,
                 roofline=dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s",
                               frac=achieved / peak, traffic=prefill_traffic(),
@@ -743,6 +755,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--shard-heads", action="store_true",
+                    help="with N > 1: split the one problem by KV heads over the ranks (strong scaling) instead of replicas")
     ap.add_argument("--no-decode-scale-up", action="store_true", help="skip the batch-64/256 decode lines")
     ap.add_argument("--case", default=None, choices=["prefill32k", "decode", "decode_persist"],
                     help="run only a small single-kernel case (for profiler captures)")

@@ -443,3 +443,25 @@ def test_a_wait_that_runs_out_ends_the_kernel_with_a_status(pa, oracle):
     assert pa.pa_prefill_status(ws) == 0
     o_ref, lse_ref, _ = oracle.prefill(Q, K, V, 64, 64, 0, use_power=False)
     compare(o, lse, o_ref, lse_ref, "after a timed-out call")
+
+
+def test_kv_head_shards_reproduce_the_whole_call(pa):
+    """Head sharding needs no exchange: the ranks' calls on head slices (run here one after the
+    other on the one GPU; they do not depend on each other) write disjoint slices of O and LSE that
+    agree bit for bit with the unsharded call."""
+    from paper_2503_03588_b200.sharding import shard_prefill_tensors
+
+    N, Hq, Hkv, D = 3000, 28, 4, 128
+    Q, K, V = (si.bf16_randn((1, N, h, D), 860 + i).cuda() for i, h in enumerate((Hq, Hkv, Hkv)))
+    rp, ci = pa.pa_build_layout(N, 64, 5, 1)
+    o_full, lse_full, ws = pa.pa_prefill(Q, K, V, rp, ci)
+    pa.pa_prefill_status(ws)
+    for world in (2, 3, 4):
+        o = torch.zeros_like(o_full)
+        lse = torch.zeros_like(lse_full)
+        for rank in range(world):
+            qs_, ks_, vs_, heads = shard_prefill_tensors(Q, K, V, world, rank)
+            o_r, lse_r, ws_r = pa.pa_prefill(qs_, ks_, vs_, rp, ci, o=o[:, :, heads])
+            pa.pa_prefill_status(ws_r)
+            lse[:, heads] = lse_r
+        assert torch.equal(o, o_full) and torch.equal(lse, lse_full), world
