@@ -235,24 +235,27 @@ def run_ours(args):
 
     w, wd = si.PREFILL_128K, si.DECODE_B8
     Qh, Kh, Vh = si.prefill_inputs(w, pin=True)
-    Q, K, V = Qh.to(dev), Kh.to(dev), Vh.to(dev)
     nqb, nnz = pa.pa_layout_size(w.seq_len, w.block, w.window_blocks, w.sink_blocks)
     flops = block_pair_flops(nnz, w)
+    n_heads_local = w.n_q_heads
     if args.shard_heads and world > 1:
         # Strong scaling without an exchange step: each rank takes whole KV heads and their query
-        # heads of the same problem (at most n_kv_heads ranks have work).
-        from paper_2503_03588_b200.sharding import shard_prefill_tensors
+        # heads of the same problem (at most n_kv_heads ranks have work; an idle rank repeats rank
+        # 0's first group, uncounted).
+        from paper_2503_03588_b200.sharding import kv_head_shard
 
-        part = shard_prefill_tensors(Q, K, V, world, rank)
-        if part is None:
-            Q, K, V, flops = Q[:, :, :7], K[:, :, :1], V[:, :, :1], 0.0   # an idle rank repeats rank 0's slice, uncounted
-        else:
-            Q, K, V, _ = part
-            flops *= Q.shape[2] / w.n_q_heads
+        qs, ks = kv_head_shard(w.n_q_heads, w.n_kv_heads, world, rank)
+        if ks.start == ks.stop:
+            qs, ks, flops = slice(0, w.n_q_heads // w.n_kv_heads), slice(0, 1), 0.0
+        Qh, Kh, Vh = (t.contiguous().pin_memory() for t in (Qh[:, :, qs], Kh[:, :, ks], Vh[:, :, ks]))
+        n_heads_local = qs.stop - qs.start
+        if flops:
+            flops *= n_heads_local / w.n_q_heads
+    Q, K, V = Qh.to(dev), Kh.to(dev), Vh.to(dev)
     row_ptr = torch.empty(nqb + 1, dtype=torch.int32, device=dev)
     col_idx = torch.empty(nnz, dtype=torch.int32, device=dev)
     O = torch.empty_like(Q)
-    LSE = torch.empty((w.batch, w.n_q_heads, w.seq_len), dtype=torch.float32, device=dev)
+    LSE = torch.empty((w.batch, n_heads_local, w.seq_len), dtype=torch.float32, device=dev)
     ws = torch.empty(4096, dtype=torch.uint8, device=dev)
 
     qd_h, kc_h, vc_h, lens = si.decode_inputs(wd)
