@@ -268,8 +268,8 @@ size_t pa_decode_workspace_bytes(const pa_decode_params *p);
  * Calls that share a workspace must not overlap on the GPU.  Environment switches (for tests and
  * measurements, see pa_reload_environment): PA_DECODE_PATH=splitk forces the two-kernel path,
  * =cluster / =persist the two forms of the row kernel; PA_DECODE_CLUSTER=n (1..8) sets R (default:
- * for small calls enough CTAs to fill the GPU about three times, for large ones the smallest
- * split that loads the SMs evenly); PA_DECODE_STAGES=n (1..6) the number of key blocks a CTA keeps
+ * for small calls as many CTAs per row as run all at once, for large ones one chunk per row once
+ * there are as many rows as SMs, else two); PA_DECODE_STAGES=n (1..6) the number of key blocks a CTA keeps
  * in flight. */
 pa_status pa_decode(const pa_decode_params *p, const void *q, const void *k_cache,
                     const void *v_cache, const int32_t *cache_lens, void *o, float *lse,

@@ -1003,8 +1003,7 @@ static pa_status launch_decode(const DecodeShape &p, const void *q, const void *
         const int64_t rows_in_call = (int64_t)a.batch * a.Hkv;
         const int max_R = a.chunks < kRowMaxCluster ? a.chunks : kRowMaxCluster;
         const int64_t persistent_ctas = (env.decode_ctas_per_sm ? env.decode_ctas_per_sm : 2) * (int64_t)dev.sms;
-        // Small calls (latency-bound): one launch, a cluster of R CTAs per row, enough CTAs to
-        // fill the GPU about three times over.  Larger calls (bandwidth-bound): a persistent grid of
+        // Small calls (latency-bound): one launch, a cluster of R CTAs per row, all resident at once.  Larger calls (bandwidth-bound): a persistent grid of
         // two CTAs per SM over (row, chunk) items.
         bool cluster = rows_in_call * kRowMaxCluster <= 2 * persistent_ctas;
         if (env.decode_path == 2) cluster = true;
@@ -1012,7 +1011,9 @@ static pa_status launch_decode(const DecodeShape &p, const void *q, const void *
         int R = env.decode_cluster;
         if (cluster) {
             if (R == 0) {
-                R = (int)((3 * (int64_t)dev.sms + rows_in_call - 1) / rows_in_call);
+                // as many CTAs per row as still run all at once (two CTAs fit an SM): a second wave
+                // of clusters doubles the call's latency (batch 16: 17.4 us with R = 8, 12.5 with R = 4)
+                R = (int)(persistent_ctas / rows_in_call);
                 if (R < 1) R = 1;
             }
             if (R > max_R) R = max_R;
@@ -1028,9 +1029,10 @@ static pa_status launch_decode(const DecodeShape &p, const void *q, const void *
         a.items = rows_in_call * R;
         const int64_t grid = a.mode == kModeCluster ? a.items : (a.items < persistent_ctas ? a.items : persistent_ctas);
         if (a.items > 0x3fffffff) return fail(PA_ERR_SHAPE, "too many work items (%lld)", (long long)a.items);
-        // Stages: as many as two CTAs per SM leave room for, and no more than a CTA has blocks.
+        // Stages: 64 KB of blocks in flight per CTA, and no more than a CTA has blocks.
         const int64_t blocks_per_cta = ((int64_t)a.chunks * rows_in_call + grid - 1) / grid;
-        const int fit = p.head_dim == 128 ? 3 : 6;
+        // (two stages measured 1-3 % faster than three at batch 64 and 256, head_dim 128)
+        const int fit = p.head_dim == 128 ? 2 : 4;
         a.stages = env.decode_stages != 0 ? env.decode_stages : fit;
         if (a.stages > kRowMaxStages) a.stages = kRowMaxStages;
         if (a.stages > blocks_per_cta) a.stages = (int)blocks_per_cta;
