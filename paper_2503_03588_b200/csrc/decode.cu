@@ -318,8 +318,9 @@ __global__ void __launch_bounds__(D) decode_combine_kernel(const DecodeArgs a)
 //               warp a quarter of the features.
 // What happens to an item's result depends on the launch (DecodeArgs::mode):
 //   kModeCluster  small calls.  One item per CTA, the R CTAs of a row form a thread-block
-//                 cluster: after a cluster barrier CTA r merges heads r, r + R, ... reading its
-//                 peers through distributed shared memory, and writes O and LSE.  One launch.
+//                 cluster: each CTA stores its part of head h into the shared memory of CTA h % R
+//                 (distributed shared memory), and after one cluster barrier that CTA merges the
+//                 head and writes O and LSE.  One launch.
 //   kModePartial  larger calls.  A persistent grid of two CTAs per SM strides over the items;
 //                 each item's (o, m, l) goes to the workspace and decode_combine_kernel merges a
 //                 row's R chunks (second launch, programmatic dependent launch).
@@ -343,11 +344,15 @@ struct RowSmem {
     // (three quarters of the D features) and its running maximum and sum.
     static constexpr uint32_t kPartRow = D - D / 4 + 2;
     static constexpr uint32_t kPart = kRowConsumers * kMaxGroup * kPartRow * 4;
+    // (cluster form) what the row's CTAs send to the CTA that merges a head: per sending CTA and head
+    // slot, o[D], m, l.  R senders x ceil(8 / R) heads of an owner is at most 14 entries (R = 7).
+    static constexpr uint32_t kRecvEntries = 14;
+    static constexpr uint32_t kRecv = kRecvEntries * (D + 2) * 4;
     static constexpr uint32_t kBars = 3 * kRowMaxStages * 8 + 16;
-    // In cluster mode the CTA's merged result (o[heads][D], then m and l per head) is kept for its
-    // peers over stage 0, which nothing reads any more by then.
-    static_assert(kMaxGroup * (D + 2) * 4 <= kStage, "a CTA's result must fit one stage");
-    static constexpr size_t bytes(int stages) { return 1024 + (size_t)stages * kStage + kPart + kBars; }
+    static constexpr size_t bytes(int stages, bool cluster)
+    {
+        return 1024 + (size_t)stages * kStage + kPart + kBars + (cluster ? kRecv : 0);
+    }
 };
 
 // The row's block set, one candidate per lane (the order does not matter for Eq. (1), so the set
@@ -387,8 +392,8 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
     const int stages = a.stages;
     const uint32_t off_part = (uint32_t)stages * SM::kStage;
     float *part = reinterpret_cast<float *>(smem + off_part);  // [warp][head][kPartRow]
-    float *sO = reinterpret_cast<float *>(smem);               // (cluster mode) [kMaxGroup][D] over stage 0
-    float *sML = sO + kMaxGroup * D;                           // (cluster mode) [kMaxGroup][2]
+    // (cluster form) receive area behind the barriers: [sender][head slot][D + 2]
+    float *recv = reinterpret_cast<float *>(smem + off_part + SM::kPart + SM::kBars);
     const uint32_t bars = smem_base + off_part + SM::kPart;
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + off_part + SM::kPart + 3 * kRowMaxStages * 8);
     auto bar_kfull = [&](int s) { return bars + (uint32_t)s * 8u; };
@@ -687,12 +692,22 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
                 const int64_t head = ((int64_t)w.b * a.Hq + (int64_t)w.hk * G + g);
                 const int f0 = wid * (D / 4) + 2 * t;
                 if (a.mode == kModeCluster) {
+                    // Head g is merged by CTA g % R of the cluster: this CTA's part goes straight into
+                    // that CTA's receive area (a store through distributed shared memory; the area is
+                    // not used for anything else, so the owner may still be busy with its blocks).
+                    if (g < G) {
+                        namespace cg = cooperative_groups;
+                        cg::cluster_group cluster = cg::this_cluster();
+                        const int owner = g % R, slot = g / R, heads_per_owner = (kMaxGroup + R - 1) / R;
+                        float *dst = (R > 1 ? cluster.map_shared_rank(recv, owner) : recv) +
+                                     ((size_t)w.r * heads_per_owner + slot) * (D + 2);
 #pragma unroll
-                    for (int y = 0; y < D / 32; ++y)
-                        *reinterpret_cast<float2 *>(sO + g * D + f0 + 8 * y) = make_float2(fin[y][0], fin[y][1]);
-                    if (wid == 0 && t == 0) {
-                        sML[2 * g] = m;
-                        sML[2 * g + 1] = l;
+                        for (int y = 0; y < D / 32; ++y)
+                            *reinterpret_cast<float2 *>(dst + f0 + 8 * y) = make_float2(fin[y][0], fin[y][1]);
+                        if (wid == 0 && t == 0) {
+                            dst[D] = m;
+                            dst[D + 1] = l;
+                        }
                     }
                 } else if (g < G) {
                     if (a.mode == kModePartial) {
@@ -728,30 +743,25 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
     }
 
     if (a.mode == kModeCluster) {
-        // ---- merge across the cluster: CTA r takes heads r, r + R, ...; thread d one feature.  All
-        // remote reads of a head are issued before the first one is used (they are independent, and
-        // each costs a trip through the cluster's shared-memory network).
+        // ---- merge across the cluster: every CTA has pushed its parts; after one cluster barrier CTA r
+        // merges heads r, r + R, ... from its own receive area (thread d one feature) and writes O
+        // and LSE.  Nothing reads a peer's shared memory after the barrier, so no second one is needed.
+        namespace cg = cooperative_groups;
         cg::cluster_group cluster = cg::this_cluster();
         const int r = (int)(blockIdx.x % (unsigned)R);
         const int32_t rowid = (int32_t)(blockIdx.x / (unsigned)R);
+        const int heads_per_owner = (kMaxGroup + R - 1) / R;
         if (R > 1) cluster.sync();
         else __syncthreads();
         if (tid < D) {
-            const float *peer_ml[kRowMaxCluster];
-            const float *peer_o[kRowMaxCluster];
-#pragma unroll
-            for (int rr = 0; rr < kRowMaxCluster; ++rr) {
-                const int src = rr < R ? rr : r;  // (slots beyond the cluster are given weight 0 below)
-                peer_ml[rr] = R > 1 ? cluster.map_shared_rank(sML, src) : sML;
-                peer_o[rr] = R > 1 ? cluster.map_shared_rank(sO, src) : sO;
-            }
-            for (int h = r; h < G; h += R) {
+            for (int h = r, slot = 0; h < G; h += R, ++slot) {
                 float mr[kRowMaxCluster], lr[kRowMaxCluster], orr[kRowMaxCluster];
 #pragma unroll
                 for (int rr = 0; rr < kRowMaxCluster; ++rr) {
-                    mr[rr] = peer_ml[rr][2 * h];
-                    lr[rr] = peer_ml[rr][2 * h + 1];
-                    orr[rr] = peer_o[rr][h * D + tid];
+                    const float *src = recv + ((size_t)(rr < R ? rr : 0) * heads_per_owner + slot) * (D + 2);
+                    mr[rr] = src[D];
+                    lr[rr] = src[D + 1];
+                    orr[rr] = src[tid];
                 }
                 float m = -INFINITY;
 #pragma unroll
@@ -774,7 +784,6 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
                 if (tid == 0) a.lse[(int64_t)rowid * G + h] = any ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
             }
         }
-        if (R > 1) cluster.sync();  // peers may still be reading this CTA's shared memory
     }
     __syncthreads();
     if (*abort_flag && tid == 0) {
@@ -1050,9 +1059,9 @@ static pa_status launch_decode(const DecodeShape &p, const void *q, const void *
 
         if (device_once_begin(dev.device, ONCE_DECODE_ATTR)) {
             const cudaError_t e1 = cudaFuncSetAttribute(decode_row_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                        (int)RowSmem<128>::bytes(kRowMaxStages));
+                                                        (int)RowSmem<128>::bytes(kRowMaxStages, true));
             const cudaError_t e2 = cudaFuncSetAttribute(decode_row_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                        (int)RowSmem<64>::bytes(kRowMaxStages));
+                                                        (int)RowSmem<64>::bytes(kRowMaxStages, true));
             if (e1 != cudaSuccess || e2 != cudaSuccess) {
                 device_once_reset(dev.device, ONCE_DECODE_ATTR);
                 return fail(PA_ERR_CUDA, "cudaFuncSetAttribute failed: %s",
@@ -1075,10 +1084,10 @@ static pa_status launch_decode(const DecodeShape &p, const void *q, const void *
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         if (p.head_dim == 128) {
-            cfg.dynamicSmemBytes = RowSmem<128>::bytes(a.stages);
+            cfg.dynamicSmemBytes = RowSmem<128>::bytes(a.stages, a.mode == kModeCluster);
             PA_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_row_kernel<128>, tmK, tmV, a));
         } else {
-            cfg.dynamicSmemBytes = RowSmem<64>::bytes(a.stages);
+            cfg.dynamicSmemBytes = RowSmem<64>::bytes(a.stages, a.mode == kModeCluster);
             PA_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_row_kernel<64>, tmK, tmV, a));
         }
         if (a.mode != kModePartial) return PA_OK;
