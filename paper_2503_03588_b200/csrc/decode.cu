@@ -332,6 +332,7 @@ constexpr int kRowConsumers = 4;                     // consumer warps
 constexpr int kRowThreads = 32 * (kRowConsumers + 1);
 constexpr int kRowMaxStages = 6;                     // shared-memory stages (key blocks in flight) per CTA
 constexpr int kRowMaxCluster = 8;                    // portable cluster size limit
+constexpr int kRowMaxSmem = 227 * 1024;              // dynamic shared memory a CTA may ask for
 constexpr long long kRowWaitCycles = 2000000000ll;   // default limit of a barrier wait: ~1 s
 enum : int32_t { kModeCluster = 0, kModePartial = 1, kModeDirect = 2 };
 
@@ -1046,6 +1047,9 @@ static pa_status launch_decode(const DecodeShape &p, const void *q, const void *
         if (a.stages > kRowMaxStages) a.stages = kRowMaxStages;
         if (a.stages > blocks_per_cta) a.stages = (int)blocks_per_cta;
         if (a.stages < 1) a.stages = 1;
+        while (a.stages > 1 && (p.head_dim == 128 ? RowSmem<128>::bytes(a.stages, a.mode == kModeCluster)
+                                                  : RowSmem<64>::bytes(a.stages, a.mode == kModeCluster)) > (size_t)kRowMaxSmem)
+            --a.stages;
 
         // Tensor maps over the cache: (feature, token, head, batch or page), one 64 x 64 box per copy.
         CUtensorMap tmK, tmV;
@@ -1059,9 +1063,9 @@ static pa_status launch_decode(const DecodeShape &p, const void *q, const void *
 
         if (device_once_begin(dev.device, ONCE_DECODE_ATTR)) {
             const cudaError_t e1 = cudaFuncSetAttribute(decode_row_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                        (int)RowSmem<128>::bytes(kRowMaxStages, true));
+                                                        kRowMaxSmem);
             const cudaError_t e2 = cudaFuncSetAttribute(decode_row_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                        (int)RowSmem<64>::bytes(kRowMaxStages, true));
+                                                        kRowMaxSmem);
             if (e1 != cudaSuccess || e2 != cudaSuccess) {
                 device_once_reset(dev.device, ONCE_DECODE_ATTR);
                 return fail(PA_ERR_CUDA, "cudaFuncSetAttribute failed: %s",
