@@ -347,6 +347,25 @@ def run_ours(args):
     dec_us = 1e3 * d0.elapsed_time(d1) / (n_sets * reps)
     dec_gbs = dec_bytes / (dec_us * 1e-6) / 1e9
 
+    # ---- what a kernel launch costs in such a graph: 128 launches of a one-element library kernel,
+    # timed the same way (the decode call's time is several of these, so launch latency is not its floor).
+    tiny = torch.zeros(1, device=dev)
+    with torch.cuda.stream(side):
+        tiny.add_(1.0)
+        torch.cuda.synchronize()
+        gf = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gf, stream=side):
+            for _ in range(n_sets * reps):
+                tiny.add_(1.0)
+        gf.replay()
+        torch.cuda.synchronize()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(side)
+        gf.replay()
+        f1.record(side)
+        torch.cuda.synchronize()
+    floor_us = 1e3 * f0.elapsed_time(f1) / (n_sets * reps)
+
     # ---- the same calls issued eagerly (no graph): device time per call and the host's time to
     # enqueue one (argument checks, cached tensor maps, the launch), which a graph replay hides.
     def eager(fn, n):
@@ -603,6 +622,7 @@ def run_ours(args):
                 prefill_32k=prefill_32k, backward_32k=backward_32k,
                 decode=dict(metric="decode_kv_gbs", value=dec_gbs, unit="GB/s", us_per_call=dec_us,
                             kv_bytes_per_call=dec_bytes, peak=peaks["hbm_gbs"], frac=dec_gbs / peaks["hbm_gbs"],
+                            launch_floor_us=floor_us,
                             bound="hbm", timing=f"CUDA graph of {n_sets * reps} calls rotating over {n_sets} seeded length sets",
                             workload=wd.name, scale_up=scale_up, eager=eager_decode, many_steps=decode_many),
                 eager_prefill=eager_prefill, parity=parity,
