@@ -137,12 +137,14 @@ __device__ __forceinline__ Unit decode_unit(const PrefillArgs &a, uint32_t u)
 {
     Unit r;
     uint32_t rem;
+    // Order: head quad fastest, then query block (long rows first), then KV head, then batch entry:
+    // the CTAs work on one KV head at a time, whose K and V (67 MB at 128K tokens) stay in L2.
     u = divmod(u, (uint32_t)a.nsub, a.inv_nsub, rem);
     r.sub = (int32_t)rem;
-    u = divmod(u, (uint32_t)a.Hkv, a.inv_Hkv, rem);
-    r.hk = (int32_t)rem;
-    r.b = (int32_t)divmod(u, (uint32_t)a.nqb, a.inv_nqb, rem);
+    u = divmod(u, (uint32_t)a.nqb, a.inv_nqb, rem);
     r.i = a.nqb - 1 - (int32_t)rem;  // long rows first
+    r.b = (int32_t)divmod(u, (uint32_t)a.Hkv, a.inv_Hkv, rem);
+    r.hk = (int32_t)rem;
     r.rs = __ldg(a.row_ptr + r.i);
     r.n = __ldg(a.row_ptr + r.i + 1) - r.rs;
     if (a.cu_seqlens) {
