@@ -56,26 +56,36 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// delta[b, h, t] = sum_d dO[b, t, h, d] O[b, t, h, d]; one warp per (token, head) row.
+// delta[b, h, t] = sum_d dO[b, t, h, d] O[b, t, h, d]; D / 8 lanes per (token, head) row, 16 bytes per lane.
 template <int D>
 __global__ void backward_delta_kernel(const BackwardArgs a)
 {
-    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
+    constexpr int kLanes = D / 8;              // lanes that share a row
+    constexpr int kRowsPerWarp = 32 / kLanes;
+    const int lane = threadIdx.x & 31, sub = lane % kLanes;
+    const int64_t row = ((int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * kRowsPerWarp + lane / kLanes;
     const int64_t rows = (int64_t)a.batch * a.N * a.Hq;
-    if (row >= rows) return;
-    const int h = (int)(row % a.Hq);
-    const int64_t t = (row / a.Hq) % a.N, b = row / ((int64_t)a.Hq * a.N);
-    const __nv_bfloat16 *po = a.o + b * a.o_sb + t * a.o_ss + (int64_t)h * a.o_sh;
-    const __nv_bfloat16 *pg = a.d_o + b * a.o_sb + t * a.o_ss + (int64_t)h * a.o_sh;
     float acc = 0.f;
-    for (int d = 2 * lane; d < D; d += 64) {
-        const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(po + d));
-        const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(pg + d));
-        acc += x.x * y.x + x.y * y.y;
+    int h = 0;
+    int64_t t = 0, b = 0;
+    if (row < rows) {
+        h = (int)(row % a.Hq);
+        t = (row / a.Hq) % a.N;
+        b = row / ((int64_t)a.Hq * a.N);
+        const int64_t off = b * a.o_sb + t * a.o_ss + (int64_t)h * a.o_sh + 8 * sub;
+        const uint4 x = *reinterpret_cast<const uint4 *>(a.o + off);
+        const uint4 y = *reinterpret_cast<const uint4 *>(a.d_o + off);
+        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 xf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&xs[e]));
+            const float2 yf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ys[e]));
+            acc += xf.x * yf.x + xf.y * yf.y;
+        }
     }
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) a.delta[(b * a.Hq + h) * a.N + t] = acc;
+#pragma unroll
+    for (int o = kLanes / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (row < rows && sub == 0) a.delta[(b * a.Hq + h) * a.N + t] = acc;
 }
 
 // Does row i of the CSR list block j?  (rows are ascending: binary search)
@@ -231,12 +241,11 @@ __device__ __forceinline__ void pack_a(const float (&x)[8][4], uint32_t (&w)[4][
 
 // dQ: one CTA per (query block, query head); warp w owns query rows 16 w .. 16 w + 15.
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads) backward_dq_kernel(const BackwardArgs a)
+__global__ void __launch_bounds__(kBwdThreads, 3) backward_dq_kernel(const BackwardArgs a)
 {
     using T = BwdTile<D>;
     extern __shared__ __align__(16) uint8_t bwd_smem[];
-    // Q and dO tiles of the row, then two (K, V) buffers: the next key block loads while this one is worked on.
-    const uint32_t sQ = ptx::smem_u32(bwd_smem), sG = sQ + T::kBytes, sKV = sG + T::kBytes;
+    const uint32_t sQ = ptx::smem_u32(bwd_smem), sG = sQ + T::kBytes, sK = sG + T::kBytes, sV = sK + T::kBytes;
     const int i = a.nqb - 1 - (int)blockIdx.x, h = blockIdx.y, b = blockIdx.z, hk = h / a.G;  // long rows first
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, g = lane >> 2, t = lane & 3;
     const int r0 = 16 * wid;
@@ -259,24 +268,13 @@ __global__ void __launch_bounds__(kBwdThreads) backward_dq_kernel(const Backward
 
     const __nv_bfloat16 *kbase = a.k + b * a.k_sb + (int64_t)hk * a.k_sh;
     const __nv_bfloat16 *vbase = a.v + b * a.v_sb + (int64_t)hk * a.v_sh;
-    auto load_kv = [&](int32_t e) {
-        const int32_t jj = a.col_idx[e];
-        const uint32_t dst = sKV + (uint32_t)((e - e0) & 1) * 2u * T::kBytes;
-        load_tile<D>(dst, kbase, a.k_ss, (int64_t)jj * kBwdBlk, a.N, tid);
-        load_tile<D>(dst + T::kBytes, vbase, a.v_ss, (int64_t)jj * kBwdBlk, a.N, tid);
-        asm volatile("cp.async.commit_group;\n" ::: "memory");
-    };
-    if (e0 < e1) load_kv(e0);
     for (int32_t e = e0; e < e1; ++e) {
         const int32_t j = a.col_idx[e];
-        const uint32_t sK = sKV + (uint32_t)((e - e0) & 1) * 2u * T::kBytes, sV = sK + T::kBytes;
-        if (e + 1 < e1) {
-            load_kv(e + 1);  // (its buffer was released by the barrier that closed step e - 1)
-            asm volatile("cp.async.wait_group 1;\n" ::: "memory");
-        } else {
-            asm volatile("cp.async.wait_group 0;\n" ::: "memory");
-        }
-        __syncthreads();  // this step's tiles (and, first time, Q and dO) are in shared memory for every warp
+        __syncthreads();  // every warp has finished with the previous K and V tiles
+        load_tile<D>(sK, kbase, a.k_ss, (int64_t)j * kBwdBlk, a.N, tid);
+        load_tile<D>(sV, vbase, a.v_ss, (int64_t)j * kBwdBlk, a.N, tid);
+        asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
+        __syncthreads();
         float s[8][4], dp[8][4];
         tile_product<D>(sQ, r0, sK, lane, s);   // S = Q K^T
         tile_product<D>(sG, r0, sV, lane, dp);  // dP = dO V^T
@@ -293,7 +291,6 @@ __global__ void __launch_bounds__(kBwdThreads) backward_dq_kernel(const Backward
         uint32_t w[4][4];
         pack_a(s, w);
         tile_accumulate<D>(w, sK, lane, dq);  // dQ += dS K
-        __syncthreads();  // every warp has finished with this buffer
     }
 #pragma unroll
     for (int x = 0; x < 2; ++x) {
@@ -313,9 +310,9 @@ __global__ void __launch_bounds__(kBwdThreads) backward_dkv_kernel(const Backwar
 {
     using T = BwdTile<D>;
     extern __shared__ __align__(16) uint8_t bwd_smem[];
-    // K and V tiles of the column, then two (Q, dO) buffers with their row statistics.
-    const uint32_t sK = ptx::smem_u32(bwd_smem), sV = sK + T::kBytes, sQG = sV + T::kBytes;
-    float *s_stat = reinterpret_cast<float *>(bwd_smem + 6 * T::kBytes);  // [buffer][lse2 | delta][64]
+    const uint32_t sK = ptx::smem_u32(bwd_smem), sV = sK + T::kBytes, sQ = sV + T::kBytes, sG = sQ + T::kBytes;
+    float *s_lse2 = reinterpret_cast<float *>(bwd_smem + 4 * T::kBytes);  // [64] per query of the tile
+    float *s_delta = s_lse2 + kBwdBlk;
     const int32_t c = blockIdx.x;
     const int hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, g = lane >> 2, t = lane & 3;
@@ -340,36 +337,22 @@ __global__ void __launch_bounds__(kBwdThreads) backward_dkv_kernel(const Backwar
         dk[e][0] = dk[e][1] = dk[e][2] = dk[e][3] = 0.f;
         dv[e][0] = dv[e][1] = dv[e][2] = dv[e][3] = 0.f;
     }
-    // The chunk is walked once per query head of the group: step number n -> (head, query block).
-    const int32_t per_head = e1 - e0, n_steps = per_head * a.G;
-    auto load_qg = [&](int32_t n) {
-        const int h = hk * a.G + n / per_head;
-        const int32_t ii = a.row_idx[e0 + n % per_head];
-        const uint32_t dst = sQG + (uint32_t)(n & 1) * 2u * T::kBytes;
-        load_tile<D>(dst, a.q + b * a.q_sb + (int64_t)h * a.q_sh, a.q_ss, (int64_t)ii * kBwdBlk, a.N, tid);
-        load_tile<D>(dst + T::kBytes, a.d_o + b * a.o_sb + (int64_t)h * a.o_sh, a.o_ss, (int64_t)ii * kBwdBlk, a.N, tid);
-        if (tid < kBwdBlk) {
-            const int64_t q = (int64_t)ii * kBwdBlk + tid;
-            const float lse = q < a.N ? a.lse[((int64_t)b * a.Hq + h) * a.N + q] : INFINITY;
-            float *st = s_stat + (n & 1) * 2 * kBwdBlk;
-            st[tid] = (lse == -INFINITY || lse == INFINITY) ? INFINITY : lse * 1.4426950408889634f;
-            st[kBwdBlk + tid] = q < a.N ? a.delta[((int64_t)b * a.Hq + h) * a.N + q] : 0.f;
-        }
-        asm volatile("cp.async.commit_group;\n" ::: "memory");
-    };
-    if (n_steps > 0) load_qg(0);
-    {
-        for (int32_t n = 0; n < n_steps; ++n) {
-            const int32_t i = a.row_idx[e0 + n % per_head];
-            const uint32_t sQ = sQG + (uint32_t)(n & 1) * 2u * T::kBytes, sG = sQ + T::kBytes;
-            const float *s_lse2 = s_stat + (n & 1) * 2 * kBwdBlk, *s_delta = s_lse2 + kBwdBlk;
-            if (n + 1 < n_steps) {
-                load_qg(n + 1);  // (its buffer was released by the barrier that closed step n - 1)
-                asm volatile("cp.async.wait_group 1;\n" ::: "memory");
-            } else {
-                asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+    for (int h = hk * a.G; h < (hk + 1) * a.G; ++h) {
+        const __nv_bfloat16 *qbase = a.q + b * a.q_sb + (int64_t)h * a.q_sh;
+        const __nv_bfloat16 *gbase = a.d_o + b * a.o_sb + (int64_t)h * a.o_sh;
+        for (int32_t e = e0; e < e1; ++e) {
+            const int32_t i = a.row_idx[e];
+            __syncthreads();  // every warp has finished with the previous Q and dO tiles
+            load_tile<D>(sQ, qbase, a.q_ss, (int64_t)i * kBwdBlk, a.N, tid);
+            load_tile<D>(sG, gbase, a.o_ss, (int64_t)i * kBwdBlk, a.N, tid);
+            if (tid < kBwdBlk) {
+                const int64_t q = (int64_t)i * kBwdBlk + tid;
+                const float lse = q < a.N ? a.lse[((int64_t)b * a.Hq + h) * a.N + q] : INFINITY;
+                s_lse2[tid] = (lse == -INFINITY || lse == INFINITY) ? INFINITY : lse * 1.4426950408889634f;
+                s_delta[tid] = q < a.N ? a.delta[((int64_t)b * a.Hq + h) * a.N + q] : 0.f;
             }
-            __syncthreads();  // this step's tiles and statistics (and, first time, K and V) are visible to every warp
+            asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
+            __syncthreads();
             float s[8][4], dp[8][4];
             tile_product<D>(sK, r0, sQ, lane, s);   // S^T = K Q^T: rows = keys, columns = queries
             tile_product<D>(sV, r0, sG, lane, dp);  // dP^T = V dO^T
@@ -390,7 +373,6 @@ __global__ void __launch_bounds__(kBwdThreads) backward_dkv_kernel(const Backwar
             pack_a(dp, wd);
             tile_accumulate<D>(wp, sG, lane, dv);  // dV += P^T dO
             tile_accumulate<D>(wd, sQ, lane, dk);  // dK += dS^T Q
-            __syncthreads();  // every warp has finished with this buffer
         }
     }
     // A column that many rows list is spread over several CTAs: the parts are added up in memory.
@@ -450,7 +432,7 @@ static pa_status check_backward(const pa_prefill_params *p, int64_t nnz)
 template <int D>
 static pa_status launch_backward(const BackwardArgs &a, int64_t nnz, int device, cudaStream_t st)
 {
-    constexpr int kSmemDq = 6 * BwdTile<D>::kBytes, kSmemDkv = 6 * BwdTile<D>::kBytes + 4 * kBwdBlk * 4;
+    constexpr int kSmemDq = 4 * BwdTile<D>::kBytes, kSmemDkv = 4 * BwdTile<D>::kBytes + 2 * kBwdBlk * 4;
     if (device_once_begin(device, D == 128 ? ONCE_BACKWARD_ATTR : ONCE_BACKWARD_ATTR_64)) {
         const cudaError_t e1 = cudaFuncSetAttribute(backward_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemDq);
         const cudaError_t e2 = cudaFuncSetAttribute(backward_dkv_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemDkv);
@@ -460,7 +442,8 @@ static pa_status launch_backward(const BackwardArgs &a, int64_t nnz, int device,
         }
     }
     const int64_t rows = (int64_t)a.batch * a.N * a.Hq;
-    backward_delta_kernel<D><<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(a);
+    constexpr int kDeltaRowsPerBlock = 8 * (32 / (D / 8));  // eight warps, each 32 / (D / 8) rows
+    backward_delta_kernel<D><<<(unsigned)((rows + kDeltaRowsPerBlock - 1) / kDeltaRowsPerBlock), 256, 0, st>>>(a);
     const unsigned col_blocks = (unsigned)((a.nqb + 7) / 8);
     csc_count_kernel<<<col_blocks, 256, 0, st>>>(a);
     layout_scan_kernel<<<1, 1024, 0, st>>>(a.nqb, a.col_ptr);
