@@ -51,6 +51,7 @@ constexpr int kVStages = 3;             // V block ring depth (a V block is need
 constexpr uint32_t kTmemCols = 512;    // slot s: S at columns 128 s, P buffers at 128 s + 64 + 32 b, O at 256 + s D
 // A step's row sum above this limit sends the step through the exact path (new reference).
 constexpr float kSumLimit = 1048576.0f;  // 2^20
+constexpr int kTurnAtColumn = 16;  // column of a pass at which the other slot gets its turn (a multiple of 4 below 64)
 constexpr float kRescaleThreshold = 8.0f;  // base-2 logits: rescale O only when the row max grows by more
 constexpr long long kWaitCycles = 4000000000ll;  // default limit of a barrier wait: ~2 s at 2 GHz
 
@@ -558,9 +559,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         sum2[e] = ptx::add_f32x2(sum2[e], ptx::pack_f32x2(p0, p1));
                         pk[(c >> 1) + e] = ptx::cvt_bf16x2(p0, p1);
                     }
+                    // The turn is passed on a quarter of the way into the pass: the other slot needs
+                    // some 350 cycles to see it (measured), which then run beside the rest of this pass.
+                    if (c == kTurnAtColumn && lane == 0) ptx::mbar_arrive(bar(BAR_TURN + (s ^ 1)));
                 }
                 }
-                if (lane == 0) ptx::mbar_arrive(bar(BAR_TURN + (s ^ 1)));
                 float sum;
                 {
                     float s0, s1, s2, s3;
