@@ -406,6 +406,12 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
     const int g = lane >> 2, t = lane & 3;
     const int G = a.G;
 
+    // (item and row counts fit 31 bits; checked on the host)
+    const uint32_t n_items = (uint32_t)a.items;
+    const uint32_t it0 = blockIdx.x, it_step = gridDim.x;
+    // The first item's cache length is on the critical path of a small call: its load starts before
+    // the barrier set-up.
+    const int32_t len_first = it0 < n_items ? a.lens[(it0 / (uint32_t)R) / (uint32_t)a.Hkv] : 0;
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
             ptx::mbar_init(bar_kfull(s), 1);
@@ -426,12 +432,11 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
         int32_t b, hk, r;        // sequence, KV head, chunk
         int32_t row, last_keys;  // the query's block row; keys of the diagonal block
         int32_t cand;            // this lane's candidate key block or -1
+        int32_t rank;            // its number among the candidates that exist (lane order)
         int32_t page;            // (paged cache) its page
         uint32_t have;           // lanes whose candidate exists
         int32_t n, mine;         // blocks of the row, blocks of this chunk
     };
-    // (item and row counts fit 31 bits; checked on the host)
-    const uint32_t n_items = (uint32_t)a.items;
     auto item_len = [&](uint32_t it) -> int32_t {  // the sequence's cache length (issued early: a global load)
         return it < n_items ? a.lens[(it / (uint32_t)R) / (uint32_t)a.Hkv] : 0;
     };
@@ -450,14 +455,16 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
         w.page = 0;
         if (a.table && w.cand >= 0) w.page = a.table[(int64_t)w.b * a.table_stride + w.cand];
         w.have = __ballot_sync(0xffffffffu, w.cand >= 0);
+        w.rank = __popc(w.have & ((1u << lane) - 1u));
         w.n = __popc(w.have);
         w.mine = w.n > w.r ? (w.n - w.r + R - 1) / R : 0;
         return w;
     };
     // Key block number i of the item: the (r + i R)-th candidate that exists (lane that holds it).
-    auto lane_of = [&](const Item &w, int i) { return (int)__fns(w.have, 0, w.r + i * R + 1) & 31; };
-
-    const uint32_t it0 = blockIdx.x, it_step = gridDim.x;
+    auto lane_of = [&](const Item &w, int i) {
+        const uint32_t hit = __ballot_sync(0xffffffffu, w.cand >= 0 && w.rank == w.r + i * R);
+        return (__ffs(hit) - 1) & 31;
+    };
 
     if (wid == kRowConsumers) {
         // ------------------------------------------------------------------ producer
@@ -467,7 +474,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
         }
         bool ok = true;
         uint32_t ci = 0;  // blocks issued so far by this CTA (ring position)
-        int32_t len_next = item_len(it0);
+        int32_t len_next = len_first;
         for (uint32_t it = it0; it < n_items; it += it_step) {
             const Item w = make_item(it, len_next);
             len_next = item_len(it + it_step);
@@ -521,7 +528,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
         load_q(it0);
         bool ok = true;
         uint32_t ci = 0;
-        int32_t len_next = item_len(it0);
+        int32_t len_next = len_first;
         for (uint32_t it = it0; it < n_items && ok; it += it_step) {
             const Item w = make_item(it, len_next);
             len_next = item_len(it + it_step);
@@ -738,8 +745,9 @@ __global__ void __launch_bounds__(kRowThreads, 2) decode_row_kernel(const __grid
                     }
                 }
             }
-            // The hand-over area is written again only after every warp has read it.
-            asm volatile("bar.sync 1, %0;\n" ::"n"(32 * kRowConsumers) : "memory");
+            // The hand-over area is written again only after every warp has read it (the cluster form
+            // has one item per CTA: nothing follows).
+            if (a.mode != kModeCluster) asm volatile("bar.sync 1, %0;\n" ::"n"(32 * kRowConsumers) : "memory");
         }
     }
 
