@@ -48,7 +48,8 @@ const char *pa_last_error_message(void);
 /* major * 10000 + minor * 100 + patch */
 int pa_version(void);
 
-/* Environment switches (PA_VALIDATE, PA_DECODE_PATH, PA_DECODE_CLUSTER, PA_DECODE_STAGES; each is
+/* Environment switches (PA_VALIDATE, PA_DECODE_PATH, PA_DECODE_CLUSTER, PA_DECODE_STAGES,
+ * PA_DECODE_CTAS_PER_SM; each is
  * described at the call it affects) are read once, when a call first needs them.  This re-reads
  * them; tests and measurement scripts call it after changing the environment. */
 void pa_reload_environment(void);
@@ -270,7 +271,7 @@ size_t pa_decode_workspace_bytes(const pa_decode_params *p);
  * =cluster / =persist the two forms of the row kernel; PA_DECODE_CLUSTER=n (1..8) sets R (default:
  * for small calls as many CTAs per row as run all at once, for large ones one chunk per row once
  * there are as many rows as SMs, else two); PA_DECODE_STAGES=n (1..6) the number of key blocks a CTA keeps
- * in flight. */
+ * in flight; PA_DECODE_CTAS_PER_SM=n the size of the persistent grid (default 2 per SM). */
 pa_status pa_decode(const pa_decode_params *p, const void *q, const void *k_cache,
                     const void *v_cache, const int32_t *cache_lens, void *o, float *lse,
                     void *workspace, size_t workspace_bytes, void *stream);
