@@ -49,12 +49,12 @@ const char *pa_last_error_message(void);
 int pa_version(void);
 
 /* Environment switches (PA_VALIDATE, PA_DECODE_PATH, PA_DECODE_CLUSTER, PA_DECODE_STAGES,
- * PA_DECODE_CTAS_PER_SM; each is
+ * PA_DECODE_CTAS_PER_SM, PA_BACKWARD_PATH; each is
  * described at the call it affects) are read once, when a call first needs them.  This re-reads
  * them; tests and measurement scripts call it after changing the environment. */
 void pa_reload_environment(void);
 
-/* Limit, in GPU clock cycles, of every bounded barrier wait inside the prefill and decode kernels
+/* Limit, in GPU clock cycles, of every bounded barrier wait inside the prefill, backward and decode kernels
  * (a wait that runs out ends the kernel with PA_ERR_TIMEOUT in its status block, see
  * pa_prefill_status and pa_decode_status).  cycles <= 0 restores the defaults of one to two
  * seconds.  Process-wide; applies to calls made after it returns. */
@@ -215,12 +215,15 @@ pa_status pa_prefill_status(const void *workspace, void *stream, int32_t *detail
  * pa_prefill returned; d_o: device bf16 with the strides of o.  dq: device fp32 [batch, seq_len,
  * n_q_heads, head_dim] contiguous; dk, dv: device fp32 [batch, seq_len, n_kv_heads, head_dim]
  * contiguous (cleared by the call).  workspace: device, 256-byte aligned,
- * >= pa_prefill_backward_workspace_bytes(p, nnz) (the row sums delta and the transposed layout).
- * Two memsets and seven kernels are enqueued.  S and P are recomputed tile by tile on the warp-level
- * tensor-core MMA (bf16 operands, fp32 accumulation).  A key block that many query blocks list (a
- * sink block is listed by all) is spread over several CTAs that add their parts with fp32 atomics,
- * so dk and dv of such blocks may differ in the last bits from run to run.
- * Errors: as pa_prefill.
+ * >= pa_prefill_backward_workspace_bytes(p, nnz) (a status block, the row sums delta and the
+ * transposed layout).  Three memsets and seven kernels are enqueued.  S and P are recomputed tile by
+ * tile on the tensor cores (bf16 operands, fp32 accumulation): head_dim 128 on tcgen05 with
+ * accumulators in tensor memory, head_dim 64 (and head_dim 128 under PA_BACKWARD_PATH=mma) on the
+ * warp-level MMA.  A key block that many query blocks list (a sink block is listed by all) is spread
+ * over several CTAs that add their parts with fp32 atomics, so dk and dv of such blocks may differ
+ * in the last bits from run to run.
+ * Errors: as pa_prefill.  The tcgen05 kernels bound their barrier waits like the prefill kernel;
+ * pa_prefill_status(workspace, ...) on the backward workspace reports a wait that ran out.
  * ------------------------------------------------------------------------------------------ */
 size_t pa_prefill_backward_workspace_bytes(const pa_prefill_params *p, int64_t nnz);
 pa_status pa_prefill_backward(const pa_prefill_params *p, const void *q, const void *k, const void *v,

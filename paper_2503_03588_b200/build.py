@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(PKG, "libpowerattn.so")
-SOURCES = ["api.cu", "layout.cu", "decode.cu", "prefill_sm100.cu", "backward.cu"]
+SOURCES = ["api.cu", "layout.cu", "decode.cu", "prefill_sm100.cu", "backward.cu", "backward_sm100.cu"]
 
 
 def _nvcc() -> str:

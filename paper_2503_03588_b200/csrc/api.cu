@@ -97,6 +97,8 @@ static void read_env_locked()
     g_env.decode_cluster = env_int("PA_DECODE_CLUSTER", 1, 8);
     g_env.decode_stages = env_int("PA_DECODE_STAGES", 1, 8);
     g_env.decode_ctas_per_sm = env_int("PA_DECODE_CTAS_PER_SM", 1, 64);
+    const char *bw = getenv("PA_BACKWARD_PATH");
+    g_env.backward_mma = bw && bw[0] == 'm';
     const char *v = getenv("PA_VALIDATE");
     g_env.validate = v && v[0] == '1';
     g_env_known = true;

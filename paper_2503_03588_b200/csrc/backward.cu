@@ -21,30 +21,14 @@
 #include <cuda_bf16.h>
 #include <math.h>
 
+#include "backward.cuh"
 #include "common.cuh"
 #include "scan.cuh"
 #include "sm100_ptx.cuh"
 
 namespace pa {
 
-constexpr int kBwdBlk = 64;       // tokens per block
 constexpr int kBwdThreads = 128;  // four warps, 16 rows of the tile each
-constexpr int kBwdChunk = 32;     // query blocks per CTA of the dK / dV kernel
-
-struct BackwardArgs {
-    const __nv_bfloat16 *q, *k, *v, *o, *d_o;
-    const float *lse;          // [batch, Hq, N]
-    const int32_t *row_ptr, *col_idx;
-    float *delta;              // [batch, Hq, N]
-    int32_t *col_ptr;          // [nqb + 1]: extents of the transposed lists
-    int32_t *row_idx;          // [nnz]: query blocks that list each key block, ascending
-    int32_t *chunk_ptr;        // [nqb + 1]: first chunk of each column
-    float *dq, *dk, *dv;       // fp32, contiguous [batch, N, H, D]
-    int64_t q_sb, q_ss, q_sh, k_sb, k_ss, k_sh, v_sb, v_ss, v_sh, o_sb, o_ss, o_sh;
-    int64_t N;
-    int32_t nqb, batch, Hq, Hkv, G;
-    float scale, scale_log2;
-};
 
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1)
@@ -395,11 +379,12 @@ __global__ void __launch_bounds__(kBwdThreads) backward_dkv_kernel(const Backwar
 
 namespace pa {
 
-// Workspace: delta [batch, Hq, N] fp32, then col_ptr [nqb + 1], chunk_ptr [nqb + 1], row_idx [nnz] int32.
+// Workspace: status block (256 bytes), delta [batch, Hq, N] fp32, then col_ptr [nqb + 1], chunk_ptr [nqb + 1],
+// row_idx [nnz] int32.
 static size_t backward_workspace_bytes(const pa_prefill_params *p, int64_t nnz)
 {
     const int64_t nqb = (p->seq_len + kBwdBlk - 1) / kBwdBlk;
-    size_t bytes = (size_t)p->batch * p->n_q_heads * p->seq_len * sizeof(float);
+    size_t bytes = kBwdStatusBytes + (size_t)p->batch * p->n_q_heads * p->seq_len * sizeof(float);
     bytes = (bytes + 255) & ~(size_t)255;
     bytes += (size_t)(2 * (nqb + 1) + nnz) * sizeof(int32_t);
     return (bytes + 255) & ~(size_t)255;
@@ -430,7 +415,7 @@ static pa_status check_backward(const pa_prefill_params *p, int64_t nnz)
 }
 
 template <int D>
-static pa_status launch_backward(const BackwardArgs &a, int64_t nnz, int device, cudaStream_t st)
+static pa_status launch_backward(const BackwardArgs &a, const pa_prefill_params *p, int64_t nnz, int device, cudaStream_t st)
 {
     constexpr int kSmemDq = 4 * BwdTile<D>::kBytes, kSmemDkv = 4 * BwdTile<D>::kBytes + 2 * kBwdBlk * 4;
     if (device_once_begin(device, D == 128 ? ONCE_BACKWARD_ATTR : ONCE_BACKWARD_ATTR_64)) {
@@ -449,6 +434,11 @@ static pa_status launch_backward(const BackwardArgs &a, int64_t nnz, int device,
     layout_scan_kernel<<<1, 1024, 0, st>>>(a.nqb, a.col_ptr);
     layout_scan_kernel<<<1, 1024, 0, st>>>(a.nqb, a.chunk_ptr);
     csc_fill_kernel<<<col_blocks, 256, 0, st>>>(a);
+    // head_dim 128: dQ, dK and dV on the tcgen05 tensor cores (PA_BACKWARD_PATH=mma keeps the warp-level kernels).
+    if (D == 128 && !env_switches().backward_mma) {
+        PA_CUDA_OK(cudaGetLastError());
+        return launch_backward_sm100(a, p, nnz, device, st);
+    }
     backward_dq_kernel<D><<<dim3((unsigned)a.nqb, (unsigned)a.Hq, (unsigned)a.batch), kBwdThreads, kSmemDq, st>>>(a);
     // (an upper bound on the number of chunks; CTAs beyond the real count return at once)
     const int64_t max_chunks = nnz / kBwdChunk + a.nqb;
@@ -497,8 +487,9 @@ extern "C" pa_status pa_prefill_backward(const pa_prefill_params *p, const void 
     a.col_idx = col_idx;
     const int64_t nqb = (p->seq_len + kBwdBlk - 1) / kBwdBlk;
     uint8_t *ws = static_cast<uint8_t *>(workspace);
-    a.delta = reinterpret_cast<float *>(ws);
-    size_t off = ((size_t)p->batch * p->n_q_heads * p->seq_len * sizeof(float) + 255) & ~(size_t)255;
+    a.status = reinterpret_cast<int32_t *>(ws);
+    a.delta = reinterpret_cast<float *>(ws + kBwdStatusBytes);
+    size_t off = (kBwdStatusBytes + (size_t)p->batch * p->n_q_heads * p->seq_len * sizeof(float) + 255) & ~(size_t)255;
     a.col_ptr = reinterpret_cast<int32_t *>(ws + off);
     a.chunk_ptr = a.col_ptr + (nqb + 1);
     a.row_idx = a.chunk_ptr + (nqb + 1);
@@ -513,10 +504,13 @@ extern "C" pa_status pa_prefill_backward(const pa_prefill_params *p, const void 
     a.G = p->n_q_heads / p->n_kv_heads;
     a.scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
     a.scale_log2 = a.scale * 1.4426950408889634f;
+    a.npairs = (a.G + 1) / 2;
+    a.wait_cycles = 0;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t kv_bytes = (size_t)p->batch * p->seq_len * p->n_kv_heads * p->head_dim * sizeof(float);
+    PA_CUDA_OK(cudaMemsetAsync(workspace, 0, kBwdStatusBytes, st));
     PA_CUDA_OK(cudaMemsetAsync(dk, 0, kv_bytes, st));
     PA_CUDA_OK(cudaMemsetAsync(dv, 0, kv_bytes, st));
-    return p->head_dim == 128 ? launch_backward<128>(a, nnz, dev.device, st) : launch_backward<64>(a, nnz, dev.device, st);
+    return p->head_dim == 128 ? launch_backward<128>(a, p, nnz, dev.device, st) : launch_backward<64>(a, p, nnz, dev.device, st);
 }

@@ -26,7 +26,7 @@ struct DeviceInfo {
 pa_status current_sm100_device(DeviceInfo *out);
 
 // One-time per-device set-up steps (kernel attributes) are keyed by these slots.
-enum DeviceOnce : int { ONCE_PREFILL_ATTR = 0, ONCE_DECODE_ATTR, ONCE_BACKWARD_ATTR, ONCE_BACKWARD_ATTR_64, ONCE_COUNT };
+enum DeviceOnce : int { ONCE_PREFILL_ATTR = 0, ONCE_DECODE_ATTR, ONCE_BACKWARD_ATTR, ONCE_BACKWARD_ATTR_64, ONCE_BACKWARD_TC_ATTR, ONCE_COUNT };
 // True exactly once per (device, slot); the caller then performs the step and, if it fails, calls
 // device_once_reset so that a later call tries again.
 bool device_once_begin(int device, DeviceOnce slot);
@@ -40,6 +40,7 @@ struct EnvSwitches {
     int decode_stages;   // PA_DECODE_STAGES=1..8, 0 = chosen from the problem size
     int decode_ctas_per_sm;  // PA_DECODE_CTAS_PER_SM=n: size of the persistent grid (default 2 per SM)
     int validate;        // PA_VALIDATE=1
+    int backward_mma;    // PA_BACKWARD_PATH=mma: the warp-level MMA kernels for head_dim 128 too
 };
 EnvSwitches env_switches();
 
