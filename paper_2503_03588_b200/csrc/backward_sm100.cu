@@ -3,8 +3,9 @@
 //
 // Two kernels, both with the same skeleton of 384 threads:
 //   warp 0       TMA producer (bf16 tiles, 128-byte swizzle, into rings of shared-memory stages)
-//   warp 1       tcgen05 issuer (one elected lane)
+//   warp 1       tcgen05 issuer of S and dP (one elected lane)
 //   warp 2       tensor-memory allocation
+//   warp 3       tcgen05 issuer of the second products
 //   warps 4-7    compute group 0: even steps
 //   warps 8-11   compute group 1: odd steps
 // A step is one (query block, key block) pair for a pair of query heads stacked on the 64 tokens of
@@ -153,15 +154,14 @@ dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
         }
         __syncwarp();
     } else if (warp == 1) {
-        // -------------------------------------------------------------- tcgen05 issuer
+        // -------------------------------------------------------------- tcgen05 issuer of S and dP
         const bool leader = ptx::elect_one();
-        constexpr uint32_t idesc_s = idesc_bf16(128, 64, 0, 0);   // S, dP: both operands K-major
-        constexpr uint32_t idesc_dq = idesc_bf16(128, D, 0, 1);   // dQ: A = dS (tensor memory), B = K feature-contiguous
+        constexpr uint32_t idesc_s = idesc_bf16(128, 64, 0, 0);   // both operands K-major
         const uint32_t q_lo = ((smem_base + SM::kQ) >> 4) | (1u << 16);
         const uint32_t g_lo = ((smem_base + SM::kG) >> 4) | (1u << 16);
         bool ok = true;
-        for (int e = 0; e <= n && ok && n > 0; ++e) {
-            if (e < n) {
+        for (int e = 0; e < n && ok; ++e) {
+            {
                 const uint32_t bf = e & 1, st = e % kDqStages;
                 if (e == 0) ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_QG_FULL), 0, 1));
                 if (ok) ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_KV_FULL + st), (e / kDqStages) & 1, 3));
@@ -184,8 +184,15 @@ dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
                 }
                 __syncwarp();
             }
-            if (e >= 1) {
-                const int e1 = e - 1;
+        }
+    } else if (warp == 3) {
+        // -------------------------------------------------------------- tcgen05 issuer of dQ
+        // (its own warp: a single issuer that served both kinds in order held each back behind the other's waits)
+        const bool leader = ptx::elect_one();
+        constexpr uint32_t idesc_dq = idesc_bf16(128, D, 0, 1);   // A = dS (tensor memory), B = K feature-contiguous
+        bool ok = true;
+        for (int e1 = 0; e1 < n && ok; ++e1) {
+            {
                 const uint32_t bf = e1 & 1, st = e1 % kDqStages;
                 ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_DS_FULL + bf), (e1 >> 1) & 1, 5));
                 if (!ok) break;
@@ -412,15 +419,14 @@ dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         }
         __syncwarp();
     } else if (warp == 1) {
-        // -------------------------------------------------------------- tcgen05 issuer
+        // -------------------------------------------------------------- tcgen05 issuer of S and dP
         const bool leader = ptx::elect_one();
-        constexpr uint32_t idesc_s = idesc_bf16(128, 64, 0, 0);    // S, dP: both operands K-major
-        constexpr uint32_t idesc_t = idesc_bf16(128, 64, 1, 1);    // dV^T, dK^T: A feature-contiguous, B key-contiguous
+        constexpr uint32_t idesc_s = idesc_bf16(128, 64, 0, 0);    // both operands K-major
         const uint32_t k_lo = ((smem_base + SM::kK) >> 4) | (1u << 16);
         const uint32_t v_lo = ((smem_base + SM::kV) >> 4) | (1u << 16);
         bool ok = __all_sync(0xffffffffu, wait_bar(bar(KV_KV_FULL), 0, 1));
-        for (int e = 0; e <= n && ok; ++e) {
-            if (e < n) {
+        for (int e = 0; e < n && ok; ++e) {
+            {
                 const uint32_t bf = e & 1;
                 ok = __all_sync(0xffffffffu, wait_bar(bar(KV_QG_FULL + bf), (e >> 1) & 1, 3));
                 if (ok && e >= 2) ok = __all_sync(0xffffffffu, wait_bar(bar(KV_S_TAKEN + bf), ((e >> 1) - 1) & 1, 4));
@@ -442,8 +448,16 @@ dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 }
                 __syncwarp();
             }
-            if (e >= 1) {
-                const int e1 = e - 1;
+        }
+    } else if (warp == 3) {
+        // -------------------------------------------------------------- tcgen05 issuer of dV^T and dK^T
+        // (its own warp: a Q / dO stage is free for the next load only when these have read it, and a
+        // single in-order issuer put them behind the next step's S and dP)
+        const bool leader = ptx::elect_one();
+        constexpr uint32_t idesc_t = idesc_bf16(128, 64, 1, 1);    // A feature-contiguous, B key-contiguous
+        bool ok = true;
+        for (int e1 = 0; e1 < n && ok; ++e1) {
+            {
                 const uint32_t bf = e1 & 1;
                 ok = __all_sync(0xffffffffu, wait_bar(bar(KV_PD_FULL + bf), (e1 >> 1) & 1, 5));
                 if (!ok) break;
