@@ -415,7 +415,8 @@ static pa_status check_backward(const pa_prefill_params *p, int64_t nnz)
 }
 
 template <int D>
-static pa_status launch_backward(const BackwardArgs &a, const pa_prefill_params *p, int64_t nnz, int device, cudaStream_t st)
+static pa_status launch_backward(const BackwardArgs &a, const pa_prefill_params *p, int64_t nnz, int device, int sms,
+                                 cudaStream_t st)
 {
     constexpr int kSmemDq = 4 * BwdTile<D>::kBytes, kSmemDkv = 4 * BwdTile<D>::kBytes + 2 * kBwdBlk * 4;
     if (device_once_begin(device, D == 128 ? ONCE_BACKWARD_ATTR : ONCE_BACKWARD_ATTR_64)) {
@@ -437,7 +438,7 @@ static pa_status launch_backward(const BackwardArgs &a, const pa_prefill_params 
     // head_dim 128: dQ, dK and dV on the tcgen05 tensor cores (PA_BACKWARD_PATH=mma keeps the warp-level kernels).
     if (D == 128 && !env_switches().backward_mma) {
         PA_CUDA_OK(cudaGetLastError());
-        return launch_backward_sm100(a, p, nnz, device, st);
+        return launch_backward_sm100(a, p, nnz, device, sms, st);
     }
     backward_dq_kernel<D><<<dim3((unsigned)a.nqb, (unsigned)a.Hq, (unsigned)a.batch), kBwdThreads, kSmemDq, st>>>(a);
     // (an upper bound on the number of chunks; CTAs beyond the real count return at once)
@@ -512,5 +513,5 @@ extern "C" pa_status pa_prefill_backward(const pa_prefill_params *p, const void 
     PA_CUDA_OK(cudaMemsetAsync(workspace, 0, kBwdStatusBytes, st));
     PA_CUDA_OK(cudaMemsetAsync(dk, 0, kv_bytes, st));
     PA_CUDA_OK(cudaMemsetAsync(dv, 0, kv_bytes, st));
-    return p->head_dim == 128 ? launch_backward<128>(a, p, nnz, dev.device, st) : launch_backward<64>(a, p, nnz, dev.device, st);
+    return p->head_dim == 128 ? launch_backward<128>(a, p, nnz, dev.device, dev.sms, st) : launch_backward<64>(a, p, nnz, dev.device, dev.sms, st);
 }

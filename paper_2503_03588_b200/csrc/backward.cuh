@@ -34,6 +34,7 @@ struct BackwardArgs {
 };
 
 // dQ, dK, dV for head_dim 128 on tcgen05 (delta and the transposed lists are already in the workspace).
-pa_status launch_backward_sm100(const BackwardArgs &a, const pa_prefill_params *p, int64_t nnz, int device, cudaStream_t st);
+pa_status launch_backward_sm100(const BackwardArgs &a, const pa_prefill_params *p, int64_t nnz, int device, int sms,
+                                cudaStream_t st);
 
 }  // namespace pa

@@ -54,29 +54,58 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int a_mn, int b_
 }
 
 // ------------------------------------------------------------------------------------- dQ
-constexpr int kDqStages = 4;  // K + V ring
+// Persistent: one CTA per SM walks items (query block, head pair, batch entry), long rows first.
+// Steps are numbered through the CTA's whole run, so ring positions, buffers and barrier parities do
+// not care about item boundaries.  Q and dO have one buffer: the next item's tiles are requested when
+// the current item's last S and dP have been issued and arrive while its last steps are computed
+// and its dQ leaves tensor memory, which takes longer; the K / V ring of five stages covers a
+// stage's life from request to the dQ product that reads it last (about four steps).
+constexpr int kDqStages = 5;  // K + V ring
 struct DqSmem {
-    static constexpr uint32_t kQ = 0;                       // two halves of 128 rows x 128 B
-    static constexpr uint32_t kG = kQ + 2 * kRowTile;       // dO tile
-    static constexpr uint32_t kKV = kG + 2 * kRowTile;      // stage: K (two halves), then V
+    static constexpr uint32_t kQG = 0;                      // Q (two halves of 128 rows x 128 B), then dO
+    static constexpr uint32_t kItem = 4 * kRowTile;
+    static constexpr uint32_t kKV = kQG + kItem;            // stage: K (two halves), then V
     static constexpr uint32_t kStage = 4 * kKeyTile;
     static constexpr uint32_t kBars = kKV + kDqStages * kStage;
     static constexpr uint32_t kAlloc = kBars + 512 + 1024;
+    static_assert(kAlloc <= 227 * 1024, "shared memory budget");
 };
 enum : uint32_t {
-    DQ_QG_FULL = 0,
-    DQ_KV_FULL = 1, DQ_KV_EMPTY = DQ_KV_FULL + kDqStages,
+    DQ_QG_FULL = 0, DQ_QG_EMPTY = 1,
+    DQ_KV_FULL = 2, DQ_KV_EMPTY = DQ_KV_FULL + kDqStages,
     DQ_SD_FULL = DQ_KV_EMPTY + kDqStages,  // [buffer]: S and dP of a step are in tensor memory
     DQ_S_TAKEN = DQ_SD_FULL + 2,            // [buffer]: the group has them in registers
     DQ_DS_FULL = DQ_S_TAKEN + 2,            // [buffer]: dS is in tensor memory
     DQ_DS_FREE = DQ_DS_FULL + 2,            // [buffer]: dQ += dS K has read it
-    DQ_DONE = DQ_DS_FREE + 2,
-    DQ_BAR_COUNT = DQ_DONE + 1
+    DQ_DONE = DQ_DS_FREE + 2,               // the item's last dQ += dS K has completed
+    DQ_FREE = DQ_DONE + 1,                  // the compute groups have read dQ out of tensor memory
+    DQ_BAR_COUNT = DQ_FREE + 1
 };
+
+struct DqItem {
+    int32_t i, hk, hp, b, e0, n;
+};
+// Item index -> coordinates: query blocks from the last (longest row) to the first, and within a
+// query block the head pairs and batch entries.
+__device__ __forceinline__ DqItem dq_item(const BackwardArgs &a, uint32_t it)
+{
+    DqItem w;
+    const uint32_t per_row = (uint32_t)(a.Hkv * a.npairs * a.batch);
+    const uint32_t x = it / per_row, yz = it % per_row;
+    const uint32_t hkp = yz % (uint32_t)(a.Hkv * a.npairs);
+    w.i = a.nqb - 1 - (int32_t)x;
+    w.b = (int32_t)(yz / (uint32_t)(a.Hkv * a.npairs));
+    w.hk = (int32_t)(hkp / (uint32_t)a.npairs);
+    w.hp = (int32_t)(hkp % (uint32_t)a.npairs);
+    w.e0 = __ldg(a.row_ptr + w.i);
+    w.n = __ldg(a.row_ptr + w.i + 1) - w.e0;
+    return w;
+}
 
 __global__ void __launch_bounds__(kTcThreads, 1)
 dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmG,
-          const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const BackwardArgs a)
+          const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const BackwardArgs a,
+          const uint32_t n_items)
 {
     constexpr int D = 128;
     using SM = DqSmem;
@@ -91,24 +120,22 @@ dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
         return ptx::mbar_wait_bounded(b_, parity, abort_flag, a.status, code, a.wait_cycles, (int)PA_ERR_TIMEOUT);
     };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int i = a.nqb - 1 - (int)blockIdx.x;  // long rows first
-    const int hk = (int)blockIdx.y / a.npairs, hp = (int)blockIdx.y % a.npairs, b = blockIdx.z;
-    const int32_t e0 = a.row_ptr[i];
-    const int n = a.row_ptr[i + 1] - e0;
 
     if (threadIdx.x == 0) {
         ptx::mbar_init(bar(DQ_QG_FULL), 1);
-        for (int s = 0; s < kDqStages; ++s) {
-            ptx::mbar_init(bar(DQ_KV_FULL + s), 1);
-            ptx::mbar_init(bar(DQ_KV_EMPTY + s), 1);
-        }
+        ptx::mbar_init(bar(DQ_QG_EMPTY), 2);  // one commit from each of the S and dP issuers
         for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(bar(DQ_SD_FULL + s), 1);
+            ptx::mbar_init(bar(DQ_SD_FULL + s), 2);
             ptx::mbar_init(bar(DQ_S_TAKEN + s), 4);
             ptx::mbar_init(bar(DQ_DS_FULL + s), 4);
             ptx::mbar_init(bar(DQ_DS_FREE + s), 1);
         }
+        for (int s = 0; s < kDqStages; ++s) {
+            ptx::mbar_init(bar(DQ_KV_FULL + s), 1);
+            ptx::mbar_init(bar(DQ_KV_EMPTY + s), 1);
+        }
         ptx::mbar_init(bar(DQ_DONE), 1);
+        ptx::mbar_init(bar(DQ_FREE), 8);
         *abort_flag = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
@@ -127,74 +154,94 @@ dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
     if (warp < 4) ptx::setmaxnreg_dec<PA_BWD_REG_CTRL>();
     if (warp == 0) {
         // -------------------------------------------------------------- TMA producer
-        if (lane == 0 && n > 0) {
+        if (lane == 0) {
             ptx::prefetch_tensormap(&tmQ);
             ptx::prefetch_tensormap(&tmG);
             ptx::prefetch_tensormap(&tmK);
             ptx::prefetch_tensormap(&tmV);
-            const int h0 = hk * a.G + 2 * hp;
-            ptx::mbar_expect_tx(bar(DQ_QG_FULL), 4 * kRowTile);
-            for (int dh = 0; dh < 2; ++dh) {
-                ptx::tma_load_4d(smem_base + SM::kQ + dh * kRowTile, &tmQ, bar(DQ_QG_FULL), dh * 64, i * kBwdBlk, h0, b);
-                ptx::tma_load_4d(smem_base + SM::kG + dh * kRowTile, &tmG, bar(DQ_QG_FULL), dh * 64, i * kBwdBlk, h0, b);
-            }
-            int32_t j = __ldg(a.col_idx + e0);
-            for (int e = 0; e < n; ++e) {
-                const int32_t jn = e + 1 < n ? __ldg(a.col_idx + e0 + e + 1) : 0;
-                const uint32_t st = e % kDqStages;
-                if (e >= kDqStages && !wait_bar(bar(DQ_KV_EMPTY + st), (e / kDqStages - 1) & 1, 2)) break;
-                ptx::mbar_expect_tx(bar(DQ_KV_FULL + st), SM::kStage);
-                const uint32_t dst = smem_base + SM::kKV + st * SM::kStage;
+            uint32_t c = 0, k = 0;  // steps and (non-empty) items so far
+            bool ok = true;
+            for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+                const DqItem w = dq_item(a, it);
+                if (w.n <= 0) continue;
+                if (k >= 1 && !wait_bar(bar(DQ_QG_EMPTY), (k - 1) & 1, 1)) break;
+                const int h0 = w.hk * a.G + 2 * w.hp;
+                const uint32_t qdst = smem_base + SM::kQG;
+                ptx::mbar_expect_tx(bar(DQ_QG_FULL), SM::kItem);
                 for (int dh = 0; dh < 2; ++dh) {
-                    ptx::tma_load_4d(dst + dh * kKeyTile, &tmK, bar(DQ_KV_FULL + st), dh * 64, j * kBwdBlk, hk, b);
-                    ptx::tma_load_4d(dst + 2 * kKeyTile + dh * kKeyTile, &tmV, bar(DQ_KV_FULL + st), dh * 64, j * kBwdBlk, hk, b);
+                    ptx::tma_load_4d(qdst + dh * kRowTile, &tmQ, bar(DQ_QG_FULL), dh * 64, w.i * kBwdBlk, h0, w.b);
+                    ptx::tma_load_4d(qdst + 2 * kRowTile + dh * kRowTile, &tmG, bar(DQ_QG_FULL), dh * 64, w.i * kBwdBlk, h0, w.b);
                 }
-                j = jn;
+                int32_t j = __ldg(a.col_idx + w.e0);
+                for (int e = 0; e < w.n; ++e, ++c) {
+                    const int32_t jn = e + 1 < w.n ? __ldg(a.col_idx + w.e0 + e + 1) : 0;
+                    const uint32_t st = c % kDqStages;
+                    if (c >= (uint32_t)kDqStages && !wait_bar(bar(DQ_KV_EMPTY + st), (c / kDqStages - 1) & 1, 2)) {
+                        ok = false;
+                        break;
+                    }
+                    ptx::mbar_expect_tx(bar(DQ_KV_FULL + st), SM::kStage);
+                    const uint32_t dst = smem_base + SM::kKV + st * SM::kStage;
+                    for (int dh = 0; dh < 2; ++dh) {
+                        ptx::tma_load_4d(dst + dh * kKeyTile, &tmK, bar(DQ_KV_FULL + st), dh * 64, j * kBwdBlk, w.hk, w.b);
+                        ptx::tma_load_4d(dst + 2 * kKeyTile + dh * kKeyTile, &tmV, bar(DQ_KV_FULL + st), dh * 64, j * kBwdBlk, w.hk, w.b);
+                    }
+                    j = jn;
+                }
+                ++k;
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
-        // -------------------------------------------------------------- tcgen05 issuer of S and dP
+    } else if (warp == 1 || warp == 2) {
+        // -------------------------------------------------------------- tcgen05 issuers of S (warp 1) and dP (warp 2)
+        // (a warp each: issuing a step's sixteen MMAs and its three waits from one warp took longer
+        // than the tensor cores need for them)
         const bool leader = ptx::elect_one();
+        const bool is_dp = __shfl_sync(0xffffffffu, warp, 0) == 2;
         constexpr uint32_t idesc_s = idesc_bf16(128, 64, 0, 0);   // both operands K-major
-        const uint32_t q_lo = ((smem_base + SM::kQ) >> 4) | (1u << 16);
-        const uint32_t g_lo = ((smem_base + SM::kG) >> 4) | (1u << 16);
+        // A = Q (S) or dO (dP); B = the K or V half of the stage.
+        const uint32_t a_lo = ((smem_base + SM::kQG + (is_dp ? 2 * kRowTile : 0u)) >> 4) | (1u << 16);
+        uint32_t c = 0, k = 0;
         bool ok = true;
-        for (int e = 0; e < n && ok; ++e) {
-            {
-                const uint32_t bf = e & 1, st = e % kDqStages;
-                if (e == 0) ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_QG_FULL), 0, 1));
-                if (ok) ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_KV_FULL + st), (e / kDqStages) & 1, 3));
-                if (ok && e >= 2) ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_S_TAKEN + bf), ((e >> 1) - 1) & 1, 4));
+        for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+            const int n = __shfl_sync(0xffffffffu, dq_item(a, it).n, 0);
+            if (n <= 0) continue;
+            for (int e = 0; e < n && ok; ++e, ++c) {
+                const uint32_t bf = c & 1, st = c % kDqStages;
+                if (e == 0) ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_QG_FULL), k & 1, 3));
+                if (ok) ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_KV_FULL + st), (c / kDqStages) & 1, 4));
+                if (ok && c >= 2) ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_S_TAKEN + bf), ((c >> 1) - 1) & 1, 5));
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 if (leader) {
-                    const uint32_t k_lo = ((smem_base + SM::kKV + st * SM::kStage) >> 4) | (1u << 16);
-                    const uint32_t v_lo = k_lo + ((2 * kKeyTile) >> 4);
-                    const uint32_t t_s = tmem_base + 160 * bf, t_dp = t_s + 64;
+                    const uint32_t b_lo = ((smem_base + SM::kKV + st * SM::kStage + (is_dp ? 2 * kKeyTile : 0u)) >> 4) | (1u << 16);
+                    const uint32_t t_d = tmem_base + 160 * bf + (is_dp ? 64u : 0u);
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk)
-                        ptx::umma_ss_lohi(t_s, q_lo + (((kk / 4) * kRowTile + (kk % 4) * 32) >> 4), kDescHi,
-                                          k_lo + (((kk / 4) * kKeyTile + (kk % 4) * 32) >> 4), kDescHi, idesc_s, kk > 0 ? 1u : 0u);
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk)
-                        ptx::umma_ss_lohi(t_dp, g_lo + (((kk / 4) * kRowTile + (kk % 4) * 32) >> 4), kDescHi,
-                                          v_lo + (((kk / 4) * kKeyTile + (kk % 4) * 32) >> 4), kDescHi, idesc_s, kk > 0 ? 1u : 0u);
+                        ptx::umma_ss_lohi(t_d, a_lo + (((kk / 4) * kRowTile + (kk % 4) * 32) >> 4), kDescHi,
+                                          b_lo + (((kk / 4) * kKeyTile + (kk % 4) * 32) >> 4), kDescHi, idesc_s, kk > 0 ? 1u : 0u);
                     ptx::umma_commit(bar(DQ_SD_FULL + bf));
+                    if (e == n - 1) ptx::umma_commit(bar(DQ_QG_EMPTY));  // this warp has read the item's Q (dO) tile
                 }
                 __syncwarp();
             }
+            ++k;
         }
     } else if (warp == 3) {
         // -------------------------------------------------------------- tcgen05 issuer of dQ
         // (its own warp: a single issuer that served both kinds in order held each back behind the other's waits)
         const bool leader = ptx::elect_one();
         constexpr uint32_t idesc_dq = idesc_bf16(128, D, 0, 1);   // A = dS (tensor memory), B = K feature-contiguous
+        uint32_t c = 0, k = 0;
         bool ok = true;
-        for (int e1 = 0; e1 < n && ok; ++e1) {
-            {
-                const uint32_t bf = e1 & 1, st = e1 % kDqStages;
-                ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_DS_FULL + bf), (e1 >> 1) & 1, 5));
+        for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+            const int n = __shfl_sync(0xffffffffu, dq_item(a, it).n, 0);
+            if (n <= 0) continue;
+            for (int e = 0; e < n && ok; ++e, ++c) {
+                const uint32_t bf = c & 1, st = c % kDqStages;
+                ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_DS_FULL + bf), (c >> 1) & 1, 6));
+                // The previous item's dQ must have left tensor memory.
+                if (ok && e == 0 && k > 0) ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_FREE), (k - 1) & 1, 7));
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 if (leader) {
@@ -204,91 +251,127 @@ dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
 #pragma unroll
                     for (int kk = 0; kk < kBwdBlk / 16; ++kk)
                         ptx::umma_ts_lohi(tmem_base + kColDq, t_ds + kk * 8, kb + ((kk * 2048) >> 4), kDescHi, idesc_dq,
-                                          (e1 > 0 || kk > 0) ? 1u : 0u);
+                                          (e > 0 || kk > 0) ? 1u : 0u);
                     ptx::umma_commit(bar(DQ_KV_EMPTY + st));
                     ptx::umma_commit(bar(DQ_DS_FREE + bf));
-                    if (e1 == n - 1) ptx::umma_commit(bar(DQ_DONE));
+                    if (e == n - 1) ptx::umma_commit(bar(DQ_DONE));
                 }
                 __syncwarp();
             }
+            ++k;
         }
     } else if (warp >= 4) {
         // -------------------------------------------------------------- compute groups
         ptx::setmaxnreg_inc<PA_BWD_REG_COMP>();
         const int wg = (warp - 4) >> 2, quad = warp & 3;
         const int row = quad * 32 + lane, qrow = row & 63;
-        const int head_local = 2 * hp + (row >> 6);
-        const int head = hk * a.G + head_local;
-        const int64_t q = (int64_t)i * kBwdBlk + qrow;
-        const bool valid = head_local < a.G && q < a.N;
-        float lse2 = INFINITY, delta = 0.f;
-        if (valid) {
-            const float lse = a.lse[((int64_t)b * a.Hq + head) * a.N + q];
-            // (a row the layout left empty has no weights: P = 0)
-            lse2 = (lse == -INFINITY || lse == INFINITY) ? INFINITY : lse * 1.4426950408889634f;
-            delta = a.delta[((int64_t)b * a.Hq + head) * a.N + q];
-        }
-        const bool last_is_diag = n > 0 && __ldg(a.col_idx + e0 + n - 1) == i;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
+        // An item's row data for this thread: output row, LSE (base 2), delta, whether the row ends on
+        // its diagonal block.  Fetched one item ahead, so the loads are not waited for at an item's start.
+        struct RowData {
+            DqItem w;
+            float lse2, delta;
+            bool valid, last_is_diag;
+            int64_t out;
+        };
+        auto fetch = [&](uint32_t it) {
+            RowData r;
+            r.w.n = -1;
+            r.lse2 = INFINITY;
+            r.delta = 0.f;
+            r.valid = r.last_is_diag = false;
+            r.out = 0;
+            if (it >= n_items) return r;
+            r.w = dq_item(a, it);
+            const int head_local = 2 * r.w.hp + (row >> 6);
+            const int head = r.w.hk * a.G + head_local;
+            const int64_t q = (int64_t)r.w.i * kBwdBlk + qrow;
+            r.valid = head_local < a.G && q < a.N;
+            r.out = (((int64_t)r.w.b * a.N + q) * a.Hq + head) * D + 64 * wg;
+            if (r.valid) {
+                const int64_t at = ((int64_t)r.w.b * a.Hq + head) * a.N + q;
+                const float lse = __ldg(a.lse + at);
+                // (a row the layout left empty has no weights: P = 0)
+                r.lse2 = (lse == -INFINITY || lse == INFINITY) ? INFINITY : lse * 1.4426950408889634f;
+                r.delta = __ldg(a.delta + at);
+            }
+            r.last_is_diag = r.w.n > 0 && __ldg(a.col_idx + r.w.e0 + r.w.n - 1) == r.w.i;
+            return r;
+        };
+        uint32_t c = 0, k = 0;
         bool ok = true;
-        for (int e = wg; e < n; e += 2) {
-            ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_SD_FULL + wg), (e >> 1) & 1, 6));
+        RowData next = fetch(blockIdx.x);
+        for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+            const RowData r = next;
+            next = fetch(it + gridDim.x);
+            float *dst = a.dq + r.out;
+            const int n = r.w.n;
+            if (n <= 0) {
+                if (r.valid)
+                    for (int x = 0; x < 64; x += 4) *reinterpret_cast<float4 *>(dst + x) = make_float4(0.f, 0.f, 0.f, 0.f);
+                continue;
+            }
+            const float lse2 = r.lse2, delta = r.delta;
+            for (int e = 0; e < n; ++e, ++c) {
+                if ((int)(c & 1) != wg) continue;
+                ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_SD_FULL + wg), (c >> 1) & 1, 8));
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                uint32_t s[64], dp[64];
+                ptx::tmem_ld32(t_lane + 160 * wg, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+                ptx::tmem_ld32(t_lane + 160 * wg + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+                ptx::tmem_ld32(t_lane + 160 * wg + 64, *reinterpret_cast<uint32_t(*)[32]>(&dp[0]));
+                ptx::tmem_ld32(t_lane + 160 * wg + 96, *reinterpret_cast<uint32_t(*)[32]>(&dp[32]));
+                ptx::tmem_wait_ld();
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(DQ_S_TAKEN + wg));
+                // Algorithm 1's causal term acts inside the diagonal pair only (the row's last block).
+                const int lim = (r.last_is_diag && e == n - 1) ? qrow : 63;
+                uint32_t pk[32];
+#pragma unroll
+                for (int x = 0; x < 64; x += 2) {
+                    float ds[2];
+#pragma unroll
+                    for (int y = 0; y < 2; ++y) {
+                        const float p = (x + y <= lim) ? ptx::ex2(fmaf(__uint_as_float(s[x + y]), a.scale_log2, -lse2)) : 0.f;
+                        ds[y] = p * (__uint_as_float(dp[x + y]) - delta);
+                    }
+                    pk[x >> 1] = ptx::cvt_bf16x2(ds[0], ds[1]);
+                }
+                if (c >= 2) {
+                    ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_DS_FREE + wg), ((c >> 1) - 1) & 1, 9));
+                    if (!ok) break;
+                }
+                ptx::tmem_st32(t_lane + 160 * wg + 128, pk);
+                ptx::tmem_wait_st();
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(DQ_DS_FULL + wg));
+            }
+            if (!ok) break;
+            // dQ = scale x the accumulator: group 0 writes features 0..63 of its rows, group 1 the rest.
+            ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_DONE), k & 1, 10));
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            uint32_t s[64], dp[64];
-            ptx::tmem_ld32(t_lane + 160 * wg, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-            ptx::tmem_ld32(t_lane + 160 * wg + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-            ptx::tmem_ld32(t_lane + 160 * wg + 64, *reinterpret_cast<uint32_t(*)[32]>(&dp[0]));
-            ptx::tmem_ld32(t_lane + 160 * wg + 96, *reinterpret_cast<uint32_t(*)[32]>(&dp[32]));
+            uint32_t acc[2][32];
+            ptx::tmem_ld32(t_lane + kColDq + 64 * wg, acc[0]);
+            ptx::tmem_ld32(t_lane + kColDq + 64 * wg + 32, acc[1]);
             ptx::tmem_wait_ld();
+            // dQ is in registers: tensor memory may take the next item's first dS K.
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar(DQ_S_TAKEN + wg));
-            // Algorithm 1's causal term acts inside the diagonal pair only (the row's last block).
-            const int lim = (last_is_diag && e == n - 1) ? qrow : 63;
-            uint32_t pk[32];
+            if (lane == 0) ptx::mbar_arrive(bar(DQ_FREE));
+            if (r.valid) {
 #pragma unroll
-            for (int c = 0; c < 64; c += 2) {
-                float ds[2];
+                for (int ch = 0; ch < 2; ++ch)
 #pragma unroll
-                for (int x = 0; x < 2; ++x) {
-                    const float p = (c + x <= lim) ? ptx::ex2(fmaf(__uint_as_float(s[c + x]), a.scale_log2, -lse2)) : 0.f;
-                    ds[x] = p * (__uint_as_float(dp[c + x]) - delta);
-                }
-                pk[c >> 1] = ptx::cvt_bf16x2(ds[0], ds[1]);
+                    for (int x = 0; x < 32; x += 4)
+                        *reinterpret_cast<float4 *>(dst + 32 * ch + x) =
+                            make_float4(__uint_as_float(acc[ch][x]) * a.scale, __uint_as_float(acc[ch][x + 1]) * a.scale,
+                                        __uint_as_float(acc[ch][x + 2]) * a.scale, __uint_as_float(acc[ch][x + 3]) * a.scale);
             }
-            if (e >= 2) {
-                ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_DS_FREE + wg), ((e >> 1) - 1) & 1, 7));
-                if (!ok) break;
-            }
-            ptx::tmem_st32(t_lane + 160 * wg + 128, pk);
-            ptx::tmem_wait_st();
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar(DQ_DS_FULL + wg));
-        }
-        // dQ = scale x the accumulator: group 0 writes features 0..63 of its rows, group 1 the rest.
-        float *dst = a.dq + (((int64_t)b * a.N + q) * a.Hq + head) * D + 64 * wg;
-        if (n > 0) {
-            if (ok) ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_DONE), 0, 8));
-            if (ok) {
-                ptx::tc_fence_after_sync();
-#pragma unroll
-                for (int ch = 0; ch < 2; ++ch) {
-                    uint32_t acc[32];
-                    ptx::tmem_ld32(t_lane + kColDq + 64 * wg + 32 * ch, acc);
-                    ptx::tmem_wait_ld();
-                    if (valid) {
-#pragma unroll
-                        for (int c = 0; c < 32; c += 4)
-                            *reinterpret_cast<float4 *>(dst + 32 * ch + c) =
-                                make_float4(__uint_as_float(acc[c]) * a.scale, __uint_as_float(acc[c + 1]) * a.scale,
-                                            __uint_as_float(acc[c + 2]) * a.scale, __uint_as_float(acc[c + 3]) * a.scale);
-                    }
-                }
-            }
-        } else if (valid) {
-            for (int c = 0; c < 64; c += 4) *reinterpret_cast<float4 *>(dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+            ++k;
         }
     }
 
@@ -594,7 +677,8 @@ dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 }
 
 // ---------------------------------------------------------------------------------- host side
-pa_status launch_backward_sm100(const BackwardArgs &args, const pa_prefill_params *p, int64_t nnz, int device, cudaStream_t st)
+pa_status launch_backward_sm100(const BackwardArgs &args, const pa_prefill_params *p, int64_t nnz, int device, int sms,
+                                cudaStream_t st)
 {
     BackwardArgs a = args;
     a.npairs = (a.G + 1) / 2;
@@ -618,8 +702,9 @@ pa_status launch_backward_sm100(const BackwardArgs &args, const pa_prefill_param
             return fail(PA_ERR_CUDA, "cudaFuncSetAttribute failed: %s", cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
         }
     }
-    if ((int64_t)a.Hkv * a.npairs > 65535) return fail(PA_ERR_SHAPE, "too many head pairs for one launch");
-    dq_kernel<<<dim3((unsigned)a.nqb, (unsigned)(a.Hkv * a.npairs), (unsigned)a.batch), kTcThreads, DqSmem::kAlloc, st>>>(tmQ, tmG, tmK, tmV, a);
+    const int64_t n_items = (int64_t)a.nqb * a.Hkv * a.npairs * a.batch;
+    if (n_items > (int64_t)0x3fffffff) return fail(PA_ERR_SHAPE, "too many work items (%lld)", (long long)n_items);
+    dq_kernel<<<(unsigned)(n_items < sms ? n_items : sms), kTcThreads, DqSmem::kAlloc, st>>>(tmQ, tmG, tmK, tmV, a, (uint32_t)n_items);
     // (an upper bound on the number of chunks; CTAs beyond the real count return at once)
     const int64_t max_chunks = nnz / kBwdChunk + a.nqb;
     dkv_kernel<<<dim3((unsigned)max_chunks, (unsigned)a.Hkv, (unsigned)a.batch), kTcThreads, DkvSmem::kAlloc, st>>>(tmQ, tmG, tmK, tmV, a);
