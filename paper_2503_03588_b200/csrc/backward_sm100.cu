@@ -58,15 +58,17 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int a_mn, int b_
 // Steps are numbered through the CTA's whole run, so ring positions, buffers and barrier parities do
 // not care about item boundaries.  Q and dO have one buffer: the next item's tiles are requested when
 // the current item's last S and dP have been issued and arrive while its last steps are computed
-// and its dQ leaves tensor memory, which takes longer; the K / V ring of five stages covers a
-// stage's life from request to the dQ product that reads it last (about four steps).
-constexpr int kDqStages = 5;  // K + V ring
+// and its dQ leaves tensor memory, which takes longer; the K / V ring of four stages covers a
+// stage's life from request to the dQ product that reads it last.
+constexpr int kDqStages = 4;  // K + V ring
+constexpr uint32_t kDqOutPitch = 80;  // bytes per staged row of 16 fp32 (conflict-free 16-byte stores, 4-byte loads)
 struct DqSmem {
     static constexpr uint32_t kQG = 0;                      // Q (two halves of 128 rows x 128 B), then dO
     static constexpr uint32_t kItem = 4 * kRowTile;
     static constexpr uint32_t kKV = kQG + kItem;            // stage: K (two halves), then V
     static constexpr uint32_t kStage = 4 * kKeyTile;
-    static constexpr uint32_t kBars = kKV + kDqStages * kStage;
+    static constexpr uint32_t kOut = kKV + kDqStages * kStage;  // per compute warp: 32 rows x 16 fp32 of dQ on their way out
+    static constexpr uint32_t kBars = kOut + 8 * 32 * kDqOutPitch;
     static constexpr uint32_t kAlloc = kBars + 512 + 1024;
     static_assert(kAlloc <= 227 * 1024, "shared memory budget");
 };
@@ -362,14 +364,32 @@ dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar(DQ_FREE));
-            if (r.valid) {
+            // A thread holds 64 features of its own row: stored from here, every instruction would touch
+            // 32 rows (32 memory transactions for 512 bytes, and the shared-memory pipe they block is the
+            // one the barrier waits of all roles go through).  The warp turns 16 features at a time
+            // through its shared-memory patch, so that an instruction writes two rows' 64 contiguous bytes.
+            {
+                const uint32_t patch = smem_base + SM::kOut + (uint32_t)(warp - 4) * 32u * kDqOutPitch;
+                const int64_t out0 = __shfl_sync(0xffffffffu, r.out, 0);  // lane 0's row; the warp's rows follow at Hq D
+                const int64_t q0 = (int64_t)r.w.i * kBwdBlk + (quad & 1) * 32;
+                const bool head_ok = 2 * r.w.hp + (quad >> 1) < a.G;
+                const int sub = lane >> 4, col = lane & 15;
 #pragma unroll
-                for (int ch = 0; ch < 2; ++ch)
+                for (int blk = 0; blk < 4; ++blk) {
 #pragma unroll
-                    for (int x = 0; x < 32; x += 4)
-                        *reinterpret_cast<float4 *>(dst + 32 * ch + x) =
-                            make_float4(__uint_as_float(acc[ch][x]) * a.scale, __uint_as_float(acc[ch][x + 1]) * a.scale,
-                                        __uint_as_float(acc[ch][x + 2]) * a.scale, __uint_as_float(acc[ch][x + 3]) * a.scale);
+                    for (int x = 0; x < 16; x += 4) {
+                        const uint32_t *v = &acc[blk >> 1][16 * (blk & 1) + x];
+                        ptx::st_shared_v4(patch + (uint32_t)lane * kDqOutPitch + 4u * x, v[0], v[1], v[2], v[3]);
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int rr = 0; rr < 16; ++rr) {
+                        const int rho = 2 * rr + sub;
+                        const float v = *reinterpret_cast<const float *>(smem + SM::kOut + ((warp - 4) * 32 + rho) * kDqOutPitch + 4 * col);
+                        if (head_ok && q0 + rho < a.N) a.dq[out0 + (int64_t)rho * a.Hq * D + 16 * blk + col] = v * a.scale;
+                    }
+                    __syncwarp();
+                }
             }
             ++k;
         }

@@ -42,8 +42,8 @@ def _run(pa, oracle, N, Hq, Hkv, D, W, S, batch=1, use_power=True, k_scale=1.0, 
     Qd, Kd, Vd, dOd = Q.cuda(), K.cuda(), V.cuda(), dO.cuda()
     o, lse, ws = pa.pa_prefill(Qd, Kd, Vd, rp, ci, softmax_scale=scale)
     pa.pa_prefill_status(ws)
-    dq, dk, dv, _ = pa.pa_prefill_backward(Qd, Kd, Vd, o, lse, dOd, rp, ci, softmax_scale=scale)
-    torch.cuda.synchronize()
+    dq, dk, dv, wsb = pa.pa_prefill_backward(Qd, Kd, Vd, o, lse, dOd, rp, ci, softmax_scale=scale)
+    pa.pa_prefill_status(wsb)   # the backward workspace starts with the same status block; synchronises
     rq, rk, rv = oracle.backward(Q, K, V, dO, 64, W, S, scale=scale if scale else None, use_power=use_power)
     what = f"N={N} Hq={Hq} Hkv={Hkv} D={D} W={W} S={S}"
     return [_compare(g, r, f"{n} {what}") for g, r, n in ((dq, rq, "dQ"), (dk, rk, "dK"), (dv, rv, "dV"))]
@@ -73,6 +73,66 @@ def test_backward_sliding_window_layout(pa, oracle):
     _run(pa, oracle, 1100, 8, 2, 128, 4, 1, use_power=False, seed=6)
 
 
+@pytest.mark.parametrize("N,Hq,Hkv,W,S", [
+    (1000, 7, 1, 5, 1),      # a 7-head group: four head pairs, the last with a padding head
+    (2100, 3, 3, 2, 0),      # one query head per KV head: every pair has a padding head
+    (4200, 8, 2, 5, 1),      # the sink column in three chunks
+])
+def test_backward_head_dim_128_on_the_warp_level_kernels(pa, pa_env, oracle, N, Hq, Hkv, W, S):
+    """head_dim 128 takes the tcgen05 kernels by default; PA_BACKWARD_PATH=mma sends it through the
+    warp-level MMA kernels that head_dim 64 uses.  Both meet the oracle."""
+    _run(pa, oracle, N, Hq, Hkv, 128, W, S, seed=N)
+    pa_env(PA_BACKWARD_PATH="mma")
+    _run(pa, oracle, N, Hq, Hkv, 128, W, S, seed=N)
+
+
+def test_backward_many_items_per_cta(pa, oracle):
+    """12K tokens x 8 heads x batch 2: 1500 (query block, head pair) items for the persistent dQ
+    kernel, several per CTA with rows of every length, and dK / dV columns in one to six chunks;
+    dK and dV are checked on sampled keys."""
+    N, Hq, Hkv, D, W, S = 12000, 8, 2, 128, 3, 1
+    Q, K, V = (si.bf16_randn((2, N, h, D), 1200 + i) for i, h in enumerate((Hq, Hkv, Hkv)))
+    dO = si.bf16_randn((2, N, Hq, D), 1204)
+    rp, ci = pa.pa_build_layout(N, 64, W, S)
+    Qd, Kd, Vd, dOd = Q.cuda(), K.cuda(), V.cuda(), dO.cuda()
+    o, lse, ws = pa.pa_prefill(Qd, Kd, Vd, rp, ci)
+    pa.pa_prefill_status(ws)
+    dq, dk, dv, wsb = pa.pa_prefill_backward(Qd, Kd, Vd, o, lse, dOd, rp, ci)
+    pa.pa_prefill_status(wsb)
+    keys = sorted({0, 63, 64, N - 1, 4095, 4096} | {int(x) for x in np.random.default_rng(1205).integers(0, N, 20)})
+    rq, rk, rv = oracle.backward(Q, K, V, dO, 64, W, S, key_rows=keys)
+    kidx = torch.as_tensor(keys).cuda()
+    _compare(dq, rq, "dQ 12K")
+    _compare(dk[:, kidx], rk[:, keys], "dK 12K")
+    _compare(dv[:, kidx], rv[:, keys], "dV 12K")
+
+
+def test_backward_wait_that_runs_out_ends_the_kernels_with_a_status(pa, oracle):
+    """The tcgen05 backward kernels bound every barrier wait like the prefill kernel.  With the limit
+    at one cycle an ordinary wait that is not over at its first try (the first tiles take microseconds
+    to arrive) runs out: the call returns, the status block at the head of the backward workspace
+    reports PA_ERR_TIMEOUT, and the next call, back at the default limit, is correct."""
+    N, Hq, Hkv, D, W, S = 3000, 8, 2, 128, 5, 1
+    Q, K, V = (si.bf16_randn((1, N, h, D), 1300 + i) for i, h in enumerate((Hq, Hkv, Hkv)))
+    dO = si.bf16_randn((1, N, Hq, D), 1304)
+    rp, ci = pa.pa_build_layout(N, 64, W, S)
+    Qd, Kd, Vd, dOd = Q.cuda(), K.cuda(), V.cuda(), dO.cuda()
+    o, lse, ws = pa.pa_prefill(Qd, Kd, Vd, rp, ci)
+    pa.pa_prefill_status(ws)
+    try:
+        pa.pa_set_wait_limit_cycles(1)
+        dq, dk, dv, wsb = pa.pa_prefill_backward(Qd, Kd, Vd, o, lse, dOd, rp, ci)
+        with pytest.raises(pa.PaError, match="PA_ERR_TIMEOUT"):
+            pa.pa_prefill_status(wsb)
+    finally:
+        pa.pa_set_wait_limit_cycles(0)
+    dq, dk, dv, wsb = pa.pa_prefill_backward(Qd, Kd, Vd, o, lse, dOd, rp, ci)
+    assert pa.pa_prefill_status(wsb) == 0
+    rq, rk, rv = oracle.backward(Q, K, V, dO, 64, W, S)
+    for g, r, n in ((dq, rq, "dQ"), (dk, rk, "dK"), (dv, rv, "dV")):
+        _compare(g, r, n + " after a timed-out call")
+
+
 def test_backward_at_16k_on_sampled_keys(pa, oracle):
     """A sweep-sized case: 16K tokens with the 7B-like heads.  The oracle evaluates dQ on every row
     (its first pass covers them all anyway) and dK, dV on sampled key positions: the sink block (its
@@ -84,8 +144,8 @@ def test_backward_at_16k_on_sampled_keys(pa, oracle):
     Qd, Kd, Vd, dOd = Q.cuda(), K.cuda(), V.cuda(), dO.cuda()
     o, lse, ws = pa.pa_prefill(Qd, Kd, Vd, rp, ci)
     pa.pa_prefill_status(ws)
-    dq, dk, dv, _ = pa.pa_prefill_backward(Qd, Kd, Vd, o, lse, dOd, rp, ci)
-    torch.cuda.synchronize()
+    dq, dk, dv, wsb = pa.pa_prefill_backward(Qd, Kd, Vd, o, lse, dOd, rp, ci)
+    pa.pa_prefill_status(wsb)
     keys = sorted({0, 1, 63, 64, 65, N - 1, N - 64, N - 65, 8191, 8192, 12288 + 17}
                   | {int(x) for x in np.random.default_rng(1105).integers(0, N, 24)})
     rq, rk, rv = oracle.backward(Q, K, V, dO, 64, W, S, key_rows=keys)
