@@ -1,21 +1,22 @@
 // Backward pass of the block-sparse attention (derivatives of Eq. (1), Section 3.1, under the
 // key-block lists of Algorithm 1, Section 3.3) on the sm_100a tensor cores, head_dim 128.
 //
-// Two kernels, both with the same skeleton of 384 threads:
+// Two kernels with the same skeleton:
 //   warp 0       TMA producer (bf16 tiles, 128-byte swizzle, into rings of shared-memory stages)
-//   warp 1       tcgen05 issuer of S and dP (one elected lane)
-//   warp 2       tensor-memory allocation
+//   warp 1       tcgen05 issuer of S and dP (one elected lane; the dQ kernel: of S)
+//   warp 2       tensor-memory allocation (the dQ kernel: and issuer of dP)
 //   warp 3       tcgen05 issuer of the second products
 //   warps 4-7    compute group 0: even steps
 //   warps 8-11   compute group 1: odd steps
+//   warps 12-15  (dQ kernel) epilogue: the finished dQ out of tensor memory and out to global memory
 // A step is one (query block, key block) pair for a pair of query heads stacked on the 64 tokens of
 // the query block: a 128-row tile, as in the forward kernel.  Per step the tensor cores produce
 // S = Q K^T and dP = dO V^T (128 x 64, fp32, tensor memory, two buffers: one per compute group); the
 // group's threads (thread = tile row = TMEM lane) turn them into P = exp2(S scale log2e - LSE log2e)
 // and dS = P (dP - delta), rounded to bf16; the second products accumulate in tensor memory.
 //
-//   dq_kernel   one CTA per (query block, head pair): walks the row's key blocks; dS goes back into
-//               tensor memory as the A operand of dQ += dS K (128 x 128 accumulator)
+//   dq_kernel   persistent; an item is a (query block, head pair): walks the row's key blocks; dS goes
+//               back into tensor memory as the A operand of dQ += dS K (128 x 128 accumulator)
 //   dkv_kernel  one CTA per (chunk of a key block's listing query blocks, KV head): walks the chunk
 //               for every head pair of the group; P and dS go to shared memory as the B operands of
 //               dV^T += dO^T P and dK^T += Q^T dS (feature x key accumulators, 128 x 64 each: the A
@@ -32,14 +33,19 @@
 #include "sm100_ptx.cuh"
 #include "tensor_map.cuh"
 
+// Registers per thread by role.  A warpgroup asking for more than the pool holds would wait for ever:
+// the dK / dV kernel starts 384 threads x 168, the dQ kernel (with its epilogue warps) 512 x 128.
 #define PA_BWD_REG_CTRL 56
 #define PA_BWD_REG_COMP 216
-// A warpgroup asking for more than the pool holds would wait for ever: 384 threads x 168 at launch.
 static_assert(4 * PA_BWD_REG_CTRL + 8 * PA_BWD_REG_COMP <= 12 * 168, "register split exceeds the CTA's registers");
+#define PA_DQ_REG_COMP 144
+#define PA_BWD_REG_EPI 168
+static_assert(4 * PA_BWD_REG_CTRL + 8 * PA_DQ_REG_COMP + 4 * PA_BWD_REG_EPI <= 16 * 128, "register split exceeds the CTA's registers");
 
 namespace pa {
 
 constexpr int kTcThreads = 384;
+constexpr int kDqThreads = 512;  // + four epilogue warps
 constexpr uint32_t kTcTmemCols = 512;
 constexpr long long kBwdWaitCycles = 4000000000ll;
 constexpr uint32_t kRowTile = 128 * 128;   // 128 rows x 64 features: one 128-byte-wide half of a Q or dO tile
@@ -61,14 +67,14 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int a_mn, int b_
 // and its dQ leaves tensor memory, which takes longer; the K / V ring of four stages covers a
 // stage's life from request to the dQ product that reads it last.
 constexpr int kDqStages = 4;  // K + V ring
-constexpr uint32_t kDqOutPitch = 80;  // bytes per staged row of 16 fp32 (conflict-free 16-byte stores, 4-byte loads)
+constexpr uint32_t kDqOutPitch = 144;  // bytes per staged row of 32 fp32 (conflict-free 16-byte stores, 4-byte loads)
 struct DqSmem {
     static constexpr uint32_t kQG = 0;                      // Q (two halves of 128 rows x 128 B), then dO
     static constexpr uint32_t kItem = 4 * kRowTile;
     static constexpr uint32_t kKV = kQG + kItem;            // stage: K (two halves), then V
     static constexpr uint32_t kStage = 4 * kKeyTile;
-    static constexpr uint32_t kOut = kKV + kDqStages * kStage;  // per compute warp: 32 rows x 16 fp32 of dQ on their way out
-    static constexpr uint32_t kBars = kOut + 8 * 32 * kDqOutPitch;
+    static constexpr uint32_t kOut = kKV + kDqStages * kStage;  // per epilogue warp: 32 rows x 32 fp32 of dQ on their way out
+    static constexpr uint32_t kBars = kOut + 4 * 32 * kDqOutPitch;
     static constexpr uint32_t kAlloc = kBars + 512 + 1024;
     static_assert(kAlloc <= 227 * 1024, "shared memory budget");
 };
@@ -80,7 +86,7 @@ enum : uint32_t {
     DQ_DS_FULL = DQ_S_TAKEN + 2,            // [buffer]: dS is in tensor memory
     DQ_DS_FREE = DQ_DS_FULL + 2,            // [buffer]: dQ += dS K has read it
     DQ_DONE = DQ_DS_FREE + 2,               // the item's last dQ += dS K has completed
-    DQ_FREE = DQ_DONE + 1,                  // the compute groups have read dQ out of tensor memory
+    DQ_FREE = DQ_DONE + 1,                  // the epilogue warps have read dQ out of tensor memory
     DQ_BAR_COUNT = DQ_FREE + 1
 };
 
@@ -104,7 +110,7 @@ __device__ __forceinline__ DqItem dq_item(const BackwardArgs &a, uint32_t it)
     return w;
 }
 
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kDqThreads, 1)
 dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmG,
           const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const BackwardArgs a,
           const uint32_t n_items)
@@ -137,7 +143,7 @@ dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             ptx::mbar_init(bar(DQ_KV_EMPTY + s), 1);
         }
         ptx::mbar_init(bar(DQ_DONE), 1);
-        ptx::mbar_init(bar(DQ_FREE), 8);
+        ptx::mbar_init(bar(DQ_FREE), 4);
         *abort_flag = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
@@ -262,35 +268,37 @@ dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             }
             ++k;
         }
-    } else if (warp >= 4) {
+    } else if (warp >= 4 && warp < 12) {
         // -------------------------------------------------------------- compute groups
-        ptx::setmaxnreg_inc<PA_BWD_REG_COMP>();
+        ptx::setmaxnreg_inc<PA_DQ_REG_COMP>();
         const int wg = (warp - 4) >> 2, quad = warp & 3;
         const int row = quad * 32 + lane, qrow = row & 63;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
-        // An item's row data for this thread: output row, LSE (base 2), delta, whether the row ends on
-        // its diagonal block.  Fetched one item ahead, so the loads are not waited for at an item's start.
+        // An item's row data for this thread: LSE (base 2), delta, whether the row ends on its diagonal
+        // block.  Fetched one item ahead, so the loads are not waited for at an item's start (the item's
+        // coordinates, which need the row extents, one item earlier still).
         struct RowData {
             DqItem w;
             float lse2, delta;
-            bool valid, last_is_diag;
-            int64_t out;
+            bool last_is_diag;
         };
-        auto fetch = [&](uint32_t it) {
+        auto fetch_item = [&](uint32_t it) {
+            DqItem w = {};
+            w.n = -1;
+            if (it < n_items) w = dq_item(a, it);
+            return w;
+        };
+        auto fetch = [&](uint32_t it, const DqItem &w) {
             RowData r;
-            r.w.n = -1;
+            r.w = w;
             r.lse2 = INFINITY;
             r.delta = 0.f;
-            r.valid = r.last_is_diag = false;
-            r.out = 0;
+            r.last_is_diag = false;
             if (it >= n_items) return r;
-            r.w = dq_item(a, it);
             const int head_local = 2 * r.w.hp + (row >> 6);
             const int head = r.w.hk * a.G + head_local;
             const int64_t q = (int64_t)r.w.i * kBwdBlk + qrow;
-            r.valid = head_local < a.G && q < a.N;
-            r.out = (((int64_t)r.w.b * a.N + q) * a.Hq + head) * D + 64 * wg;
-            if (r.valid) {
+            if (head_local < a.G && q < a.N) {
                 const int64_t at = ((int64_t)r.w.b * a.Hq + head) * a.N + q;
                 const float lse = __ldg(a.lse + at);
                 // (a row the layout left empty has no weights: P = 0)
@@ -300,46 +308,49 @@ dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             r.last_is_diag = r.w.n > 0 && __ldg(a.col_idx + r.w.e0 + r.w.n - 1) == r.w.i;
             return r;
         };
-        uint32_t c = 0, k = 0;
+        uint32_t c = 0;
         bool ok = true;
-        RowData next = fetch(blockIdx.x);
+        RowData next = fetch(blockIdx.x, fetch_item(blockIdx.x));
+        DqItem item2 = fetch_item(blockIdx.x + gridDim.x);
         for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
             const RowData r = next;
-            next = fetch(it + gridDim.x);
-            float *dst = a.dq + r.out;
+            next = fetch(it + gridDim.x, item2);
+            item2 = fetch_item(it + 2 * gridDim.x);
             const int n = r.w.n;
-            if (n <= 0) {
-                if (r.valid)
-                    for (int x = 0; x < 64; x += 4) *reinterpret_cast<float4 *>(dst + x) = make_float4(0.f, 0.f, 0.f, 0.f);
-                continue;
-            }
+            if (n <= 0) continue;
             const float lse2 = r.lse2, delta = r.delta;
             for (int e = 0; e < n; ++e, ++c) {
                 if ((int)(c & 1) != wg) continue;
                 ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_SD_FULL + wg), (c >> 1) & 1, 8));
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                uint32_t s[64], dp[64];
-                ptx::tmem_ld32(t_lane + 160 * wg, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-                ptx::tmem_ld32(t_lane + 160 * wg + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-                ptx::tmem_ld32(t_lane + 160 * wg + 64, *reinterpret_cast<uint32_t(*)[32]>(&dp[0]));
-                ptx::tmem_ld32(t_lane + 160 * wg + 96, *reinterpret_cast<uint32_t(*)[32]>(&dp[32]));
-                ptx::tmem_wait_ld();
-                ptx::tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(bar(DQ_S_TAKEN + wg));
                 // Algorithm 1's causal term acts inside the diagonal pair only (the row's last block).
                 const int lim = (r.last_is_diag && e == n - 1) ? qrow : 63;
                 uint32_t pk[32];
+                // Two halves of 32 keys, so that the logits of one half only are held at a time.
 #pragma unroll
-                for (int x = 0; x < 64; x += 2) {
-                    float ds[2];
-#pragma unroll
-                    for (int y = 0; y < 2; ++y) {
-                        const float p = (x + y <= lim) ? ptx::ex2(fmaf(__uint_as_float(s[x + y]), a.scale_log2, -lse2)) : 0.f;
-                        ds[y] = p * (__uint_as_float(dp[x + y]) - delta);
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t s[32], dp[32];
+                    ptx::tmem_ld32(t_lane + 160 * wg + 32 * half, s);
+                    ptx::tmem_ld32(t_lane + 160 * wg + 64 + 32 * half, dp);
+                    ptx::tmem_wait_ld();
+                    if (half == 1) {
+                        // S and dP are in registers: their buffer may take the step after next.
+                        ptx::tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(bar(DQ_S_TAKEN + wg));
                     }
-                    pk[x >> 1] = ptx::cvt_bf16x2(ds[0], ds[1]);
+#pragma unroll
+                    for (int x = 0; x < 32; x += 2) {
+                        float ds[2];
+#pragma unroll
+                        for (int y = 0; y < 2; ++y) {
+                            const float p = (32 * half + x + y <= lim)
+                                                ? ptx::ex2(fmaf(__uint_as_float(s[x + y]), a.scale_log2, -lse2)) : 0.f;
+                            ds[y] = p * (__uint_as_float(dp[x + y]) - delta);
+                        }
+                        pk[16 * half + (x >> 1)] = ptx::cvt_bf16x2(ds[0], ds[1]);
+                    }
                 }
                 if (c >= 2) {
                     ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_DS_FREE + wg), ((c >> 1) - 1) & 1, 9));
@@ -351,45 +362,62 @@ dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(bar(DQ_DS_FULL + wg));
             }
-            if (!ok) break;
-            // dQ = scale x the accumulator: group 0 writes features 0..63 of its rows, group 1 the rest.
+        }
+    } else {
+        // -------------------------------------------------------------- epilogue
+        // dQ = scale x the accumulator, off the compute groups' path: writing an item's 64 KB out takes
+        // several thousand cycles (the SM's store path), which the next item's steps run beside.  The
+        // accumulator is read into registers in one go, which frees it for the next item at once.
+        ptx::setmaxnreg_inc<PA_BWD_REG_EPI>();
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane, qrow = row & 63;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const uint32_t patch = smem_base + SM::kOut + (uint32_t)quad * 32u * kDqOutPitch;
+        const uint8_t *patch_ptr = smem + SM::kOut + quad * 32 * kDqOutPitch;
+        uint32_t k = 0;
+        bool ok = true;
+        for (uint32_t it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+            const DqItem w = dq_item(a, it);
+            const int head_local = 2 * w.hp + (row >> 6);
+            const bool head_ok = head_local < a.G;
+            const int64_t q = (int64_t)w.i * kBwdBlk + qrow;
+            const int64_t out = (((int64_t)w.b * a.N + q) * a.Hq + w.hk * a.G + head_local) * D;
+            if (w.n <= 0) {  // empty row: zero gradient, no barrier traffic
+                if (head_ok && q < a.N)
+                    for (int x = 0; x < D; x += 4) *reinterpret_cast<float4 *>(a.dq + out + x) = make_float4(0.f, 0.f, 0.f, 0.f);
+                continue;
+            }
             ok = __all_sync(0xffffffffu, wait_bar(bar(DQ_DONE), k & 1, 10));
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            uint32_t acc[2][32];
-            ptx::tmem_ld32(t_lane + kColDq + 64 * wg, acc[0]);
-            ptx::tmem_ld32(t_lane + kColDq + 64 * wg + 32, acc[1]);
+            uint32_t acc[4][32];
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) ptx::tmem_ld32(t_lane + kColDq + 32 * ch, acc[ch]);
             ptx::tmem_wait_ld();
             // dQ is in registers: tensor memory may take the next item's first dS K.
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar(DQ_FREE));
-            // A thread holds 64 features of its own row: stored from here, every instruction would touch
-            // 32 rows (32 memory transactions for 512 bytes, and the shared-memory pipe they block is the
-            // one the barrier waits of all roles go through).  The warp turns 16 features at a time
-            // through its shared-memory patch, so that an instruction writes two rows' 64 contiguous bytes.
-            {
-                const uint32_t patch = smem_base + SM::kOut + (uint32_t)(warp - 4) * 32u * kDqOutPitch;
-                const int64_t out0 = __shfl_sync(0xffffffffu, r.out, 0);  // lane 0's row; the warp's rows follow at Hq D
-                const int64_t q0 = (int64_t)r.w.i * kBwdBlk + (quad & 1) * 32;
-                const bool head_ok = 2 * r.w.hp + (quad >> 1) < a.G;
-                const int sub = lane >> 4, col = lane & 15;
+            // A thread holds its own row: stored from here, every instruction would touch 32 rows.  The
+            // warp turns 32 features at a time through its shared-memory patch, so that an instruction
+            // writes one row's 128 contiguous bytes.
+            const int64_t out0 = __shfl_sync(0xffffffffu, out, 0);  // lane 0's row; the warp's rows follow at Hq D
+            const int64_t q0 = __shfl_sync(0xffffffffu, q, 0);
 #pragma unroll
-                for (int blk = 0; blk < 4; ++blk) {
+            for (int ch = 0; ch < 4; ++ch) {
 #pragma unroll
-                    for (int x = 0; x < 16; x += 4) {
-                        const uint32_t *v = &acc[blk >> 1][16 * (blk & 1) + x];
-                        ptx::st_shared_v4(patch + (uint32_t)lane * kDqOutPitch + 4u * x, v[0], v[1], v[2], v[3]);
-                    }
-                    __syncwarp();
+                for (int x = 0; x < 32; x += 4)
+                    ptx::st_shared_v4(patch + (uint32_t)lane * kDqOutPitch + 4u * x, acc[ch][x], acc[ch][x + 1], acc[ch][x + 2],
+                                      acc[ch][x + 3]);
+                __syncwarp();
+                // (all loads first: a load behind a global store would wait for it, the two might alias)
+                float v[32];
 #pragma unroll
-                    for (int rr = 0; rr < 16; ++rr) {
-                        const int rho = 2 * rr + sub;
-                        const float v = *reinterpret_cast<const float *>(smem + SM::kOut + ((warp - 4) * 32 + rho) * kDqOutPitch + 4 * col);
-                        if (head_ok && q0 + rho < a.N) a.dq[out0 + (int64_t)rho * a.Hq * D + 16 * blk + col] = v * a.scale;
-                    }
-                    __syncwarp();
-                }
+                for (int rho = 0; rho < 32; ++rho) v[rho] = *reinterpret_cast<const float *>(patch_ptr + rho * kDqOutPitch + 4 * lane);
+                __syncwarp();
+#pragma unroll
+                for (int rho = 0; rho < 32; ++rho)
+                    if (head_ok && q0 + rho < a.N) a.dq[out0 + (int64_t)rho * a.Hq * D + 32 * ch + lane] = v[rho] * a.scale;
             }
             ++k;
         }
@@ -724,7 +752,7 @@ pa_status launch_backward_sm100(const BackwardArgs &args, const pa_prefill_param
     }
     const int64_t n_items = (int64_t)a.nqb * a.Hkv * a.npairs * a.batch;
     if (n_items > (int64_t)0x3fffffff) return fail(PA_ERR_SHAPE, "too many work items (%lld)", (long long)n_items);
-    dq_kernel<<<(unsigned)(n_items < sms ? n_items : sms), kTcThreads, DqSmem::kAlloc, st>>>(tmQ, tmG, tmK, tmV, a, (uint32_t)n_items);
+    dq_kernel<<<(unsigned)(n_items < sms ? n_items : sms), kDqThreads, DqSmem::kAlloc, st>>>(tmQ, tmG, tmK, tmV, a, (uint32_t)n_items);
     // (an upper bound on the number of chunks; CTAs beyond the real count return at once)
     const int64_t max_chunks = nnz / kBwdChunk + a.nqb;
     dkv_kernel<<<dim3((unsigned)max_chunks, (unsigned)a.Hkv, (unsigned)a.batch), kTcThreads, DkvSmem::kAlloc, st>>>(tmQ, tmG, tmK, tmV, a);
