@@ -499,7 +499,7 @@ dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(bar(KV_QG_FULL + s), 1);
             ptx::mbar_init(bar(KV_QG_EMPTY + s), 1);
-            ptx::mbar_init(bar(KV_SD_FULL + s), 1);
+            ptx::mbar_init(bar(KV_SD_FULL + s), 2);  // one commit from each of the S and dP issuers
             ptx::mbar_init(bar(KV_S_TAKEN + s), 4);
             ptx::mbar_init(bar(KV_PD_FULL + s), 4);
             ptx::mbar_init(bar(KV_PD_FREE + s), 1);
@@ -549,36 +549,30 @@ dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
-        // -------------------------------------------------------------- tcgen05 issuer of S and dP
+    } else if (warp == 1 || warp == 2) {
+        // -------------------------------------------------------------- tcgen05 issuers of S (warp 1) and dP (warp 2)
         const bool leader = ptx::elect_one();
+        const bool is_dp = __shfl_sync(0xffffffffu, warp, 0) == 2;
         constexpr uint32_t idesc_s = idesc_bf16(128, 64, 0, 0);    // both operands K-major
-        const uint32_t k_lo = ((smem_base + SM::kK) >> 4) | (1u << 16);
-        const uint32_t v_lo = ((smem_base + SM::kV) >> 4) | (1u << 16);
+        // A = Q (S) or dO (dP) of the stage; B = the key block's K or V.
+        const uint32_t b_lo = ((smem_base + (is_dp ? SM::kV : SM::kK)) >> 4) | (1u << 16);
         bool ok = __all_sync(0xffffffffu, wait_bar(bar(KV_KV_FULL), 0, 1));
         for (int e = 0; e < n && ok; ++e) {
-            {
-                const uint32_t bf = e & 1;
-                ok = __all_sync(0xffffffffu, wait_bar(bar(KV_QG_FULL + bf), (e >> 1) & 1, 3));
-                if (ok && e >= 2) ok = __all_sync(0xffffffffu, wait_bar(bar(KV_S_TAKEN + bf), ((e >> 1) - 1) & 1, 4));
-                if (!ok) break;
-                ptx::tc_fence_after_sync();
-                if (leader) {
-                    const uint32_t q_lo = ((smem_base + SM::kQG + bf * SM::kStage) >> 4) | (1u << 16);
-                    const uint32_t g_lo = q_lo + ((2 * kRowTile) >> 4);
-                    const uint32_t t_s = tmem_base + 128 * bf, t_dp = t_s + 64;
+            const uint32_t bf = e & 1;
+            ok = __all_sync(0xffffffffu, wait_bar(bar(KV_QG_FULL + bf), (e >> 1) & 1, 3));
+            if (ok && e >= 2) ok = __all_sync(0xffffffffu, wait_bar(bar(KV_S_TAKEN + bf), ((e >> 1) - 1) & 1, 4));
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            if (leader) {
+                const uint32_t a_lo = ((smem_base + SM::kQG + bf * SM::kStage + (is_dp ? 2 * kRowTile : 0u)) >> 4) | (1u << 16);
+                const uint32_t t_d = tmem_base + 128 * bf + (is_dp ? 64u : 0u);
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk)
-                        ptx::umma_ss_lohi(t_s, q_lo + (((kk / 4) * kRowTile + (kk % 4) * 32) >> 4), kDescHi,
-                                          k_lo + (((kk / 4) * kKeyTile + (kk % 4) * 32) >> 4), kDescHi, idesc_s, kk > 0 ? 1u : 0u);
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk)
-                        ptx::umma_ss_lohi(t_dp, g_lo + (((kk / 4) * kRowTile + (kk % 4) * 32) >> 4), kDescHi,
-                                          v_lo + (((kk / 4) * kKeyTile + (kk % 4) * 32) >> 4), kDescHi, idesc_s, kk > 0 ? 1u : 0u);
-                    ptx::umma_commit(bar(KV_SD_FULL + bf));
-                }
-                __syncwarp();
+                for (int kk = 0; kk < D / 16; ++kk)
+                    ptx::umma_ss_lohi(t_d, a_lo + (((kk / 4) * kRowTile + (kk % 4) * 32) >> 4), kDescHi,
+                                      b_lo + (((kk / 4) * kKeyTile + (kk % 4) * 32) >> 4), kDescHi, idesc_s, kk > 0 ? 1u : 0u);
+                ptx::umma_commit(bar(KV_SD_FULL + bf));
             }
+            __syncwarp();
         }
     } else if (warp == 3) {
         // -------------------------------------------------------------- tcgen05 issuer of dV^T and dK^T
