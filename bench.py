@@ -474,7 +474,9 @@ def run_ours(args):
     backward_32k = dict(workload=w32.name, ms=msb, value=2.5 * flops32 / (msb * 1e-3) / 1e12, unit=UNIT,
                         frac=2.5 * flops32 / (msb * 1e-3) / 1e12 / peaks["bf16_tflops"], bound="tensor",
                         flops_per_pair_head=10 * w32.block * w32.block * w32.head_dim, launches=nb,
-                        kernels="delta, transposed layout (3), dQ, dK/dV: warp-level MMA (mma.sync), fp32 outputs")
+                        kernels="delta, transposed layout (4), dQ and dK/dV on tcgen05 with accumulators in tensor memory, "
+                                "fp32 outputs")
+    pa.pa_prefill_status(wsb32)
     del Q32, K32, V32, o32, lse32, dO32, dq32, dk32, dv32
 
     # ---- decode scale-up (labelled, beside the batch-8 figure): the same per-sequence pattern at
@@ -650,6 +652,18 @@ def run_case(args):
         for _ in range(args.steps):
             pa.pa_prefill(Q, K, V, rp, ci, o=o, lse=lse, workspace=ws)
         pa.pa_prefill_status(ws)
+    elif args.case == "backward32k":
+        w = si.PREFILL_32K
+        Q, K, V = (t.to(dev) for t in si.prefill_inputs(w))
+        rp, ci = pa.pa_build_layout(w.seq_len, w.block, w.window_blocks, w.sink_blocks)
+        o, lse, ws = pa.pa_prefill(Q, K, V, rp, ci)
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(w.seed + 9)
+        dO = torch.randn(o.shape, device=dev, dtype=torch.bfloat16, generator=gen)
+        dq, dk, dv, wsb = pa.pa_prefill_backward(Q, K, V, o, lse, dO, rp, ci)
+        for _ in range(args.steps):
+            pa.pa_prefill_backward(Q, K, V, o, lse, dO, rp, ci, dq=dq, dk=dk, dv=dv, workspace=wsb)
+        pa.pa_prefill_status(wsb)
     elif args.case == "decode_persist":
         # The persistent form of the decode row kernel on a case small enough for a full-set capture:
         # batch 96 (384 rows), 16K-token caches (1.6 GB), lengths uniform in [8192, 16384].
@@ -781,7 +795,7 @@ def main():
     ap.add_argument("--shard-heads", action="store_true",
                     help="with N > 1: split the one problem by KV heads over the ranks (strong scaling) instead of replicas")
     ap.add_argument("--no-decode-scale-up", action="store_true", help="skip the batch-64/256 decode lines")
-    ap.add_argument("--case", default=None, choices=["prefill32k", "decode", "decode_persist"],
+    ap.add_argument("--case", default=None, choices=["prefill32k", "backward32k", "decode", "decode_persist"],
                     help="run only a small single-kernel case (for profiler captures)")
     ap.add_argument("--sweep", action="store_true", help="sequence-length sweep with comparison layouts")
     ap.add_argument("--sweep-max-len", type=int, default=262144)
