@@ -615,31 +615,35 @@ dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         const int wg = (warp - 4) >> 2, quad = warp & 3;
         const int row = quad * 32 + lane, qrow = row & 63;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
-        // Row statistics of step e for this thread's row: LSE (base 2) and delta; +inf / 0 for a row
-        // without weights (beyond the sequence, padding head, empty row): P = 0.
-        auto load_stats = [&](int e, float &lse2, float &delta, bool &diag) {
-            lse2 = INFINITY;
+        // Row statistics of a step for this thread's row: LSE and delta; +inf / 0 for a row without
+        // weights (beyond the sequence, padding head, empty row): P = 0.  Nothing here uses a loaded
+        // value (the thread would wait for it on the spot): the query block index is loaded two of
+        // this group's steps ahead, LSE and delta one step ahead, and they are looked at when the step
+        // they belong to begins.
+        auto step_block = [&](int e) { return e < n ? __ldg(a.row_idx + e0 + e / a.npairs) : -1; };
+        auto request_stats = [&](int e, int32_t i, float &lse, float &delta, bool &diag) {
+            lse = INFINITY;
             delta = 0.f;
             diag = false;
             if (e >= n) return;
-            const int32_t i = __ldg(a.row_idx + e0 + e / a.npairs);
             const int head_local = 2 * (e % a.npairs) + (row >> 6);
             const int64_t q = (int64_t)i * kBwdBlk + qrow;
             diag = i == j;
             if (head_local < a.G && q < a.N) {
                 const int64_t at = ((int64_t)b * a.Hq + hk * a.G + head_local) * a.N + q;
-                const float lse = __ldg(a.lse + at);
-                lse2 = (lse == -INFINITY || lse == INFINITY) ? INFINITY : lse * 1.4426950408889634f;
+                lse = __ldg(a.lse + at);
                 delta = __ldg(a.delta + at);
             }
         };
-        float lse2, delta, lse2_n, delta_n;
+        float lse_raw, delta, lse_raw_n, delta_n;
         bool diag, diag_n;
-        load_stats(wg, lse2, delta, diag);
+        int32_t i_next = step_block(wg + 2);
+        request_stats(wg, step_block(wg), lse_raw, delta, diag);
         const uint32_t p_row = smem_base + SM::kPD + wg * SM::kBuf + (uint32_t)row * 128u;
         bool ok = true;
         for (int e = wg; e < n; e += 2) {
-            load_stats(e + 2, lse2_n, delta_n, diag_n);  // (in flight during this step)
+            const int32_t i_next2 = step_block(e + 4);
+            request_stats(e + 2, i_next, lse_raw_n, delta_n, diag_n);  // (in flight during this step)
             ok = __all_sync(0xffffffffu, wait_bar(bar(KV_SD_FULL + wg), (e >> 1) & 1, 6));
             if (!ok) break;
             ptx::tc_fence_after_sync();
@@ -658,6 +662,7 @@ dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
             // Algorithm 1's causal term acts inside the diagonal pair only.
             const int lim = diag ? qrow : 63;
+            const float lse2 = (lse_raw == -INFINITY || lse_raw == INFINITY) ? INFINITY : lse_raw * 1.4426950408889634f;
 #pragma unroll
             for (int ch = 0; ch < 8; ++ch) {
                 uint32_t pp[4], pd[4];
@@ -681,9 +686,10 @@ dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar(KV_PD_FULL + wg));
-            lse2 = lse2_n;
+            lse_raw = lse_raw_n;
             delta = delta_n;
             diag = diag_n;
+            i_next = i_next2;
         }
         // Group 0 adds dK^T (x scale), group 1 dV^T: thread = feature, one key per register.
         if (ok) ok = __all_sync(0xffffffffu, wait_bar(bar(KV_DONE), 0, 8));
