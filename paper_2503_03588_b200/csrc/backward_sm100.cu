@@ -457,9 +457,8 @@ enum : uint32_t {
     KV_SD_FULL = 5,                   // [buffer]: S and dP of a step are in tensor memory
     KV_S_TAKEN = 7,                   // [buffer]: the group has them in registers
     KV_PD_FULL = 9,                   // [buffer]: P and dS are in shared memory
-    KV_PD_FREE = 11,                  // [buffer]: the second products have read them
-    KV_DONE = 13,
-    KV_BAR_COUNT = 14
+    KV_DONE = 11,
+    KV_BAR_COUNT = 12
 };
 
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -502,7 +501,6 @@ dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             ptx::mbar_init(bar(KV_SD_FULL + s), 2);  // one commit from each of the S and dP issuers
             ptx::mbar_init(bar(KV_S_TAKEN + s), 4);
             ptx::mbar_init(bar(KV_PD_FULL + s), 4);
-            ptx::mbar_init(bar(KV_PD_FREE + s), 1);
         }
         ptx::mbar_init(bar(KV_DONE), 1);
         *abort_flag = 0;
@@ -602,8 +600,7 @@ dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     for (int kk = 0; kk < 8; ++kk)
                         ptx::umma_ss_lohi(tmem_base + kColDk, qa + ((kk * 2048) >> 4), kDescHi, db + ((kk * 2048) >> 4), kDescHi,
                                           idesc_t, (e1 > 0 || kk > 0) ? 1u : 0u);
-                    ptx::umma_commit(bar(KV_QG_EMPTY + bf));
-                    ptx::umma_commit(bar(KV_PD_FREE + bf));
+                    ptx::umma_commit(bar(KV_QG_EMPTY + bf));  // (frees the P / dS buffer as well)
                     if (e1 == n - 1) ptx::umma_commit(bar(KV_DONE));
                 }
                 __syncwarp();
@@ -656,10 +653,9 @@ dkv_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar(KV_S_TAKEN + wg));
-            if (e >= 2) {
-                ok = __all_sync(0xffffffffu, wait_bar(bar(KV_PD_FREE + wg), ((e >> 1) - 1) & 1, 7));
-                if (!ok) break;
-            }
+            // (The P / dS buffer is free: the second products of step e - 2 that read it had completed
+            // before this step's Q and dO could be loaded into the stage they also read, and so before
+            // the S and dP waited for above were issued.)
             // Algorithm 1's causal term acts inside the diagonal pair only.
             const int lim = diag ? qrow : 63;
             const float lse2 = (lse_raw == -INFINITY || lse_raw == INFINITY) ? INFINITY : lse_raw * 1.4426950408889634f;
