@@ -57,6 +57,8 @@ def _run(pa, oracle, N, Hq, Hkv, D, W, S, batch=1, use_power=True, k_scale=1.0, 
     (1536, 28, 4, 128, 5, 1),    # the 7B-like head shape
     (777, 8, 2, 64, 0, 0),       # pure power-of-two pattern
     (900, 6, 2, 128, 30, 2),     # window covers everything: dense causal
+    (130, 5, 1, 128, 2, 1),      # a 5-head group: three head pairs, the last with a padding head
+    (4097, 6, 3, 128, 7, 2),     # pairs only, one token in the last block
 ])
 def test_backward_small_shapes(pa, oracle, N, Hq, Hkv, D, W, S):
     _run(pa, oracle, N, Hq, Hkv, D, W, S, batch=2, seed=N)
