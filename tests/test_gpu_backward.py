@@ -154,3 +154,20 @@ def test_backward_at_16k_on_sampled_keys(pa, oracle):
     kidx = torch.as_tensor(keys).cuda()
     print("16K backward (max, mean):", _compare(dq, rq, "dQ 16K"), _compare(dk[:, kidx], rk[:, keys], "dK 16K"),
           _compare(dv[:, kidx], rv[:, keys], "dV 16K"))
+
+
+def test_backward_on_views_of_a_packed_qkv_tensor(pa, oracle):
+    """Q, K and V as head slices of one [batch, seq, Hq + 2 Hkv, D] tensor: the kernels take the
+    strides as given (the tensor maps of the tcgen05 kernels are built from them)."""
+    N, Hq, Hkv, D, W, S = 1300, 8, 2, 128, 3, 1
+    qkv = si.bf16_randn((2, N, Hq + 2 * Hkv, D), 1400).cuda()
+    q, k, v = qkv[:, :, :Hq], qkv[:, :, Hq:Hq + Hkv], qkv[:, :, Hq + Hkv:]
+    dO = si.bf16_randn((2, N, Hq, D), 1401)
+    rp, ci = pa.pa_build_layout(N, 64, W, S)
+    o, lse, ws = pa.pa_prefill(q, k, v, rp, ci)
+    pa.pa_prefill_status(ws)
+    dq, dk, dv, wsb = pa.pa_prefill_backward(q, k, v, o, lse, dO.cuda(), rp, ci)
+    pa.pa_prefill_status(wsb)
+    rq, rk, rv = oracle.backward(q.cpu().contiguous(), k.cpu().contiguous(), v.cpu().contiguous(), dO, 64, W, S)
+    for g, r, n in ((dq, rq, "dQ"), (dk, rk, "dK"), (dv, rv, "dV")):
+        _compare(g, r, n + " packed qkv")
