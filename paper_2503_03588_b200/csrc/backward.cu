@@ -5,7 +5,10 @@
 //     delta_i = <dO_i, O_i>                      dV_j = sum_i P_ij dO_i
 //     dS_ij = P_ij (<dO_i, v_j> - delta_i)       dQ_i = scale sum_j dS_ij k_j
 //                                                dK_j = scale sum_i dS_ij q_i
-// (dK and dV also sum over the query heads that share the KV head).  Four kernels:
+// (dK and dV also sum over the query heads that share the KV head).  This file holds the entry
+// point, the kernels common to every head size (delta, the transposed layout) and the attention kernels
+// for head_dim 64; head_dim 128 takes the tcgen05 kernels of the sibling file for the two attention
+// kernels.  The kernels here:
 //   backward_delta_kernel    delta = rowsum(dO * O)
 //   csc_count / csc_fill     the CSR transposed: for every key block the query blocks that list it
 //                            (a column walks the rows below it with a binary search each, so the lists
@@ -15,7 +18,7 @@
 //                            chunk for every query head of the group; a column listed by many rows
 //                            (the sink block is listed by all of them) is spread over many CTAs,
 //                            which add their parts into dK / dV with fp32 atomics
-// Both attention kernels recompute S and P tile by tile (64 queries x 64 keys) on the warp-level
+// Both attention kernels of this file recompute S and P tile by tile (64 queries x 64 keys) on the warp-level
 // tensor-core MMA from bf16 tiles staged in padded shared memory; P and dS go back into the MMA as
 // bf16, accumulation is fp32.  Outputs are fp32.
 #include <cuda_bf16.h>
