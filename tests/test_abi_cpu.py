@@ -187,3 +187,33 @@ def test_reach_counts_against_the_paper_and_the_oracle(pa, oracle):
         pa.pa_reach_counts(rp, bad, n - 1, 3)
     with pytest.raises(pa.PaError, match="PA_ERR_INVALID_ARG"):
         pa.pa_reach_counts(rp, ci, n, 3)
+
+
+def test_backward_workspace_size_and_validation(pa):
+    """Host side of pa_prefill_backward: the workspace holds a 256-byte status block, delta
+    [batch, Hq, N] fp32 (rounded up to 256 bytes) and the transposed layout (two arrays of nqb + 1 and
+    one of nnz int32), the sum rounded up to 256 bytes; bad arguments fail before any launch."""
+    s = pa.pa_strides(0, 512, 128)
+    good = pa.pa_prefill_params(2, 4, 2, 128, 4100, 64, 0.0, s, s, s, s, pa.PA_BF16)
+    nnz = 777
+    nqb = (4100 + 63) // 64
+    delta = 256 + 2 * 4 * 4100 * 4
+    delta = (delta + 255) // 256 * 256
+    want = (delta + (2 * (nqb + 1) + nnz) * 4 + 255) // 256 * 256
+    assert pa.lib.pa_prefill_backward_workspace_bytes(ctypes.byref(good), nnz) == want
+    bad = pa.pa_prefill_params.from_buffer_copy(good); bad.o_dtype = pa.PA_F32
+    assert pa.lib.pa_prefill_backward_workspace_bytes(ctypes.byref(bad), nnz) == 0
+    buf = (ctypes.c_int32 * 64)()
+    p, null = ctypes.addressof(buf), ctypes.c_void_p(0)
+
+    def status(params, q=p, ws=p, ws_bytes=10**9, n=nnz):
+        return pa.pa_status_string(pa.lib.pa_prefill_backward(ctypes.byref(params), q, p, p, p, p, p, p, p, n, p, p, p,
+                                                              ws, ws_bytes, null))
+
+    assert status(bad) == "PA_ERR_SHAPE"
+    bad = pa.pa_prefill_params.from_buffer_copy(good); bad.head_dim = 32
+    assert status(bad) == "PA_ERR_SHAPE"
+    assert status(good, q=0) == "PA_ERR_INVALID_ARG"
+    assert status(good, q=p + 2) == "PA_ERR_ALIGNMENT"
+    assert status(good, ws_bytes=want - 1) == "PA_ERR_WORKSPACE"
+    assert status(good, n=-5) == "PA_ERR_LAYOUT"
