@@ -403,6 +403,7 @@ static pa_status check_backward(const pa_prefill_params *p, int64_t nnz)
     if (p->head_dim != 64 && p->head_dim != 128) return fail(PA_ERR_SHAPE, "head_dim must be 64 or 128");
     if (p->block != kBwdBlk) return fail(PA_ERR_SHAPE, "block must be 64");
     if (p->n_q_heads % p->n_kv_heads) return fail(PA_ERR_SHAPE, "n_q_heads must be a multiple of n_kv_heads");
+    if (p->n_q_heads < 2) return fail(PA_ERR_SHAPE, "n_q_heads must be >= 2");  // (as in pa_prefill: tiles stack two heads)
     if (p->o_dtype != PA_BF16) return fail(PA_ERR_SHAPE, "the backward pass reads O and dO as bfloat16");
     if (p->seq_len > ((int64_t)1 << 30)) return fail(PA_ERR_SHAPE, "seq_len too large");
     if (p->batch > 65535 || p->n_q_heads > 65535) return fail(PA_ERR_SHAPE, "batch and head counts must be <= 65535");
