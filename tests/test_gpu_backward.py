@@ -171,3 +171,28 @@ def test_backward_on_views_of_a_packed_qkv_tensor(pa, oracle):
     rq, rk, rv = oracle.backward(q.cpu().contiguous(), k.cpu().contiguous(), v.cpu().contiguous(), dO, 64, W, S)
     for g, r, n in ((dq, rq, "dQ"), (dk, rk, "dK"), (dv, rv, "dV")):
         _compare(g, r, n + " packed qkv")
+
+
+def test_backward_on_kv_head_shards_reproduces_the_whole_call(pa):
+    """Head sharding needs no exchange in the backward pass either: dQ belongs to the query heads and
+    dK, dV to the KV heads a rank holds.  The ranks' calls on head slices (run here one after the other
+    on the one GPU) give dQ bit for bit and dK, dV up to the order of their fp32 additions."""
+    from paper_2503_03588_b200.sharding import kv_head_shard, shard_prefill_tensors
+
+    N, Hq, Hkv, D = 3000, 28, 4, 128
+    Q, K, V = (si.bf16_randn((1, N, h, D), 1500 + i).cuda() for i, h in enumerate((Hq, Hkv, Hkv)))
+    dO = si.bf16_randn((1, N, Hq, D), 1504).cuda()
+    rp, ci = pa.pa_build_layout(N, 64, 5, 1)
+    o, lse, ws = pa.pa_prefill(Q, K, V, rp, ci)
+    pa.pa_prefill_status(ws)
+    dq_full, dk_full, dv_full, wsb = pa.pa_prefill_backward(Q, K, V, o, lse, dO, rp, ci)
+    pa.pa_prefill_status(wsb)
+    for world in (2, 4):
+        for rank in range(world):
+            qs_, ks_, vs_, heads = shard_prefill_tensors(Q, K, V, world, rank)
+            _, kv_heads = kv_head_shard(Hq, Hkv, world, rank)
+            dq, dk, dv, wsr = pa.pa_prefill_backward(qs_, ks_, vs_, o[:, :, heads], lse[:, heads].contiguous(), dO[:, :, heads], rp, ci)
+            pa.pa_prefill_status(wsr)
+            assert torch.equal(dq, dq_full[:, :, heads]), (world, rank)
+            assert torch.allclose(dk, dk_full[:, :, kv_heads], rtol=1e-4, atol=1e-5), (world, rank)
+            assert torch.allclose(dv, dv_full[:, :, kv_heads], rtol=1e-4, atol=1e-5), (world, rank)
